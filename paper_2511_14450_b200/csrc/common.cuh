@@ -1,0 +1,116 @@
+// Shared device helpers and the internal kernel-launch interface of libhyperion.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace hyp {
+
+// ---------------------------------------------------------------------------------------------
+// error plumbing
+// ---------------------------------------------------------------------------------------------
+void set_last_cuda_error(int e);
+#define HYP_CUDA_TRY(expr)                         \
+  do {                                             \
+    cudaError_t _e = (expr);                       \
+    if (_e != cudaSuccess) {                       \
+      ::hyp::set_last_cuda_error((int)_e);         \
+      return HYP_ECUDA;                            \
+    }                                              \
+  } while (0)
+
+// ---------------------------------------------------------------------------------------------
+// small device helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+// 128-bit streaming load that does not pollute L1 (weights are read exactly once per step).
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p));
+  return r;
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                               uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// ---------------------------------------------------------------------------------------------
+// per-call batch metadata as the kernels see it (all DEVICE pointers, int32)
+// ---------------------------------------------------------------------------------------------
+struct BatchMeta {
+  int n_seqs;
+  int n_tokens;             // M = sum of q_lens
+  int max_pages_per_seq;    // row stride of block_table
+  const int32_t* q_lens;    // [n_seqs]
+  const int32_t* ctx_lens;  // [n_seqs] cached tokens before this call
+  const int32_t* cu_q;      // [n_seqs+1] first row of each sequence
+  const int32_t* tok_seq;   // [M] batch-local sequence index of each row
+  const int32_t* tok_pos;   // [M] absolute position of each row
+  const int32_t* last_row;  // [n_seqs] row index of each sequence's last new token
+  const int32_t* block_table;  // [n_seqs, max_pages_per_seq] page ids (batch-local rows)
+};
+
+struct ModelDims {
+  int H, Hq, Hkv, D, F, V;
+  int qkv_rows;       // (Hq + 2 Hkv) D
+  int page_tokens;    // 16
+  float eps, theta;
+};
+
+// KV pool of ONE layer: [n_pages][2 (K,V)][Hkv][page_tokens][D] bf16
+__host__ __device__ __forceinline__ size_t kv_page_elems(int Hkv, int page_tokens, int D) {
+  return (size_t)2 * Hkv * page_tokens * D;
+}
+
+// epilogues of the projection kernels
+enum Epilogue : int {
+  EPI_STORE_BF16 = 0,  // out_bf16[m, n] = acc
+  EPI_RESID_F32 = 1,   // out_f32[m, n] += acc         (residual stream)
+  EPI_SWIGLU_BF16 = 2, // out_bf16[m, n] = silu(acc_gate) * acc_up, gate row n, up row n + N
+  EPI_STORE_F32 = 3    // out_f32[m, n] = acc          (logits)
+};
+
+// ---------------------------------------------------------------------------------------------
+// launchers (each enqueues on `st`, returns the number of kernels launched or a negative status)
+// ---------------------------------------------------------------------------------------------
+int launch_embed(const int32_t* ids, const __nv_bfloat16* E, float* x, int M, int H, int V, cudaStream_t st);
+int launch_copy_f32(const float* src, float* dst, size_t n, cudaStream_t st);
+int launch_rmsnorm(const float* x, const __nv_bfloat16* g, __nv_bfloat16* h, int M, int H, float eps,
+                   const int32_t* row_index /* optional gather of rows, may be null */, cudaStream_t st);
+int launch_rope_kv_write(__nv_bfloat16* qkv, __nv_bfloat16* kv_layer, const float2* rope_table,
+                         const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
+// out[m, n] = sum_k a[m, k] * w[n, k] for M <= 32 rows (weight-streaming, HBM-bound)
+int launch_gemm_skinny(const __nv_bfloat16* a, int lda, const __nv_bfloat16* w, int N, int K, int M,
+                       int epi, void* out, int ldo, cudaStream_t st);
+// any M, tensor-core tiles (tcgen05); tensor maps are prepared by the caller
+struct GemmPlan;
+int launch_attn_prefill(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __nv_bfloat16* attn_out,
+                        const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
+// decode attention: one query row per sequence; `scratch` holds split partials
+size_t attn_decode_scratch_bytes(int max_seqs, int Hq, int D, int max_splits);
+int attn_decode_splits(int n_seqs, int Hkv, int max_ctx);
+int launch_attn_decode(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __nv_bfloat16* attn_out,
+                       float* scratch, int n_splits, const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
+
+}  // namespace hyp

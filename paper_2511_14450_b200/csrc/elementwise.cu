@@ -1,0 +1,144 @@
+// Small HBM-trivial kernels of the decoder block: embedding gather, RMSNorm, RoPE + paged KV write.
+#include "common.cuh"
+#include "hyperion.h"
+
+namespace hyp {
+
+// x[t, :] = E[ids[t], :]  (bf16 -> fp32, exact).  Ids outside [0, V) are clamped (the host
+// cannot validate device-resident ids without a sync).
+__global__ void embed_kernel(const int32_t* __restrict__ ids, const __nv_bfloat16* __restrict__ E,
+                             float* __restrict__ x, int H, int V) {
+  const int t = blockIdx.x;
+  int id = ids[t];
+  id = id < 0 ? 0 : (id >= V ? V - 1 : id);
+  const uint4* src = reinterpret_cast<const uint4*>(E + (size_t)id * H);
+  float4* dst = reinterpret_cast<float4*>(x + (size_t)t * H);
+  for (int i = threadIdx.x; i < H / 8; i += blockDim.x) {
+    const uint4 v = src[i];
+    dst[2 * i] = make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
+    dst[2 * i + 1] = make_float4(bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w));
+  }
+}
+
+int launch_embed(const int32_t* ids, const __nv_bfloat16* E, float* x, int M, int H, int V, cudaStream_t st) {
+  embed_kernel<<<M, 128, 0, st>>>(ids, E, x, H, V);
+  return 1;
+}
+
+__global__ void copy_f32_kernel(const float4* __restrict__ src, float4* __restrict__ dst, size_t n4) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = src[i];
+}
+
+int launch_copy_f32(const float* src, float* dst, size_t n, cudaStream_t st) {
+  const size_t n4 = n / 4;  // H is a multiple of 8, so n is a multiple of 4
+  int blocks = (int)((n4 + 255) / 256);
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  if (blocks < 1) blocks = 1;
+  copy_f32_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(src), reinterpret_cast<float4*>(dst), n4);
+  return 1;
+}
+
+// h[r, :] = x[row, :] * rsqrt(mean(x[row, :]^2) + eps) * g, one CTA per output row.
+// row = row_index ? row_index[r] : r.  fp32 statistics, bf16 output.
+template <int THREADS>
+__global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ g,
+                               __nv_bfloat16* __restrict__ h, int H, float eps,
+                               const int32_t* __restrict__ row_index) {
+  __shared__ float red[THREADS / 32];
+  const int r = blockIdx.x;
+  const int row = row_index ? row_index[r] : r;
+  const float4* xr = reinterpret_cast<const float4*>(x + (size_t)row * H);
+  const int n4 = H / 4;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < n4; i += THREADS) {
+    const float4 v = xr[i];
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < THREADS / 32; ++w) tot += red[w];
+  const float rstd = rsqrtf(tot / (float)H + eps);
+  const uint2* gr = reinterpret_cast<const uint2*>(g);
+  uint2* hr = reinterpret_cast<uint2*>(h + (size_t)r * H);
+  for (int i = threadIdx.x; i < n4; i += THREADS) {
+    const float4 v = xr[i];
+    const uint2 gg = gr[i];
+    uint2 o;
+    o.x = pack_bf16(v.x * rstd * bf16_lo(gg.x), v.y * rstd * bf16_hi(gg.x));
+    o.y = pack_bf16(v.z * rstd * bf16_lo(gg.y), v.w * rstd * bf16_hi(gg.y));
+    hr[i] = o;
+  }
+}
+
+int launch_rmsnorm(const float* x, const __nv_bfloat16* g, __nv_bfloat16* h, int M, int H, float eps,
+                   const int32_t* row_index, cudaStream_t st) {
+  rmsnorm_kernel<256><<<M, 256, 0, st>>>(x, g, h, H, eps, row_index);
+  return 1;
+}
+
+// Rotate q and k of every new row by its position and append k, v to the sequence's pages.
+// qkv row layout: [Q heads | K heads | V heads], each head D wide.  q is rotated in place.
+// One thread handles 8 rotation pairs (i .. i+7, i+D/2 .. i+D/2+7) of one head of one row.
+__global__ void rope_kv_write_kernel(__nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ kv_layer,
+                                     const float2* __restrict__ rope_table, BatchMeta bm, ModelDims d) {
+  const int t = blockIdx.x;
+  const int vec_per_head = d.D / 16;
+  const int n_heads = d.Hq + 2 * d.Hkv;
+  const int pos = bm.tok_pos[t];
+  const int sq = bm.tok_seq[t];
+  const int page = bm.block_table[(size_t)sq * bm.max_pages_per_seq + pos / d.page_tokens];
+  const int slot = pos % d.page_tokens;
+  const size_t page_base = (size_t)page * kv_page_elems(d.Hkv, d.page_tokens, d.D);
+  __nv_bfloat16* row = qkv + (size_t)t * d.qkv_rows;
+  for (int w = threadIdx.x; w < n_heads * vec_per_head; w += blockDim.x) {
+    const int head = w / vec_per_head;
+    const int i0 = (w % vec_per_head) * 8;
+    __nv_bfloat16* hp = row + (size_t)head * d.D;
+    const uint4 a = *reinterpret_cast<const uint4*>(hp + i0);
+    const uint4 b = *reinterpret_cast<const uint4*>(hp + d.D / 2 + i0);
+    if (head < d.Hq + d.Hkv) {
+      const float2* cs = rope_table + (size_t)pos * (d.D / 2) + i0;
+      const uint32_t av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+      uint32_t oa[4], ob[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 c0 = cs[2 * j], c1 = cs[2 * j + 1];
+        const float x1a = bf16_lo(av[j]), x1b = bf16_hi(av[j]);
+        const float x2a = bf16_lo(bv[j]), x2b = bf16_hi(bv[j]);
+        oa[j] = pack_bf16(x1a * c0.x - x2a * c0.y, x1b * c1.x - x2b * c1.y);
+        ob[j] = pack_bf16(x2a * c0.x + x1a * c0.y, x2b * c1.x + x1b * c1.y);
+      }
+      const uint4 ra = make_uint4(oa[0], oa[1], oa[2], oa[3]), rb = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+      if (head < d.Hq) {
+        *reinterpret_cast<uint4*>(hp + i0) = ra;
+        *reinterpret_cast<uint4*>(hp + d.D / 2 + i0) = rb;
+      } else {
+        const int kvh = head - d.Hq;
+        __nv_bfloat16* dst = kv_layer + page_base + ((size_t)kvh * d.page_tokens + slot) * d.D;
+        *reinterpret_cast<uint4*>(dst + i0) = ra;
+        *reinterpret_cast<uint4*>(dst + d.D / 2 + i0) = rb;
+      }
+    } else {
+      const int kvh = head - d.Hq - d.Hkv;
+      __nv_bfloat16* dst = kv_layer + page_base + (size_t)d.Hkv * d.page_tokens * d.D +
+                           ((size_t)kvh * d.page_tokens + slot) * d.D;
+      *reinterpret_cast<uint4*>(dst + i0) = a;
+      *reinterpret_cast<uint4*>(dst + d.D / 2 + i0) = b;
+    }
+  }
+}
+
+int launch_rope_kv_write(__nv_bfloat16* qkv, __nv_bfloat16* kv_layer, const float2* rope_table,
+                         const BatchMeta& bm, const ModelDims& d, cudaStream_t st) {
+  const int work = (d.Hq + 2 * d.Hkv) * (d.D / 16);
+  int threads = ((work + 31) / 32) * 32;
+  if (threads > 512) threads = 512;
+  rope_kv_write_kernel<<<bm.n_tokens, threads, 0, st>>>(qkv, kv_layer, rope_table, bm, d);
+  return 1;
+}
+
+}  // namespace hyp

@@ -1,0 +1,26 @@
+// Tensor-core projection for any row count (prefill): operand descriptors and launcher.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace hyp {
+
+// A bf16 matrix [rows, K] row-major together with the TMA descriptor that tiles it.
+struct TcOperand {
+  CUtensorMap map;
+  const __nv_bfloat16* ptr = nullptr;
+  int rows = 0, K = 0;
+  int box_rows = 0;
+};
+typedef TcOperand TcWeight;
+typedef TcOperand TcAct;
+
+int tc_make_weight(TcWeight* w, const __nv_bfloat16* ptr, int rows, int K);
+int tc_make_act(TcAct* a, const __nv_bfloat16* ptr, int rows, int K);
+
+// out[m, n] (+)= sum_k act[m, k] * w[n, k] for m < M, n < N (SwiGLU: w holds 2N rows).
+int launch_gemm_tc(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
+                   cudaStream_t st);
+
+}  // namespace hyp

@@ -1,0 +1,610 @@
+// Stage runtime: owns weights, the paged KV pool, block tables (host side) and workspace, and
+// drives the per-block kernel sequence for prefill and decode.
+#include <algorithm>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "gemm_tc.cuh"
+#include "hyperion.h"
+
+namespace hyp {
+static thread_local int g_last_cuda_error = 0;
+void set_last_cuda_error(int e) { g_last_cuda_error = e; }
+}  // namespace hyp
+
+using namespace hyp;
+typedef __nv_bfloat16 bf16;
+
+namespace {
+
+constexpr int META_RING = 4;
+
+struct LayerW {
+  bf16 *wqkv = nullptr, *wo = nullptr, *wgu = nullptr, *wd = nullptr, *g1 = nullptr, *g2 = nullptr;
+  uint32_t loaded = 0;
+  TcWeight tc_qkv, tc_o, tc_gu, tc_d;
+};
+
+}  // namespace
+
+struct hyp_stage {
+  hyp_cfg cfg;
+  int lo = 0, hi = 0, L = 0, device = 0;
+  bool first = false, last = false;
+  ModelDims dims;
+  std::vector<LayerW> layers;
+  bf16 *embed = nullptr, *gf = nullptr, *wlm = nullptr;
+  TcWeight tc_lm;
+  uint32_t loaded_extra = 0;
+  // KV cache
+  bf16* kv_pool = nullptr;
+  size_t kv_layer_elems = 0;
+  int n_pages = 0, max_pages_per_seq = 0;
+  std::vector<int32_t> free_pages;
+  std::vector<std::vector<int32_t>> seq_pages;
+  std::vector<int32_t> seq_len;
+  // workspace
+  int max_rows = 0;
+  float* x = nullptr;
+  bf16 *h = nullptr, *qkv = nullptr, *attn = nullptr, *u = nullptr;
+  TcAct tc_h, tc_attn, tc_u;
+  float* attn_scratch = nullptr;
+  int max_splits = 32;
+  float2* rope_table = nullptr;
+  size_t workspace_bytes = 0;
+  // metadata staging
+  size_t meta_ints = 0;
+  int32_t* meta_dev = nullptr;
+  int32_t* meta_host[META_RING] = {nullptr, nullptr, nullptr, nullptr};
+  cudaEvent_t meta_ev[META_RING] = {nullptr, nullptr, nullptr, nullptr};
+  bool meta_used[META_RING] = {false, false, false, false};
+  int ring_pos = 0;
+  // staging for the *_host entry points
+  void *io_in = nullptr, *io_out = nullptr;
+  size_t io_in_bytes = 0, io_out_bytes = 0;
+  int64_t launches = 0;
+};
+
+namespace {
+
+template <typename T>
+int dev_alloc(T** p, size_t count) {
+  if (count == 0) count = 1;
+  cudaError_t e = cudaMalloc((void**)p, count * sizeof(T));
+  if (e != cudaSuccess) {
+    set_last_cuda_error((int)e);
+    *p = nullptr;
+    return e == cudaErrorMemoryAllocation ? HYP_ENOMEM : HYP_ECUDA;
+  }
+  return HYP_OK;
+}
+
+size_t tensor_elems(const hyp_stage* s, int tensor_id) {
+  const ModelDims& d = s->dims;
+  switch (tensor_id) {
+    case HYP_W_QKV: return (size_t)d.qkv_rows * d.H;
+    case HYP_W_O: return (size_t)d.H * d.Hq * d.D;
+    case HYP_W_GATE_UP: return (size_t)2 * d.F * d.H;
+    case HYP_W_DOWN: return (size_t)d.H * d.F;
+    case HYP_W_NORM1:
+    case HYP_W_NORM2:
+    case HYP_W_FINAL_NORM: return (size_t)d.H;
+    case HYP_W_EMBED:
+    case HYP_W_LM_HEAD: return (size_t)d.V * d.H;
+    default: return 0;
+  }
+}
+
+struct HostBatch {
+  int n = 0, M = 0;
+  std::vector<int32_t> packed;  // q_lens | ctx_lens | cu_q | last_row | tok_seq | tok_pos | block_table
+  size_t off_q, off_ctx, off_cu, off_last, off_tseq, off_tpos, off_bt;
+};
+
+void layout_meta(HostBatch& hb, int n, int M, int mpps) {
+  hb.n = n;
+  hb.M = M;
+  hb.off_q = 0;
+  hb.off_ctx = hb.off_q + n;
+  hb.off_cu = hb.off_ctx + n;
+  hb.off_last = hb.off_cu + n + 1;
+  hb.off_tseq = hb.off_last + n;
+  hb.off_tpos = hb.off_tseq + M;
+  hb.off_bt = hb.off_tpos + M;
+  hb.packed.assign(hb.off_bt + (size_t)n * mpps, 0);
+}
+
+BatchMeta device_meta(const hyp_stage* s, const HostBatch& hb) {
+  BatchMeta bm;
+  bm.n_seqs = hb.n;
+  bm.n_tokens = hb.M;
+  bm.max_pages_per_seq = s->max_pages_per_seq;
+  bm.q_lens = s->meta_dev + hb.off_q;
+  bm.ctx_lens = s->meta_dev + hb.off_ctx;
+  bm.cu_q = s->meta_dev + hb.off_cu;
+  bm.last_row = s->meta_dev + hb.off_last;
+  bm.tok_seq = s->meta_dev + hb.off_tseq;
+  bm.tok_pos = s->meta_dev + hb.off_tpos;
+  bm.block_table = s->meta_dev + hb.off_bt;
+  return bm;
+}
+
+int upload_meta(hyp_stage* s, const HostBatch& hb, cudaStream_t st) {
+  const int slot = s->ring_pos;
+  s->ring_pos = (s->ring_pos + 1) % META_RING;
+  if (s->meta_used[slot]) HYP_CUDA_TRY(cudaEventSynchronize(s->meta_ev[slot]));
+  std::memcpy(s->meta_host[slot], hb.packed.data(), hb.packed.size() * sizeof(int32_t));
+  HYP_CUDA_TRY(cudaMemcpyAsync(s->meta_dev, s->meta_host[slot], hb.packed.size() * sizeof(int32_t),
+                               cudaMemcpyHostToDevice, st));
+  HYP_CUDA_TRY(cudaEventRecord(s->meta_ev[slot], st));
+  s->meta_used[slot] = true;
+  return HYP_OK;
+}
+
+// Validate a batch against the stage's tables and reserve the pages it needs.  Nothing is
+// changed unless everything fits.
+int admit_batch(hyp_stage* s, const hyp_batch* b, bool decode, HostBatch& hb) {
+  if (!b || b->n_seqs < 1 || !b->seq_ids || !b->q_lens || !b->ctx_lens) return HYP_EINVAL;
+  if (b->flags & ~HYP_BATCH_ALL_LOGITS) return HYP_EINVAL;
+  const int n = b->n_seqs;
+  if (n > s->cfg.max_seqs) return HYP_ECAPACITY;
+  if (decode && n > HYP_MAX_DECODE_BATCH) return HYP_EINVAL;
+  const int PT = s->cfg.kv_block_size;
+  long M = 0;
+  size_t need_pages = 0;
+  std::vector<uint8_t> seen(s->cfg.max_seqs, 0);
+  for (int i = 0; i < n; ++i) {
+    const int id = b->seq_ids[i];
+    if (id < 0 || id >= s->cfg.max_seqs || seen[id]) return HYP_EINVAL;
+    seen[id] = 1;
+    if (b->q_lens[i] < 1 || (decode && b->q_lens[i] != 1)) return HYP_EINVAL;
+    if (b->ctx_lens[i] != s->seq_len[id]) return HYP_EINVAL;
+    const long total = (long)b->ctx_lens[i] + b->q_lens[i];
+    if (total > s->cfg.max_ctx) return HYP_ECAPACITY;
+    M += b->q_lens[i];
+    need_pages += (size_t)((total + PT - 1) / PT) - s->seq_pages[id].size();
+  }
+  if (M > s->max_rows || (!decode && M > s->cfg.max_tokens)) return HYP_ECAPACITY;
+  if (need_pages > s->free_pages.size()) return HYP_ECAPACITY;
+
+  layout_meta(hb, n, (int)M, s->max_pages_per_seq);
+  int32_t* p = hb.packed.data();
+  int row = 0;
+  for (int i = 0; i < n; ++i) {
+    const int id = b->seq_ids[i];
+    const int total = b->ctx_lens[i] + b->q_lens[i];
+    auto& pages = s->seq_pages[id];
+    while ((int)pages.size() < (total + PT - 1) / PT) {
+      pages.push_back(s->free_pages.back());
+      s->free_pages.pop_back();
+    }
+    s->seq_len[id] = total;
+    p[hb.off_q + i] = b->q_lens[i];
+    p[hb.off_ctx + i] = b->ctx_lens[i];
+    p[hb.off_cu + i] = row;
+    for (int t = 0; t < b->q_lens[i]; ++t) {
+      p[hb.off_tseq + row] = i;
+      p[hb.off_tpos + row] = b->ctx_lens[i] + t;
+      ++row;
+    }
+    p[hb.off_last + i] = row - 1;
+    std::copy(pages.begin(), pages.end(), p + hb.off_bt + (size_t)i * s->max_pages_per_seq);
+  }
+  p[hb.off_cu + n] = row;
+  return HYP_OK;
+}
+
+int check_ready(const hyp_stage* s) {
+  for (const LayerW& lw : s->layers)
+    if (lw.loaded != 0x3f) return HYP_ESTATE;
+  uint32_t want = 0;
+  if (s->first) want |= 1u << HYP_W_EMBED;
+  if (s->last) want |= (1u << HYP_W_FINAL_NORM) | (1u << HYP_W_LM_HEAD);
+  if ((s->loaded_extra & want) != want) return HYP_ESTATE;
+  return HYP_OK;
+}
+
+#define HYP_LAUNCH(call)                                   \
+  do {                                                     \
+    int _n = (call);                                       \
+    if (_n < 0) return _n;                                 \
+    s->launches += _n;                                     \
+  } while (0)
+
+// out[m, n] (+)= a[m, :] . w[n, :] with the kernel family chosen by the row count.
+int project(hyp_stage* s, const TcAct& act, const bf16* a, int lda, const TcWeight& tw, const bf16* w, int N, int K,
+            int M, int epi, void* out, int ldo, cudaStream_t st) {
+  if (M <= 32) return launch_gemm_skinny(a, lda, w, N, K, M, epi, out, ldo, st);
+  return launch_gemm_tc(act, tw, M, N, K, epi, out, ldo, st);
+}
+
+// The block sequence B_lo -> ... -> B_{hi-1} on rows already resident in s->x.
+// If `marks` is non-null an event is recorded before the first block and after every block.
+int run_blocks(hyp_stage* s, const BatchMeta& bm, bool decode, int n_splits, cudaStream_t st, cudaEvent_t* marks) {
+  const ModelDims& d = s->dims;
+  const int M = bm.n_tokens;
+  if (marks) HYP_CUDA_TRY(cudaEventRecord(marks[0], st));
+  for (int li = 0; li < s->L; ++li) {
+    LayerW& lw = s->layers[li];
+    bf16* kv_layer = s->kv_pool + (size_t)li * s->kv_layer_elems;
+    HYP_LAUNCH(launch_rmsnorm(s->x, lw.g1, s->h, M, d.H, d.eps, nullptr, st));
+    HYP_LAUNCH(project(s, s->tc_h, s->h, d.H, lw.tc_qkv, lw.wqkv, d.qkv_rows, d.H, M, EPI_STORE_BF16, s->qkv,
+                       d.qkv_rows, st));
+    HYP_LAUNCH(launch_rope_kv_write(s->qkv, kv_layer, s->rope_table, bm, d, st));
+    if (decode)
+      HYP_LAUNCH(launch_attn_decode(s->qkv, kv_layer, s->attn, s->attn_scratch, n_splits, bm, d, st));
+    else
+      HYP_LAUNCH(launch_attn_prefill(s->qkv, kv_layer, s->attn, bm, d, st));
+    HYP_LAUNCH(project(s, s->tc_attn, s->attn, d.Hq * d.D, lw.tc_o, lw.wo, d.H, d.Hq * d.D, M, EPI_RESID_F32, s->x,
+                       d.H, st));
+    HYP_LAUNCH(launch_rmsnorm(s->x, lw.g2, s->h, M, d.H, d.eps, nullptr, st));
+    HYP_LAUNCH(project(s, s->tc_h, s->h, d.H, lw.tc_gu, lw.wgu, d.F, d.H, M, EPI_SWIGLU_BF16, s->u, d.F, st));
+    HYP_LAUNCH(project(s, s->tc_u, s->u, d.F, lw.tc_d, lw.wd, d.H, d.F, M, EPI_RESID_F32, s->x, d.H, st));
+    if (marks) HYP_CUDA_TRY(cudaEventRecord(marks[li + 1], st));
+  }
+  return HYP_OK;
+}
+
+int run_stage(hyp_stage* s, const hyp_batch* b, const void* in, void* out, cudaStream_t st, bool decode) {
+  if (!s || !in || !out) return HYP_EINVAL;
+  int rc = check_ready(s);
+  if (rc) return rc;
+  HostBatch hb;
+  rc = admit_batch(s, b, decode, hb);
+  if (rc) return rc;
+  rc = upload_meta(s, hb, st);
+  if (rc) return rc;
+  const BatchMeta bm = device_meta(s, hb);
+  const ModelDims& d = s->dims;
+  const int M = hb.M;
+
+  if (s->first)
+    HYP_LAUNCH(launch_embed((const int32_t*)in, s->embed, s->x, M, d.H, d.V, st));
+  else
+    HYP_LAUNCH(launch_copy_f32((const float*)in, s->x, (size_t)M * d.H, st));
+
+  int n_splits = 1;
+  if (decode) {
+    int max_ctx = 1;
+    for (int i = 0; i < hb.n; ++i) max_ctx = std::max(max_ctx, b->ctx_lens[i] + 1);
+    n_splits = std::min(s->max_splits, attn_decode_splits(hb.n, d.Hkv, max_ctx));
+  }
+  rc = run_blocks(s, bm, decode, n_splits, st, nullptr);
+  if (rc) return rc;
+
+  if (s->last) {
+    const bool all = (b->flags & HYP_BATCH_ALL_LOGITS) != 0 || decode;
+    const int rows = all ? M : hb.n;
+    HYP_LAUNCH(launch_rmsnorm(s->x, s->gf, s->h, rows, d.H, d.eps, all ? nullptr : bm.last_row, st));
+    HYP_LAUNCH(project(s, s->tc_h, s->h, d.H, s->tc_lm, s->wlm, d.V, d.H, rows, EPI_STORE_F32, out, d.V, st));
+  } else {
+    HYP_LAUNCH(launch_copy_f32(s->x, (float*)out, (size_t)M * d.H, st));
+  }
+  cudaError_t e = cudaPeekAtLastError();
+  if (e != cudaSuccess) {
+    set_last_cuda_error((int)e);
+    return HYP_ECUDA;
+  }
+  return HYP_OK;
+}
+
+int run_stage_host(hyp_stage* s, const hyp_batch* b, const void* in, void* out, cudaStream_t st, bool decode) {
+  if (!s || !b || !in || !out || b->n_seqs < 1 || !b->q_lens) return HYP_EINVAL;
+  long M = 0;
+  for (int i = 0; i < b->n_seqs; ++i) {
+    if (b->q_lens[i] < 1) return HYP_EINVAL;
+    M += b->q_lens[i];
+  }
+  const ModelDims& d = s->dims;
+  const size_t in_bytes = s->first ? (size_t)M * sizeof(int32_t) : (size_t)M * d.H * sizeof(float);
+  const bool all = (b->flags & HYP_BATCH_ALL_LOGITS) != 0 || decode;
+  const size_t out_bytes =
+      s->last ? (size_t)(all ? M : b->n_seqs) * d.V * sizeof(float) : (size_t)M * d.H * sizeof(float);
+  if (in_bytes > s->io_in_bytes || out_bytes > s->io_out_bytes) return HYP_ECAPACITY;
+  // validate before the first copy so that a rejected call moves no data
+  {
+    HostBatch probe;
+    std::vector<int32_t> lens(s->seq_len);
+    std::vector<std::vector<int32_t>> pages(s->seq_pages);
+    std::vector<int32_t> freep(s->free_pages);
+    int rc = check_ready(s);
+    if (!rc) rc = admit_batch(s, b, decode, probe);
+    s->seq_len.swap(lens);
+    s->seq_pages.swap(pages);
+    s->free_pages.swap(freep);
+    if (rc) return rc;
+  }
+  HYP_CUDA_TRY(cudaMemcpyAsync(s->io_in, in, in_bytes, cudaMemcpyHostToDevice, st));
+  int rc = run_stage(s, b, s->io_in, s->io_out, st, decode);
+  if (rc) return rc;
+  HYP_CUDA_TRY(cudaMemcpyAsync(out, s->io_out, out_bytes, cudaMemcpyDeviceToHost, st));
+  HYP_CUDA_TRY(cudaStreamSynchronize(st));
+  return HYP_OK;
+}
+
+__global__ void fill_pattern_kernel(float* x, size_t n) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const uint32_t hsh = (uint32_t)i * 2654435761u;
+    x[i] = ((float)((hsh >> 8) & 0xffff) / 65536.0f - 0.5f) * 0.1f;
+  }
+}
+
+}  // namespace
+
+// -------------------------------------------------------------------------------------------------
+// C ABI
+// -------------------------------------------------------------------------------------------------
+extern "C" int hyp_last_cuda_error(void) { return hyp::g_last_cuda_error; }
+
+extern "C" const char* hyp_strerror(int code) {
+  switch (code) {
+    case HYP_OK: return "ok";
+    case HYP_EINVAL: return "invalid argument";
+    case HYP_ENOMEM: return "out of memory";
+    case HYP_ECAPACITY: return "capacity exceeded (KV pages, context, batch or token workspace)";
+    case HYP_EINFEASIBLE: return "no feasible solution";
+    case HYP_ECUDA: return "CUDA error (see hyp_last_cuda_error)";
+    case HYP_ESTATE: return "stage not ready: a weight tensor has not been loaded";
+    default: return "unknown status";
+  }
+}
+
+extern "C" void hyp_stage_destroy(hyp_stage* s) {
+  if (!s) return;
+  for (LayerW& lw : s->layers) {
+    cudaFree(lw.wqkv); cudaFree(lw.wo); cudaFree(lw.wgu); cudaFree(lw.wd); cudaFree(lw.g1); cudaFree(lw.g2);
+  }
+  cudaFree(s->embed); cudaFree(s->gf); cudaFree(s->wlm); cudaFree(s->kv_pool);
+  cudaFree(s->x); cudaFree(s->h); cudaFree(s->qkv); cudaFree(s->attn); cudaFree(s->u);
+  cudaFree(s->attn_scratch); cudaFree(s->rope_table); cudaFree(s->meta_dev);
+  cudaFree(s->io_in); cudaFree(s->io_out);
+  for (int i = 0; i < META_RING; ++i) {
+    if (s->meta_host[i]) cudaFreeHost(s->meta_host[i]);
+    if (s->meta_ev[i]) cudaEventDestroy(s->meta_ev[i]);
+  }
+  delete s;
+}
+
+extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cfg* cfg, hyp_stage** out) {
+  if (!cfg || !out) return HYP_EINVAL;
+  const hyp_cfg& c = *cfg;
+  if (c.n_layers_total < 1 || layer_lo < 0 || layer_hi <= layer_lo || layer_hi > c.n_layers_total) return HYP_EINVAL;
+  if (c.hidden < 8 || c.hidden % 8 || c.ffn < 8 || c.ffn % 8 || c.vocab < 1) return HYP_EINVAL;
+  if (c.n_kv_heads < 1 || c.n_q_heads < c.n_kv_heads || c.n_q_heads % c.n_kv_heads) return HYP_EINVAL;
+  const int G = c.n_q_heads / c.n_kv_heads;
+  if (!(G == 1 || G == 2 || G == 4 || G == 8)) return HYP_EINVAL;
+  if (!(c.head_dim == 64 || c.head_dim == 128)) return HYP_EINVAL;
+  if (c.kv_block_size != 16) return HYP_EINVAL;
+  if (c.max_seqs < 1 || c.max_ctx < 1 || c.max_tokens < 1 || c.kv_pages < 0) return HYP_EINVAL;
+  if (!(c.rms_eps > 0.f) || !(c.rope_theta > 1.f)) return HYP_EINVAL;
+
+  hyp_stage* s = new (std::nothrow) hyp_stage();
+  if (!s) return HYP_ENOMEM;
+  s->cfg = c;
+  s->lo = layer_lo; s->hi = layer_hi; s->L = layer_hi - layer_lo;
+  s->first = layer_lo == 0;
+  s->last = layer_hi == c.n_layers_total;
+  ModelDims& d = s->dims;
+  d.H = c.hidden; d.Hq = c.n_q_heads; d.Hkv = c.n_kv_heads; d.D = c.head_dim; d.F = c.ffn; d.V = c.vocab;
+  d.qkv_rows = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+  d.page_tokens = c.kv_block_size; d.eps = c.rms_eps; d.theta = c.rope_theta;
+
+  int rc = HYP_OK;
+#define TRY(expr) do { rc = (expr); if (rc) { hyp_stage_destroy(s); return rc; } } while (0)
+#define TRY_CUDA(expr) do { cudaError_t _e = (expr); if (_e != cudaSuccess) { set_last_cuda_error((int)_e); \
+    hyp_stage_destroy(s); return _e == cudaErrorMemoryAllocation ? HYP_ENOMEM : HYP_ECUDA; } } while (0)
+  TRY_CUDA(cudaGetDevice(&s->device));
+  s->layers.resize(s->L);
+  for (LayerW& lw : s->layers) {
+    TRY(dev_alloc(&lw.wqkv, tensor_elems(s, HYP_W_QKV)));
+    TRY(dev_alloc(&lw.wo, tensor_elems(s, HYP_W_O)));
+    TRY(dev_alloc(&lw.wgu, tensor_elems(s, HYP_W_GATE_UP)));
+    TRY(dev_alloc(&lw.wd, tensor_elems(s, HYP_W_DOWN)));
+    TRY(dev_alloc(&lw.g1, (size_t)d.H));
+    TRY(dev_alloc(&lw.g2, (size_t)d.H));
+  }
+  if (s->first) TRY(dev_alloc(&s->embed, tensor_elems(s, HYP_W_EMBED)));
+  if (s->last) {
+    TRY(dev_alloc(&s->gf, (size_t)d.H));
+    TRY(dev_alloc(&s->wlm, tensor_elems(s, HYP_W_LM_HEAD)));
+  }
+  // KV pool: [layer][page][K,V][Hkv][16][D]
+  s->max_pages_per_seq = (c.max_ctx + c.kv_block_size - 1) / c.kv_block_size;
+  s->n_pages = c.kv_pages > 0 ? c.kv_pages : c.max_seqs * s->max_pages_per_seq;
+  s->kv_layer_elems = (size_t)s->n_pages * kv_page_elems(d.Hkv, d.page_tokens, d.D);
+  TRY(dev_alloc(&s->kv_pool, s->kv_layer_elems * s->L));
+  TRY_CUDA(cudaMemset(s->kv_pool, 0, s->kv_layer_elems * s->L * sizeof(bf16)));
+  s->free_pages.resize(s->n_pages);
+  for (int i = 0; i < s->n_pages; ++i) s->free_pages[i] = s->n_pages - 1 - i;
+  s->seq_pages.assign(c.max_seqs, {});
+  s->seq_len.assign(c.max_seqs, 0);
+  // workspace (row capacity covers a full prefill call or a full decode batch; rows are padded to
+  // the GEMM tile height so that tile loads never leave the allocation)
+  s->max_rows = std::max(c.max_tokens, std::min(c.max_seqs, HYP_MAX_DECODE_BATCH));
+  const size_t rows_pad = ((size_t)s->max_rows + 127) / 128 * 128;
+  TRY(dev_alloc(&s->x, rows_pad * d.H));
+  TRY(dev_alloc(&s->h, rows_pad * d.H));
+  TRY(dev_alloc(&s->qkv, rows_pad * d.qkv_rows));
+  TRY(dev_alloc(&s->attn, rows_pad * d.Hq * d.D));
+  TRY(dev_alloc(&s->u, rows_pad * d.F));
+  TRY_CUDA(cudaMemset(s->h, 0, rows_pad * d.H * sizeof(bf16)));
+  TRY_CUDA(cudaMemset(s->attn, 0, rows_pad * d.Hq * d.D * sizeof(bf16)));
+  TRY_CUDA(cudaMemset(s->u, 0, rows_pad * d.F * sizeof(bf16)));
+  const size_t scratch_bytes =
+      attn_decode_scratch_bytes(std::min(c.max_seqs, HYP_MAX_DECODE_BATCH), d.Hq, d.D, s->max_splits);
+  TRY(dev_alloc(&s->attn_scratch, scratch_bytes / sizeof(float)));
+  s->workspace_bytes = rows_pad * ((size_t)d.H * 6 + ((size_t)d.qkv_rows + d.Hq * d.D + d.F) * 2) + scratch_bytes;
+  // rotary table: cos/sin of pos * theta^(-2i/D), angles evaluated in double on the host
+  {
+    const int half = d.D / 2;
+    std::vector<float2> tab((size_t)c.max_ctx * half);
+    for (int p = 0; p < c.max_ctx; ++p)
+      for (int i = 0; i < half; ++i) {
+        const double ang = (double)p * std::pow((double)c.rope_theta, -2.0 * i / d.D);
+        tab[(size_t)p * half + i] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+      }
+    TRY(dev_alloc(&s->rope_table, tab.size()));
+    TRY_CUDA(cudaMemcpy(s->rope_table, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice));
+  }
+  // metadata staging
+  s->meta_ints = (size_t)4 * c.max_seqs + 1 + (size_t)2 * s->max_rows + (size_t)c.max_seqs * s->max_pages_per_seq;
+  TRY(dev_alloc(&s->meta_dev, s->meta_ints));
+  for (int i = 0; i < META_RING; ++i) {
+    TRY_CUDA(cudaMallocHost((void**)&s->meta_host[i], s->meta_ints * sizeof(int32_t)));
+    TRY_CUDA(cudaEventCreateWithFlags(&s->meta_ev[i], cudaEventDisableTiming));
+  }
+  // staging for host-buffer calls
+  s->io_in_bytes = (size_t)s->max_rows * (s->first ? sizeof(int32_t) : d.H * sizeof(float));
+  s->io_out_bytes = s->last ? (size_t)std::max(c.max_seqs, std::min(s->max_rows, 64)) * d.V * sizeof(float)
+                            : (size_t)s->max_rows * d.H * sizeof(float);
+  TRY_CUDA(cudaMalloc(&s->io_in, s->io_in_bytes));
+  TRY_CUDA(cudaMalloc(&s->io_out, s->io_out_bytes));
+  // tensor-core operand descriptors over the fixed workspace buffers
+  TRY(tc_make_act(&s->tc_h, s->h, (int)rows_pad, d.H));
+  TRY(tc_make_act(&s->tc_attn, s->attn, (int)rows_pad, d.Hq * d.D));
+  TRY(tc_make_act(&s->tc_u, s->u, (int)rows_pad, d.F));
+  for (LayerW& lw : s->layers) {
+    TRY(tc_make_weight(&lw.tc_qkv, lw.wqkv, d.qkv_rows, d.H));
+    TRY(tc_make_weight(&lw.tc_o, lw.wo, d.H, d.Hq * d.D));
+    TRY(tc_make_weight(&lw.tc_gu, lw.wgu, 2 * d.F, d.H));
+    TRY(tc_make_weight(&lw.tc_d, lw.wd, d.H, d.F));
+  }
+  if (s->last) TRY(tc_make_weight(&s->tc_lm, s->wlm, d.V, d.H));
+#undef TRY
+#undef TRY_CUDA
+  *out = s;
+  return HYP_OK;
+}
+
+extern "C" int hyp_stage_load(hyp_stage* s, int32_t layer, int32_t tensor_id, const void* src, size_t bytes,
+                              void* stream) {
+  if (!s || !src) return HYP_EINVAL;
+  void* dst = nullptr;
+  uint32_t* mask = nullptr;
+  if (tensor_id >= HYP_W_QKV && tensor_id <= HYP_W_NORM2) {
+    if (layer < s->lo || layer >= s->hi) return HYP_EINVAL;
+    LayerW& lw = s->layers[layer - s->lo];
+    bf16* ptrs[6] = {lw.wqkv, lw.wo, lw.wgu, lw.wd, lw.g1, lw.g2};
+    dst = ptrs[tensor_id];
+    mask = &lw.loaded;
+  } else if (tensor_id == HYP_W_EMBED) {
+    if (!s->first || layer != -1) return HYP_EINVAL;
+    dst = s->embed;
+    mask = &s->loaded_extra;
+  } else if (tensor_id == HYP_W_FINAL_NORM || tensor_id == HYP_W_LM_HEAD) {
+    if (!s->last || layer != s->cfg.n_layers_total) return HYP_EINVAL;
+    dst = tensor_id == HYP_W_FINAL_NORM ? (void*)s->gf : (void*)s->wlm;
+    mask = &s->loaded_extra;
+  } else {
+    return HYP_EINVAL;
+  }
+  if (bytes != tensor_elems(s, tensor_id) * sizeof(bf16)) return HYP_EINVAL;
+  HYP_CUDA_TRY(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  *mask |= 1u << tensor_id;
+  return HYP_OK;
+}
+
+extern "C" int hyp_stage_prefill(hyp_stage* s, const hyp_batch* b, const void* in, void* out, void* stream) {
+  return run_stage(s, b, in, out, (cudaStream_t)stream, false);
+}
+extern "C" int hyp_stage_decode(hyp_stage* s, const hyp_batch* b, const void* in, void* out, void* stream) {
+  return run_stage(s, b, in, out, (cudaStream_t)stream, true);
+}
+extern "C" int hyp_stage_prefill_host(hyp_stage* s, const hyp_batch* b, const void* in, void* out, void* stream) {
+  return run_stage_host(s, b, in, out, (cudaStream_t)stream, false);
+}
+extern "C" int hyp_stage_decode_host(hyp_stage* s, const hyp_batch* b, const void* in, void* out, void* stream) {
+  return run_stage_host(s, b, in, out, (cudaStream_t)stream, true);
+}
+
+extern "C" int hyp_stage_free_seq(hyp_stage* s, int32_t seq_id) {
+  if (!s || seq_id < 0 || seq_id >= s->cfg.max_seqs) return HYP_EINVAL;
+  auto& pages = s->seq_pages[seq_id];
+  for (auto it = pages.rbegin(); it != pages.rend(); ++it) s->free_pages.push_back(*it);
+  pages.clear();
+  s->seq_len[seq_id] = 0;
+  return HYP_OK;
+}
+
+extern "C" int hyp_stage_seq_len(const hyp_stage* s, int32_t seq_id) {
+  if (!s || seq_id < 0 || seq_id >= s->cfg.max_seqs) return HYP_EINVAL;
+  return s->seq_len[seq_id];
+}
+
+extern "C" int hyp_stage_free_pages(const hyp_stage* s) {
+  if (!s) return HYP_EINVAL;
+  return (int)s->free_pages.size();
+}
+
+extern "C" int64_t hyp_stage_launch_count(const hyp_stage* s) { return s ? s->launches : 0; }
+
+extern "C" int hyp_stage_profile(hyp_stage* s, int32_t mode, int32_t batch, int32_t ctx, int32_t iters,
+                                 float* layer_ms, size_t* layer_bytes, void* stream) {
+  if (!s || !layer_ms || !layer_bytes || (mode != 0 && mode != 1) || batch < 1 || ctx < 1 || iters < 1)
+    return HYP_EINVAL;
+  int rc = check_ready(s);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  const bool decode = mode == 1;
+  const int PT = s->cfg.kv_block_size;
+  const int total = decode ? ctx + 1 : ctx;
+  const long M = decode ? batch : (long)batch * ctx;
+  if (batch > s->cfg.max_seqs || total > s->cfg.max_ctx || M > s->max_rows) return HYP_ECAPACITY;
+  if (decode && batch > HYP_MAX_DECODE_BATCH) return HYP_EINVAL;
+  const int pages_per = (total + PT - 1) / PT;
+  if ((size_t)batch * pages_per > s->free_pages.size()) return HYP_ECAPACITY;
+
+  // scratch sequences on pages borrowed from the free list (not removed: nothing persists)
+  HostBatch hb;
+  layout_meta(hb, batch, (int)M, s->max_pages_per_seq);
+  int32_t* p = hb.packed.data();
+  int row = 0;
+  for (int i = 0; i < batch; ++i) {
+    const int ql = decode ? 1 : ctx, cl = decode ? ctx : 0;
+    p[hb.off_q + i] = ql;
+    p[hb.off_ctx + i] = cl;
+    p[hb.off_cu + i] = row;
+    for (int t = 0; t < ql; ++t) {
+      p[hb.off_tseq + row] = i;
+      p[hb.off_tpos + row] = cl + t;
+      ++row;
+    }
+    p[hb.off_last + i] = row - 1;
+    for (int k = 0; k < pages_per; ++k)
+      p[hb.off_bt + (size_t)i * s->max_pages_per_seq + k] = s->free_pages[s->free_pages.size() - 1 - (i * pages_per + k)];
+  }
+  p[hb.off_cu + batch] = row;
+  rc = upload_meta(s, hb, st);
+  if (rc) return rc;
+  const BatchMeta bm = device_meta(s, hb);
+  const int n_splits = decode ? std::min(s->max_splits, attn_decode_splits(batch, s->dims.Hkv, total)) : 1;
+
+  std::vector<cudaEvent_t> ev((size_t)(s->L + 1) * iters, nullptr);
+  for (auto& e : ev) HYP_CUDA_TRY(cudaEventCreate(&e));
+  rc = HYP_OK;
+  for (int it = -1; it < iters && rc == HYP_OK; ++it) {
+    fill_pattern_kernel<<<148 * 4, 256, 0, st>>>(s->x, (size_t)M * s->dims.H);
+    s->launches += 1;
+    rc = run_blocks(s, bm, decode, n_splits, st, it < 0 ? nullptr : &ev[(size_t)it * (s->L + 1)]);
+  }
+  if (rc == HYP_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = HYP_ECUDA;
+  if (rc == HYP_OK) {
+    std::vector<float> samples(iters);
+    for (int li = 0; li < s->L; ++li) {
+      for (int it = 0; it < iters; ++it)
+        cudaEventElapsedTime(&samples[it], ev[(size_t)it * (s->L + 1) + li], ev[(size_t)it * (s->L + 1) + li + 1]);
+      std::sort(samples.begin(), samples.end());
+      layer_ms[li] = samples[iters / 2];
+      const ModelDims& d = s->dims;
+      const size_t wbytes = ((size_t)d.qkv_rows * d.H + (size_t)d.H * d.Hq * d.D + (size_t)3 * d.F * d.H + 2 * d.H) * 2;
+      layer_bytes[li] = wbytes + s->kv_layer_elems * sizeof(bf16) + s->workspace_bytes / s->L;
+    }
+  }
+  for (auto& e : ev) cudaEventDestroy(e);
+  // the scratch rows wrote K/V into free pages only; live sequences were not touched
+  return rc;
+}

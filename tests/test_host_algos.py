@@ -1,0 +1,127 @@
+"""Library host algorithms (through the C ABI, no GPU needed) against the oracle: bit-exact
+boundaries and tau for hyp_split_dp, identical node for hyp_sched_rt; error codes; ABI exports."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import split as osp
+from paper_2511_14450_b200 import hyperion as hyp
+from paper_2511_14450_b200 import inputs
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    declared = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        text = open(os.path.join(ROOT, "include", fn)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        declared |= set(re.findall(r"\b(hyp_[a-z0-9_]+)\s*\(", text))
+    assert declared, "no declarations parsed"
+    L = hyp.lib()
+    for name in sorted(declared):
+        assert hasattr(L, name), f"{name} declared in include/ but not exported"
+    assert declared == set(hyp.SIGNATURES), (declared ^ set(hyp.SIGNATURES))
+
+
+@pytest.mark.parametrize("N", range(1, 13))
+def test_split_dp_exact_equals_enumeration_bit_exact(N):
+    for T in range(1, min(N, 5) + 1):
+        for s in range(6):
+            f, m, C, M = inputs.split_instance(N, T, stream=1000 * N + 10 * T + s, integer=(s % 2 == 1),
+                                               tight_memory=(s >= 4))
+            p_e, tau_e = osp.enumerate_split(f, m, C, M)
+            if p_e is None:
+                with pytest.raises(hyp.HyperionError) as ei:
+                    hyp.hyp_split_dp(f, m, C, M)
+                assert ei.value.code == hyp.HYP_EINFEASIBLE
+                continue
+            p, tau = hyp.hyp_split_dp(f, m, C, M)
+            assert p == p_e and tau == tau_e          # bit-exact, including the tie-break
+
+
+def test_split_dp_ties_with_integer_costs():
+    # many equal-bottleneck partitions: the canonical one must come back
+    r = np.random.default_rng(5)
+    for _ in range(60):
+        N, T = int(r.integers(3, 12)), int(r.integers(2, 5))
+        if N < T:
+            continue
+        f = r.integers(1, 3, N).astype(float)
+        m = np.ones(N)
+        C = np.ones(T)
+        M = np.full(T, float(r.integers(2, N + 1)))
+        p_e, tau_e = osp.enumerate_split(f, m, C, M)
+        if p_e is None:
+            continue
+        assert hyp.hyp_split_dp(f, m, C, M) == (p_e, tau_e)
+
+
+def test_split_dp_bisection_mode_matches_algorithm_1_step_for_step():
+    for s in range(30):
+        N, T = 5 + s % 8, 2 + s % 3
+        f, m, C, M = inputs.split_instance(N, T, stream=5000 + s, tight_memory=(s % 4 == 0))
+        eps = 1e-3 * (f.sum() / C.min())
+        p_o, tau_o, _ = osp.hypsplit_dp_bisect(f, m, C, M, eps)
+        if p_o is None:
+            with pytest.raises(hyp.HyperionError):
+                hyp.hyp_split_dp(f, m, C, M, eps)
+            continue
+        assert hyp.hyp_split_dp(f, m, C, M, eps) == (p_o, tau_o)
+        # and it is within eps of the exact optimum
+        assert hyp.hyp_split_dp(f, m, C, M)[1] <= tau_o <= hyp.hyp_split_dp(f, m, C, M)[1] + eps
+
+
+def test_split_dp_config0_instance_and_40_layer_uniform():
+    u = inputs.uniform_f64(inputs.SEED_SPLIT, 0, 8)
+    f, m, C, M = 1.0 + u, np.ones(8), [67.0, 157.0, 200.0], [2.0, 4.0, 8.0]
+    assert hyp.hyp_split_dp(f, m, C, M) == osp.enumerate_split(f, m, C, M)
+    assert hyp.hyp_split_dp([1.0] * 40, [1.0] * 40, [1.0] * 3, [1e9] * 3) == ((12, 26), 14.0)
+
+
+def test_split_dp_errors():
+    ok = ([1.0, 2.0], [1.0, 1.0], [1.0, 1.0], [5.0, 5.0])
+    assert hyp.hyp_split_dp(*ok)[0] == (1,)
+    bad = [
+        ([1.0, -2.0], ok[1], ok[2], ok[3]), (ok[0], [1.0, float("nan")], ok[2], ok[3]),
+        (ok[0], ok[1], [1.0, 0.0], ok[3]), (ok[0], ok[1], ok[2], [5.0, -1.0]),
+    ]
+    for args in bad:
+        with pytest.raises(hyp.HyperionError) as ei:
+            hyp.hyp_split_dp(*args)
+        assert ei.value.code == hyp.HYP_EINVAL
+    with pytest.raises(hyp.HyperionError) as ei:
+        hyp.hyp_split_dp([1.0], [1.0], [1.0, 1.0], [5.0, 5.0])      # N < T
+    assert ei.value.code == hyp.HYP_EINFEASIBLE
+    with pytest.raises(hyp.HyperionError) as ei:
+        hyp.hyp_split_dp(ok[0], ok[1], ok[2], ok[3], eps=-1.0)
+    assert ei.value.code == hyp.HYP_EINVAL
+
+
+def test_sched_rt_matches_oracle():
+    r = np.random.default_rng(11)
+    for _ in range(300):
+        K = int(r.integers(1, 10))
+        nodes_o, nodes_l = [], []
+        for _k in range(K):
+            nd = {"C": float(r.integers(1, 6)), "M_avail": float(r.integers(0, 5)), "F_rem": float(r.integers(0, 5)),
+                  "F_wait": [float(v) for v in r.integers(0, 7, int(r.integers(0, 4)))],
+                  "available": bool(r.integers(0, 4))}
+            nodes_o.append(nd)
+            nodes_l.append((nd["C"], nd["M_avail"], nd["F_rem"], sum(nd["F_wait"]), int(nd["available"])))
+        want = osp.hypsched_rt_scan(4.0, 2.0, nodes_o)
+        if want < 0:
+            with pytest.raises(hyp.HyperionError) as ei:
+                hyp.hyp_sched_rt(4.0, 2.0, nodes_l)
+            assert ei.value.code == hyp.HYP_EINFEASIBLE
+        else:
+            assert hyp.hyp_sched_rt(4.0, 2.0, nodes_l) == want
+
+
+def test_strerror_covers_all_codes():
+    L = hyp.lib()
+    seen = {L.hyp_strerror(c).decode() for c in range(0, -7, -1)}
+    assert len(seen) == 7 and "unknown status" not in seen
+    assert L.hyp_strerror(-99).decode() == "unknown status"
