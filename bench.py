@@ -1,0 +1,319 @@
+"""Benchmark of the stage hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+A step is one KV-cached decode step of the whole stage (every block's kernels) over one batch.
+Workload: 14 contiguous Phi-3-medium-shaped blocks (the first stage of a 14/13/13 split), decode
+batch 8, 1024-token paged KV context per sequence (pages of 16), bf16 seeded random-init weights,
+teacher-forced token ids.  With N > 1 every rank runs an independent replica of the stage on its own
+GPU (request-level replication, no data-path collective); the value is all ranks' tokens divided by
+the slowest rank's time.
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "stage_decode_tokens_per_s"
+UNIT = "tokens/s"
+N_LAYERS_STAGE = 14
+BATCH = 8
+CTX0 = 1024
+FALLBACK_HBM_GBS = 6650.0
+
+
+def workload_config(steps, warmup):
+    return {
+        "workload": "configs[2]: one pipeline stage of 14 contiguous Phi-3-medium-shaped layers, decode batch 8, "
+                    "1024-token KV context per sequence, paged KV block 16, bf16 random init, teacher-forced",
+        "layers": N_LAYERS_STAGE, "batch": BATCH, "ctx_start": CTX0, "kv_block": 16,
+        "parallelism": "replicas (one stage per GPU, no collective)",
+        "l2": "inputs larger than L2: 9.5 GB of weights are streamed once per step",
+    }
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as fh:
+            d = json.load(fh)
+        return float(d["hbm_gbs"]), "measured", d
+    return FALLBACK_HBM_GBS, "fallback", {}
+
+
+# ------------------------------------------------------------------------------------------
+# distributed aggregation (host logic; exercised with gloo on CPU by the tests)
+# ------------------------------------------------------------------------------------------
+def aggregate_over_ranks(local_ms: float, local_units: float, dist=None, device="cpu"):
+    """Whole-job view of a timed region: (max time over ranks, units summed over ranks)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return local_ms, local_units
+    import torch
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([local_units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for ln in self.proc.stdout:
+            self.lines.append((time.time(), ln.strip()))
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for ts, ln in self.lines:
+            if t0 is not None and not (t0 - 0.05 <= ts <= t1 + 0.15):
+                continue
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------
+# CPU baseline: the oracle, as it stands, on a bounded sample
+# ------------------------------------------------------------------------------------------
+def oracle_decode_sample(steps: int, warmup: int):
+    """Time the oracle's literal KV-cached decode on a sample of the workload: ONE sequence through
+    ONE block with a 1024-token cache (seeded random K/V), `steps` single-token steps.  Returns
+    (tokens/s scaled to the 14-block stage, seconds per token-block, threads used, description)."""
+    import numpy as np
+    from oracle import decoder as od
+    from paper_2511_14450_b200 import inputs
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    sh = inputs.phi3_medium_shape()
+    osh = od.Shape(sh.hidden, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.ffn, sh.vocab, sh.rms_eps, sh.rope_theta)
+    w = {k: inputs.bf16_bits_to_f64(v) for k, v in inputs.layer_weights(sh, 0).items()}
+    cs = od.CachedStage([w], osh)
+    cs.k[0] = inputs.bf16_bits_to_f64(inputs.normal_bf16(7, 1, (CTX0, sh.n_kv_heads, sh.head_dim), std=1.0))
+    cs.v[0] = inputs.bf16_bits_to_f64(inputs.normal_bf16(7, 2, (CTX0, sh.n_kv_heads, sh.head_dim), std=1.0))
+    cs.n_cached = CTX0
+    x = inputs.bf16_bits_to_f64(inputs.normal_bf16(7, 3, (warmup + steps, sh.hidden), std=1.0))
+    for i in range(warmup):
+        cs.step(x[i:i + 1])
+    t0 = time.perf_counter()
+    for i in range(warmup, warmup + steps):
+        cs.step(x[i:i + 1])
+    dt = (time.perf_counter() - t0) / steps
+    desc = (f"{steps} decode steps of 1 sequence through 1 of the {N_LAYERS_STAGE} blocks at a {CTX0}-token cache "
+            f"(float64 numpy oracle); tokens/s = 1 / ({N_LAYERS_STAGE} x seconds per token-block)")
+    return 1.0 / (N_LAYERS_STAGE * dt), dt, cores, desc
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, min(args.steps, 16))
+    warm = max(1, min(args.warmup, 3))
+    tps, dt, cores, desc = oracle_decode_sample(steps, warm)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warm, "ms_per_step": dt * 1e3 * N_LAYERS_STAGE * BATCH, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(steps, warm),
+        "cpu_baseline": {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------
+# the library arm
+# ------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2511_14450_b200 import hyperion as hyp
+    from paper_2511_14450_b200 import inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    K, W = args.steps, max(args.warmup, 3)
+    sh = inputs.phi3_medium_shape()
+    max_ctx = CTX0 + W + 2 * K + 16
+    st = hyp.Stage(sh, 0, N_LAYERS_STAGE, max_seqs=BATCH, max_ctx=max_ctx, max_tokens=CTX0)
+    for layer in range(N_LAYERS_STAGE):
+        st.load_layer(layer, inputs.layer_weights(sh, layer, device="cuda"))
+        torch.cuda.synchronize()
+    st.load_embed(inputs.embed_weights(sh, device="cuda"))
+    torch.cuda.synchronize()
+
+    stream = torch.cuda.current_stream()
+    slots = list(range(BATCH))
+    hidden = torch.empty(CTX0, sh.hidden, dtype=torch.float32, device="cuda")
+    for b in slots:          # untimed: fill the KV cache with a 1024-token prefill per sequence
+        ids = inputs.token_ids(inputs.SEED_PROMPTS, 100 * rank + b, CTX0, sh.vocab, device="cuda")
+        st.prefill([b], [CTX0], [0], ids, hidden)
+    torch.cuda.synchronize()
+    total_steps = W + 2 * K
+    forced = torch.stack([inputs.token_ids(inputs.SEED_FORCED, 100 * rank + b, total_steps, sh.vocab)
+                          for b in slots], dim=1).contiguous()            # [steps, B]
+    forced_dev = forced.cuda()
+    out = torch.empty(BATCH, sh.hidden, dtype=torch.float32, device="cuda")
+
+    ctx = CTX0
+    for i in range(W):
+        st.decode(slots, [ctx] * BATCH, forced_dev[i], out)
+        ctx += 1
+    torch.cuda.synchronize()
+
+    # --- device-resident timed region ---------------------------------------------------------
+    hyp.hyp_stage_kernel_timing(st.handle, hyp.HYP_K_GEMM_GATE_UP, K * N_LAYERS_STAGE)
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = hyp.hyp_stage_launch_count(st.handle)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    torch.cuda.profiler.start()          # lets a profiler attach to the timed region only
+    e0.record(stream)
+    ctx_sum = 0
+    for i in range(K):
+        st.decode(slots, [ctx] * BATCH, forced_dev[W + i], out)
+        ctx_sum += ctx + 1
+        ctx += 1
+    e1.record(stream)
+    torch.cuda.synchronize()
+    torch.cuda.profiler.stop()
+    t_wall1 = time.time()
+    if world > 1:
+        dist.barrier()
+    local_ms = e0.elapsed_time(e1)
+    launches = hyp.hyp_stage_launch_count(st.handle) - launches0
+    clocks = sampler.stop(t_wall0, t_wall1)
+    n_k, k_ms = hyp.hyp_stage_kernel_timing_read(st.handle)
+    hyp.hyp_stage_kernel_timing(st.handle, -1, 0)
+    ms, tokens = aggregate_over_ranks(local_ms, BATCH * K, dist if world > 1 else None, "cuda")
+
+    # --- end-to-end: host buffers through the C ABI, copies inside the timed region -------------
+    ids_host = forced.pin_memory()
+    out_host = torch.empty(BATCH, sh.hidden, dtype=torch.float32).pin_memory()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record(stream)
+    for i in range(K):
+        hyp.hyp_stage_decode_host(st.handle, slots, [ctx] * BATCH, ids_host[W + K + i], out_host)
+        ctx += 1
+    e3.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms, e2e_tokens = aggregate_over_ranks(e2.elapsed_time(e3), BATCH * K, dist if world > 1 else None, "cuda")
+
+    # --- roofline of the dominant kernel (gate/up projection with fused SwiGLU) -------------------
+    peak, peak_src, _ = measured_peaks()
+    gu_bytes = 2 * sh.ffn * sh.hidden * 2 + BATCH * sh.hidden * 2 + BATCH * sh.ffn * 2
+    achieved = (gu_bytes / 1e9) / (k_ms / n_k / 1e3) if n_k else None
+    weight_bytes = N_LAYERS_STAGE * (sh.layer_linear_params * 2 + 4 * sh.hidden)
+    kv_bytes_per_ctx = N_LAYERS_STAGE * BATCH * 2 * sh.n_kv_heads * sh.head_dim * 2
+    step_bytes = weight_bytes + kv_bytes_per_ctx * (ctx_sum / K)
+    step_gbs = step_bytes / 1e9 / (local_ms / K / 1e3)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": tokens / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": workload_config(K, W),
+            "e2e": {"value": e2e_tokens / (e2e_ms / 1e3), "unit": UNIT,
+                    "h2d_bytes_per_step": BATCH * 4, "d2h_bytes_per_step": BATCH * sh.hidden * 4},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "roofline": {"bound": "hbm", "kernel": "gemm_skinny_kernel<SwiGLU> (gate/up projection)",
+                         "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": (achieved / peak) if achieved else None, "peak_source": f"of {peak_src}",
+                         "bytes_per_launch": gu_bytes, "launches_timed": n_k,
+                         "avg_launch_us": (k_ms / n_k * 1e3) if n_k else None, "traffic": None},
+            "step_roofline": {"bound": "hbm", "bytes_per_step": step_bytes, "achieved": step_gbs, "peak": peak,
+                              "unit": "GB/s", "frac": step_gbs / peak, "frac_of_nominal_8TBs": step_gbs / 8000.0},
+        }
+        if not args.no_cpu_baseline and world == 1:
+            tps, dt, cores, desc = oracle_decode_sample(4, 1)
+            line["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+        print(json.dumps(line))
+    st.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=128)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -148,6 +148,19 @@ HYP_API int hyp_stage_decode_host(hyp_stage* s, const hyp_batch* batch, const vo
 HYP_API int hyp_stage_profile(hyp_stage* s, int32_t mode, int32_t batch, int32_t ctx, int32_t iters,
                       float* layer_ms, size_t* layer_bytes, void* stream);
 
+/* Kernel classes of the block sequence, for per-launch timing. */
+enum {
+  HYP_K_GEMM_QKV = 0, HYP_K_GEMM_O = 1, HYP_K_GEMM_GATE_UP = 2, HYP_K_GEMM_DOWN = 3,
+  HYP_K_ATTN = 4, HYP_K_NORM = 5, HYP_K_ROPE = 6, HYP_K_LM_HEAD = 7
+};
+/* Bracket every launch of one kernel class with a CUDA event pair on the call's stream (at most
+ * max_samples launches are recorded; kernel_class = -1 switches timing off).  Creating the events
+ * happens here, not in prefill/decode.  Measurement aid for roofline reporting. */
+HYP_API int hyp_stage_kernel_timing(hyp_stage* s, int32_t kernel_class, int32_t max_samples);
+/* Wait for the recorded pairs, return their count and summed duration (HOST outputs), and reset
+ * the sample counter. */
+HYP_API int hyp_stage_kernel_timing_read(hyp_stage* s, int32_t* n_samples, double* total_ms);
+
 /* Return a sequence's KV pages to the pool and zero its cached length. */
 HYP_API int hyp_stage_free_seq(hyp_stage* s, int32_t seq_id);
 /* Tokens currently cached for a slot, or a negative status. */

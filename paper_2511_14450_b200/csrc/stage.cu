@@ -67,6 +67,10 @@ struct hyp_stage {
   void *io_in = nullptr, *io_out = nullptr;
   size_t io_in_bytes = 0, io_out_bytes = 0;
   int64_t launches = 0;
+  // optional per-launch timing of one kernel class
+  int time_cls = -1;
+  std::vector<cudaEvent_t> time_ev;
+  int time_n = 0;
 };
 
 namespace {
@@ -215,6 +219,18 @@ int check_ready(const hyp_stage* s) {
     s->launches += _n;                                     \
   } while (0)
 
+// Same as HYP_LAUNCH, bracketed by an event pair when kernel class `cls` is being timed.
+#define HYP_LAUNCH_T(cls, call)                                                             \
+  do {                                                                                      \
+    const bool _t = s->time_cls == (cls) && (size_t)(2 * s->time_n + 1) < s->time_ev.size(); \
+    if (_t) HYP_CUDA_TRY(cudaEventRecord(s->time_ev[2 * s->time_n], st));                   \
+    HYP_LAUNCH(call);                                                                       \
+    if (_t) {                                                                               \
+      HYP_CUDA_TRY(cudaEventRecord(s->time_ev[2 * s->time_n + 1], st));                     \
+      s->time_n += 1;                                                                       \
+    }                                                                                       \
+  } while (0)
+
 // out[m, n] (+)= a[m, :] . w[n, :] with the kernel family chosen by the row count.
 int project(hyp_stage* s, const TcAct& act, const bf16* a, int lda, const TcWeight& tw, const bf16* w, int N, int K,
             int M, int epi, void* out, int ldo, cudaStream_t st) {
@@ -231,19 +247,21 @@ int run_blocks(hyp_stage* s, const BatchMeta& bm, bool decode, int n_splits, cud
   for (int li = 0; li < s->L; ++li) {
     LayerW& lw = s->layers[li];
     bf16* kv_layer = s->kv_pool + (size_t)li * s->kv_layer_elems;
-    HYP_LAUNCH(launch_rmsnorm(s->x, lw.g1, s->h, M, d.H, d.eps, nullptr, st));
-    HYP_LAUNCH(project(s, s->tc_h, s->h, d.H, lw.tc_qkv, lw.wqkv, d.qkv_rows, d.H, M, EPI_STORE_BF16, s->qkv,
-                       d.qkv_rows, st));
-    HYP_LAUNCH(launch_rope_kv_write(s->qkv, kv_layer, s->rope_table, bm, d, st));
+    HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g1, s->h, M, d.H, d.eps, nullptr, st));
+    HYP_LAUNCH_T(HYP_K_GEMM_QKV, project(s, s->tc_h, s->h, d.H, lw.tc_qkv, lw.wqkv, d.qkv_rows, d.H, M,
+                                         EPI_STORE_BF16, s->qkv, d.qkv_rows, st));
+    HYP_LAUNCH_T(HYP_K_ROPE, launch_rope_kv_write(s->qkv, kv_layer, s->rope_table, bm, d, st));
     if (decode)
-      HYP_LAUNCH(launch_attn_decode(s->qkv, kv_layer, s->attn, s->attn_scratch, n_splits, bm, d, st));
+      HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_decode(s->qkv, kv_layer, s->attn, s->attn_scratch, n_splits, bm, d, st));
     else
-      HYP_LAUNCH(launch_attn_prefill(s->qkv, kv_layer, s->attn, bm, d, st));
-    HYP_LAUNCH(project(s, s->tc_attn, s->attn, d.Hq * d.D, lw.tc_o, lw.wo, d.H, d.Hq * d.D, M, EPI_RESID_F32, s->x,
-                       d.H, st));
-    HYP_LAUNCH(launch_rmsnorm(s->x, lw.g2, s->h, M, d.H, d.eps, nullptr, st));
-    HYP_LAUNCH(project(s, s->tc_h, s->h, d.H, lw.tc_gu, lw.wgu, d.F, d.H, M, EPI_SWIGLU_BF16, s->u, d.F, st));
-    HYP_LAUNCH(project(s, s->tc_u, s->u, d.F, lw.tc_d, lw.wd, d.H, d.F, M, EPI_RESID_F32, s->x, d.H, st));
+      HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_prefill(s->qkv, kv_layer, s->attn, bm, d, st));
+    HYP_LAUNCH_T(HYP_K_GEMM_O, project(s, s->tc_attn, s->attn, d.Hq * d.D, lw.tc_o, lw.wo, d.H, d.Hq * d.D, M,
+                                       EPI_RESID_F32, s->x, d.H, st));
+    HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g2, s->h, M, d.H, d.eps, nullptr, st));
+    HYP_LAUNCH_T(HYP_K_GEMM_GATE_UP, project(s, s->tc_h, s->h, d.H, lw.tc_gu, lw.wgu, d.F, d.H, M, EPI_SWIGLU_BF16,
+                                             s->u, d.F, st));
+    HYP_LAUNCH_T(HYP_K_GEMM_DOWN, project(s, s->tc_u, s->u, d.F, lw.tc_d, lw.wd, d.H, d.F, M, EPI_RESID_F32, s->x,
+                                          d.H, st));
     if (marks) HYP_CUDA_TRY(cudaEventRecord(marks[li + 1], st));
   }
   return HYP_OK;
@@ -280,7 +298,8 @@ int run_stage(hyp_stage* s, const hyp_batch* b, const void* in, void* out, cudaS
     const bool all = (b->flags & HYP_BATCH_ALL_LOGITS) != 0 || decode;
     const int rows = all ? M : hb.n;
     HYP_LAUNCH(launch_rmsnorm(s->x, s->gf, s->h, rows, d.H, d.eps, all ? nullptr : bm.last_row, st));
-    HYP_LAUNCH(project(s, s->tc_h, s->h, d.H, s->tc_lm, s->wlm, d.V, d.H, rows, EPI_STORE_F32, out, d.V, st));
+    HYP_LAUNCH_T(HYP_K_LM_HEAD,
+                 project(s, s->tc_h, s->h, d.H, s->tc_lm, s->wlm, d.V, d.H, rows, EPI_STORE_F32, out, d.V, st));
   } else {
     HYP_LAUNCH(launch_copy_f32(s->x, (float*)out, (size_t)M * d.H, st));
   }
@@ -366,6 +385,7 @@ extern "C" void hyp_stage_destroy(hyp_stage* s) {
     if (s->meta_host[i]) cudaFreeHost(s->meta_host[i]);
     if (s->meta_ev[i]) cudaEventDestroy(s->meta_ev[i]);
   }
+  for (cudaEvent_t e : s->time_ev) cudaEventDestroy(e);
   delete s;
 }
 
@@ -541,6 +561,33 @@ extern "C" int hyp_stage_free_pages(const hyp_stage* s) {
 }
 
 extern "C" int64_t hyp_stage_launch_count(const hyp_stage* s) { return s ? s->launches : 0; }
+
+extern "C" int hyp_stage_kernel_timing(hyp_stage* s, int32_t kernel_class, int32_t max_samples) {
+  if (!s || kernel_class < -1 || kernel_class > HYP_K_LM_HEAD || max_samples < 0) return HYP_EINVAL;
+  s->time_cls = kernel_class;
+  s->time_n = 0;
+  while (s->time_ev.size() < (size_t)2 * max_samples) {
+    cudaEvent_t e;
+    HYP_CUDA_TRY(cudaEventCreate(&e));
+    s->time_ev.push_back(e);
+  }
+  return HYP_OK;
+}
+
+extern "C" int hyp_stage_kernel_timing_read(hyp_stage* s, int32_t* n_samples, double* total_ms) {
+  if (!s || !n_samples || !total_ms) return HYP_EINVAL;
+  double tot = 0.0;
+  for (int i = 0; i < s->time_n; ++i) {
+    HYP_CUDA_TRY(cudaEventSynchronize(s->time_ev[2 * i + 1]));
+    float ms = 0.f;
+    HYP_CUDA_TRY(cudaEventElapsedTime(&ms, s->time_ev[2 * i], s->time_ev[2 * i + 1]));
+    tot += ms;
+  }
+  *n_samples = s->time_n;
+  *total_ms = tot;
+  s->time_n = 0;
+  return HYP_OK;
+}
 
 extern "C" int hyp_stage_profile(hyp_stage* s, int32_t mode, int32_t batch, int32_t ctx, int32_t iters,
                                  float* layer_ms, size_t* layer_bytes, void* stream) {

@@ -58,6 +58,8 @@ SIGNATURES = {
     "hyp_stage_decode_host": (C.c_int, [C.c_void_p, C.POINTER(hyp_batch), C.c_void_p, C.c_void_p, C.c_void_p]),
     "hyp_stage_profile": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_float),
                                     C.POINTER(C.c_size_t), C.c_void_p]),
+    "hyp_stage_kernel_timing": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32]),
+    "hyp_stage_kernel_timing_read": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_double)]),
     "hyp_stage_free_seq": (C.c_int, [C.c_void_p, C.c_int32]),
     "hyp_stage_seq_len": (C.c_int, [C.c_void_p, C.c_int32]),
     "hyp_stage_free_pages": (C.c_int, [C.c_void_p]),
@@ -174,6 +176,21 @@ def hyp_stage_profile(stage, n_layers: int, mode: int, batch: int, ctx: int, ite
     _check(lib().hyp_stage_profile(stage, mode, batch, ctx, iters, ms, by, _stream_handle(stream)),
            "hyp_stage_profile")
     return list(ms), list(by)
+
+
+(HYP_K_GEMM_QKV, HYP_K_GEMM_O, HYP_K_GEMM_GATE_UP, HYP_K_GEMM_DOWN, HYP_K_ATTN, HYP_K_NORM, HYP_K_ROPE,
+ HYP_K_LM_HEAD) = range(8)
+
+
+def hyp_stage_kernel_timing(stage, kernel_class: int, max_samples: int):
+    _check(lib().hyp_stage_kernel_timing(stage, kernel_class, max_samples), "hyp_stage_kernel_timing")
+
+
+def hyp_stage_kernel_timing_read(stage):
+    """Returns (launches recorded, their summed milliseconds)."""
+    n, ms = C.c_int32(), C.c_double()
+    _check(lib().hyp_stage_kernel_timing_read(stage, C.byref(n), C.byref(ms)), "hyp_stage_kernel_timing_read")
+    return n.value, ms.value
 
 
 def hyp_stage_free_seq(stage, seq_id: int):
