@@ -49,7 +49,9 @@ typedef enum {
   HYP_EINFEASIBLE = -4, /* hyp_split_dp: no memory-feasible partition (or N < T);                 */
                         /* hyp_sched_rt: no available node with enough memory                     */
   HYP_ECUDA = -5,       /* a CUDA call failed; hyp_last_cuda_error() gives the cudaError_t        */
-  HYP_ESTATE = -6       /* stage not ready (a weight tensor was never loaded)                     */
+  HYP_ESTATE = -6,      /* stage not ready (a weight tensor was never loaded)                     */
+  HYP_ETIMEOUT = -7     /* a bounded device-side wait expired inside a kernel; reported by the     */
+                        /* calls that synchronise (*_host, hyp_stage_profile); results are invalid */
 } hyp_status;
 
 typedef struct hyp_stage hyp_stage; /* opaque, library-owned */

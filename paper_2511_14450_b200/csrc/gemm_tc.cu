@@ -1,30 +1,385 @@
-// Bring-up body: row chunks through the weight-streaming kernel (replaced by tcgen05 tiles).
+// Tensor-core projection for prefill: out[m, n] (+)= sum_k act[m, k] * w[n, k], bf16 in, fp32 accumulate.
+//
+// Persistent, warp-specialised sm_100a kernel:
+//   warp 0   one lane issues TMA tile loads (128B-swizzled, K-major) into a 4-stage shared-memory ring;
+//   warp 1   one lane issues tcgen05.mma (128 x 256 x 16 per instruction) into tensor memory; the
+//            accumulator is double-buffered (2 x 256 columns) so the epilogue of tile i overlaps the
+//            main loop of tile i+1;
+//   warps 2-5  read the accumulator with tcgen05.ld and apply the epilogue (bf16 store, residual add,
+//            SiLU(gate) * up, fp32 store) straight to global memory.
+// For the SwiGLU epilogue the 256 accumulator columns are 128 gate columns and the 128 matching up
+// columns (two weight boxes per stage), so gate and up never leave the chip.
+// Every mbarrier wait is bounded: on expiry the kernel records an error code and unwinds.
+#include <cuda.h>
+
 #include "gemm_tc.cuh"
 #include "hyperion.h"
 
 namespace hyp {
 
-int tc_make_weight(TcWeight* w, const __nv_bfloat16* ptr, int rows, int K) {
-  w->ptr = ptr; w->rows = rows; w->K = K;
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+constexpr int TC_THREADS = 192;
+constexpr uint64_t WAIT_LIMIT_NS = 4000000000ull;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint64_t globaltimer() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false after WAIT_LIMIT_NS or once another role has raised `abort_flag`.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (int i = 0; i < 64; ++i)
+    if (mbar_try(bar, parity)) return true;
+  const uint64_t t0 = globaltimer();
+  while (true) {
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (globaltimer() - t0 > WAIT_LIMIT_NS) return false;
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;            // leading byte offset: not used by swizzled K-major layouts
+  d |= (uint64_t)(1024 >> 4) << 32;  // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;            // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;            // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 256.
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+template <int EPI>
+__device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[16], const uint32_t (&v2)[16], void* out, int ldo,
+                                               int row, int col, int N) {
+  const size_t o = (size_t)row * ldo + col;
+  const bool full = col + 16 <= N;
+  if (EPI == EPI_STORE_BF16 || EPI == EPI_SWIGLU_BF16) {
+    float f[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float a = __uint_as_float(v[i]);
+      f[i] = (EPI == EPI_SWIGLU_BF16) ? a / (1.f + __expf(-a)) * __uint_as_float(v2[i]) : a;
+    }
+    __nv_bfloat16* p = reinterpret_cast<__nv_bfloat16*>(out) + o;
+    if (full) {
+      uint4 w0 = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+      uint4 w1 = make_uint4(pack_bf16(f[8], f[9]), pack_bf16(f[10], f[11]), pack_bf16(f[12], f[13]),
+                            pack_bf16(f[14], f[15]));
+      reinterpret_cast<uint4*>(p)[0] = w0;
+      reinterpret_cast<uint4*>(p)[1] = w1;
+    } else {
+#pragma unroll
+      for (int i = 0; i < 16; ++i)
+        if (col + i < N) p[i] = __float2bfloat16_rn(f[i]);
+    }
+  } else {
+    float* p = reinterpret_cast<float*>(out) + o;
+    if (full) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float4 a = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
+                               __uint_as_float(v[4 * i + 3]));
+        if (EPI == EPI_RESID_F32) {
+          const float4 b = reinterpret_cast<const float4*>(p)[i];
+          a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+        }
+        reinterpret_cast<float4*>(p)[i] = a;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 16; ++i)
+        if (col + i < N) p[i] = (EPI == EPI_RESID_F32 ? p[i] : 0.f) + __uint_as_float(v[i]);
+    }
+  }
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int M, int N, int K,
+               void* __restrict__ out, int ldo, int* __restrict__ err) {
+  constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
+  constexpr int BN_OUT = SWIGLU ? BN / 2 : BN;  // output columns per tile
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* aligned = smem_raw + (base - smem_u32(smem_raw));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(aligned + STAGES * STAGE_BYTES);
+  // bars: full[STAGES] | empty[STAGES] | tmem_full[2] | tmem_empty[2] | tmem base (u32) | abort (int)
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN_OUT - 1) / BN_OUT;
+  const int n_tiles = tiles_m * tiles_n;
+  const int KB = (K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 128);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---------------- TMA producer ----------------
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile % tiles_m) * BM;
+        const int n0 = (tile / tiles_m) * BN_OUT;
+        const int rb0 = n0, rb1 = SWIGLU ? N + n0 : n0 + 128;
+        for (int kb = 0; kb < KB; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) { ok = false; break; }
+          const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
+          mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+          tma_load_2d(sa, &tm_a, kb * BK, m0, full_bar(stage));
+          tma_load_2d(sb, &tm_b, kb * BK, rb0, full_bar(stage));
+          tma_load_2d(sb + B_BYTES / 2, &tm_b, kb * BK, rb1, full_bar(stage));
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicCAS(err, 0, 1);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ---------------- MMA issuer ----------------
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < KB; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
+          const uint64_t da = smem_desc(sa), db = smem_desc(sb);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            tc_mma(d_tmem, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), IDESC,
+                   (kb | k) != 0 ? 1u : 0u);
+          tc_commit(empty_bar(stage));
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        tc_commit(tfull_bar(acc));
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1;
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicCAS(err, 0, 2);
+      }
+    }
+  } else {
+    // ---------------- epilogue warps ----------------
+    const int q = warp & 3;  // tensor-memory lane quarter this warp may read
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      const int m0 = (tile % tiles_m) * BM;
+      const int n0 = (tile / tiles_m) * BN_OUT;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int row = m0 + 32 * q + lane;
+      const uint32_t t0 = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * BN);
+#pragma unroll 2
+      for (int c = 0; c < BN_OUT; c += 16) {
+        if (n0 + c >= N) break;  // uniform across the warp
+        uint32_t v[16], v2[16];
+        tmem_ld16(t0 + c, v);
+        if (SWIGLU) tmem_ld16(t0 + BN / 2 + c, v2);
+        tmem_ld_wait();
+        if (row < M) epilogue_chunk<EPI>(v, v2, out, ldo, row, n0 + c, N);
+      }
+      tc_fence_before();
+      mbar_arrive(tempty_bar(acc));
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1;
+    }
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      atomicCAS(err, 0, 3);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+int make_map(TcOperand* op, const __nv_bfloat16* ptr, int rows, int K) {
+  op->ptr = ptr;
+  op->rows = rows;
+  op->K = K;
+  op->box_rows = 128;
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return HYP_ECUDA;
+  if ((K % 8) != 0 || ((uintptr_t)ptr & 15) != 0) return HYP_EINVAL;
+  const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)BK, 128u};
+  const cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = enc(&op->map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)ptr, dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error((int)r);
+    return HYP_ECUDA;
+  }
   return HYP_OK;
 }
-int tc_make_act(TcAct* a, const __nv_bfloat16* ptr, int rows, int K) {
-  a->ptr = ptr; a->rows = rows; a->K = K;
+
+int* g_err_flag = nullptr;  // one device word per process: first non-zero code wins
+
+template <int EPI>
+int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* out, int ldo, cudaStream_t st) {
+  static bool configured = false;
+  static int num_sms = 0;
+  if (!configured) {
+    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    int dev = 0;
+    HYP_CUDA_TRY(cudaGetDevice(&dev));
+    HYP_CUDA_TRY(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
+    configured = true;
+  }
+  constexpr int BN_OUT = EPI == EPI_SWIGLU_BF16 ? BN / 2 : BN;
+  const int tiles = ((M + BM - 1) / BM) * ((N + BN_OUT - 1) / BN_OUT);
+  const int grid = tiles < num_sms ? tiles : num_sms;
+  gemm_tc_kernel<EPI><<<grid, TC_THREADS, SMEM_BYTES, st>>>(act.map, w.map, M, N, K, out, ldo, g_err_flag);
+  return 1;
+}
+
+}  // namespace
+
+int tc_make_weight(TcWeight* w, const __nv_bfloat16* ptr, int rows, int K) { return make_map(w, ptr, rows, K); }
+int tc_make_act(TcAct* a, const __nv_bfloat16* ptr, int rows, int K) { return make_map(a, ptr, rows, K); }
+
+int tc_prepare() {
+  if (!g_err_flag) {
+    HYP_CUDA_TRY(cudaMalloc((void**)&g_err_flag, sizeof(int)));
+    HYP_CUDA_TRY(cudaMemset(g_err_flag, 0, sizeof(int)));
+  }
+  return HYP_OK;
+}
+
+int tc_error_flag(int* value_out) {
+  *value_out = 0;
+  if (!g_err_flag) return HYP_OK;
+  HYP_CUDA_TRY(cudaMemcpy(value_out, g_err_flag, sizeof(int), cudaMemcpyDeviceToHost));
   return HYP_OK;
 }
 
 int launch_gemm_tc(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
                    cudaStream_t st) {
-  int n = 0;
-  const size_t esz = (epi == EPI_STORE_BF16 || epi == EPI_SWIGLU_BF16) ? 2 : 4;
-  for (int m0 = 0; m0 < M; m0 += 32) {
-    const int rows = M - m0 < 32 ? M - m0 : 32;
-    int rc = launch_gemm_skinny(act.ptr + (size_t)m0 * K, K, w.ptr, N, K, rows, epi,
-                                (char*)out + (size_t)m0 * ldo * esz, ldo, st);
-    if (rc < 0) return rc;
-    n += rc;
+  if (M < 1 || N < 1 || K < 8 || act.K != K || w.K != K || M > act.rows || !g_err_flag) return HYP_EINVAL;
+  switch (epi) {
+    case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16>(act, w, M, N, K, out, ldo, st);
+    case EPI_RESID_F32: return launch_epi<EPI_RESID_F32>(act, w, M, N, K, out, ldo, st);
+    case EPI_SWIGLU_BF16: return launch_epi<EPI_SWIGLU_BF16>(act, w, M, N, K, out, ldo, st);
+    case EPI_STORE_F32: return launch_epi<EPI_STORE_F32>(act, w, M, N, K, out, ldo, st);
+    default: return HYP_EINVAL;
   }
-  return n;
 }
 
 }  // namespace hyp

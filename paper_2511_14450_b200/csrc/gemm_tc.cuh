@@ -19,6 +19,11 @@ typedef TcOperand TcAct;
 int tc_make_weight(TcWeight* w, const __nv_bfloat16* ptr, int rows, int K);
 int tc_make_act(TcAct* a, const __nv_bfloat16* ptr, int rows, int K);
 
+// One-time set-up of the device-side error word (allocates; call from stage creation, not from the hot path).
+int tc_prepare();
+// Reads the error word (synchronises the device): 0 = no kernel gave up on a wait.
+int tc_error_flag(int* value_out);
+
 // out[m, n] (+)= sum_k act[m, k] * w[n, k] for m < M, n < N (SwiGLU: w holds 2N rows).
 int launch_gemm_tc(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
                    cudaStream_t st);

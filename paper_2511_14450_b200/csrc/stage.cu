@@ -342,7 +342,10 @@ int run_stage_host(hyp_stage* s, const hyp_batch* b, const void* in, void* out, 
   if (rc) return rc;
   HYP_CUDA_TRY(cudaMemcpyAsync(out, s->io_out, out_bytes, cudaMemcpyDeviceToHost, st));
   HYP_CUDA_TRY(cudaStreamSynchronize(st));
-  return HYP_OK;
+  int dev_err = 0;
+  rc = tc_error_flag(&dev_err);
+  if (rc) return rc;
+  return dev_err ? HYP_ETIMEOUT : HYP_OK;
 }
 
 __global__ void fill_pattern_kernel(float* x, size_t n) {
@@ -368,6 +371,7 @@ extern "C" const char* hyp_strerror(int code) {
     case HYP_EINFEASIBLE: return "no feasible solution";
     case HYP_ECUDA: return "CUDA error (see hyp_last_cuda_error)";
     case HYP_ESTATE: return "stage not ready: a weight tensor has not been loaded";
+    case HYP_ETIMEOUT: return "a device-side wait expired inside a kernel (results invalid)";
     default: return "unknown status";
   }
 }
@@ -484,6 +488,7 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
   TRY_CUDA(cudaMalloc(&s->io_in, s->io_in_bytes));
   TRY_CUDA(cudaMalloc(&s->io_out, s->io_out_bytes));
   // tensor-core operand descriptors over the fixed workspace buffers
+  TRY(tc_prepare());
   TRY(tc_make_act(&s->tc_h, s->h, (int)rows_pad, d.H));
   TRY(tc_make_act(&s->tc_attn, s->attn, (int)rows_pad, d.Hq * d.D));
   TRY(tc_make_act(&s->tc_u, s->u, (int)rows_pad, d.F));
@@ -639,6 +644,11 @@ extern "C" int hyp_stage_profile(hyp_stage* s, int32_t mode, int32_t batch, int3
     rc = run_blocks(s, bm, decode, n_splits, st, it < 0 ? nullptr : &ev[(size_t)it * (s->L + 1)]);
   }
   if (rc == HYP_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = HYP_ECUDA;
+  if (rc == HYP_OK) {
+    int dev_err = 0;
+    rc = tc_error_flag(&dev_err);
+    if (rc == HYP_OK && dev_err) rc = HYP_ETIMEOUT;
+  }
   if (rc == HYP_OK) {
     std::vector<float> samples(iters);
     for (int li = 0; li < s->L; ++li) {

@@ -13,6 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "lib", "libhyperion.so")
 
 HYP_OK, HYP_EINVAL, HYP_ENOMEM, HYP_ECAPACITY, HYP_EINFEASIBLE, HYP_ECUDA, HYP_ESTATE = 0, -1, -2, -3, -4, -5, -6
+HYP_ETIMEOUT = -7
 (HYP_W_QKV, HYP_W_O, HYP_W_GATE_UP, HYP_W_DOWN, HYP_W_NORM1, HYP_W_NORM2, HYP_W_EMBED, HYP_W_FINAL_NORM,
  HYP_W_LM_HEAD) = range(9)
 HYP_BATCH_ALL_LOGITS = 1

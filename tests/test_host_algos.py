@@ -122,6 +122,6 @@ def test_sched_rt_matches_oracle():
 
 def test_strerror_covers_all_codes():
     L = hyp.lib()
-    seen = {L.hyp_strerror(c).decode() for c in range(0, -7, -1)}
-    assert len(seen) == 7 and "unknown status" not in seen
+    seen = {L.hyp_strerror(c).decode() for c in range(0, -8, -1)}
+    assert len(seen) == 8 and "unknown status" not in seen
     assert L.hyp_strerror(-99).decode() == "unknown status"
