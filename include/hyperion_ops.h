@@ -1,0 +1,76 @@
+/*
+ * hyperion_ops.h - single-kernel entry points of libhyperion.
+ *
+ * These run one step of the decoder block (Section III-A of the paper names the steps: RMSNorm,
+ * grouped-query attention with rotary encoding, SwiGLU feed-forward) on caller-owned DEVICE buffers.
+ * They exist for unit tests, per-kernel measurement and for callers that assemble their own block
+ * sequence; hyp_stage_* (hyperion.h) is the full path.  All pointers are DEVICE unless marked HOST;
+ * `stream` is a cudaStream_t as void*; calls enqueue and return; status codes as in hyperion.h.
+ *
+ * KV page pool layout of ONE block (bf16): [n_pages][2 (K then V)][n_kv_heads][16 tokens][head_dim].
+ * A block table row lists, in order, the page ids that hold a sequence's tokens 0-15, 16-31, ...
+ */
+#ifndef HYPERION_OPS_H
+#define HYPERION_OPS_H
+
+#include "hyperion.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Epilogues of hyp_op_gemm. */
+enum {
+  HYP_EPI_STORE_BF16 = 0, /* out bf16 [M, ldo]: out[m, n] = acc                                     */
+  HYP_EPI_RESID_F32 = 1,  /* out fp32 [M, ldo]: out[m, n] += acc  (residual stream)                 */
+  HYP_EPI_SWIGLU_BF16 = 2,/* out bf16 [M, ldo]: SiLU(acc over weight row n) * (acc over row n + N); */
+                          /* w holds 2N rows: gate rows then up rows                                */
+  HYP_EPI_STORE_F32 = 3   /* out fp32 [M, ldo]: out[m, n] = acc                                     */
+};
+
+typedef struct {
+  int32_t n_q_heads, n_kv_heads, head_dim; /* head_dim 64 or 128; n_q_heads / n_kv_heads in 1,2,4,8 */
+} hyp_attn_shape;
+
+/* RMSNorm (Section III-A): out[m, :] = x[m, :] / sqrt(mean(x[m, :]^2) + eps) * g.
+ * x fp32 [M, H], g bf16 [H], out bf16 [M, H]; H multiple of 8. */
+HYP_API int hyp_op_rmsnorm(const float* x, const void* g, void* out, int32_t M, int32_t H, float eps, void* stream);
+
+/* Projection (the QKV, O, gate/up, down and LM-head contractions of the block):
+ * acc[m, n] = sum_k a[m, k] * w[n, k], bf16 inputs, fp32 accumulation, then `epilogue`.
+ * a bf16 [M, K] row-major, w bf16 [N (2N for SwiGLU), K] row-major, K multiple of 8, N multiple of 16
+ * unless M <= 32.  M <= 32 runs the weight-streaming kernel, larger M the tcgen05 tile kernel.
+ * The first call with M > 32 on a process allocates one device word for error reporting. */
+HYP_API int hyp_op_gemm(const void* a, const void* w, int32_t M, int32_t N, int32_t K, int32_t epilogue, void* out,
+                        int32_t ldo, void* stream);
+
+/* Number of context splits hyp_op_attn_decode would pick for this batch, and the scratch bytes
+ * that n_splits needs.  Pure host helpers. */
+HYP_API int hyp_op_attn_decode_splits(int32_t n_seqs, int32_t n_kv_heads, int32_t max_ctx);
+HYP_API size_t hyp_op_attn_decode_scratch_bytes(int32_t n_seqs, int32_t n_q_heads, int32_t head_dim, int32_t n_splits);
+
+/* Decode attention (grouped-query attention of Section III-A for one new token per sequence):
+ * out[b, h, :] = softmax_j(q[b, h, :] . k[b, j, h/G, :] / sqrt(D)) v[b, j, h/G, :] over cached
+ * positions j = 0 .. ctx_lens[b] (the new token's k, v must already be in the cache).
+ *   q          bf16 [n_seqs, q_stride], head h of row b at q + b*q_stride + h*D (already rotated)
+ *   kv_pages   one block's page pool (layout above)
+ *   block_table int32 [n_seqs, max_pages_per_seq];  ctx_lens int32 [n_seqs]
+ *   scratch    fp32, at least hyp_op_attn_decode_scratch_bytes(...) bytes: per-split partial results
+ *   out        bf16 [n_seqs, n_q_heads * D]
+ * n_splits in [1, 32]. */
+HYP_API int hyp_op_attn_decode(const hyp_attn_shape* shape, int32_t n_seqs, const void* q, int32_t q_stride,
+                               const void* kv_pages, const int32_t* block_table, int32_t max_pages_per_seq,
+                               const int32_t* ctx_lens, int32_t n_splits, float* scratch, size_t scratch_bytes,
+                               void* out, void* stream);
+
+/* Prefill attention: the same definition for M query rows; row t belongs to batch-local sequence
+ * tok_seq[t], sits at absolute position tok_pos[t] and sees cached positions 0 .. tok_pos[t].
+ *   q bf16 [M, q_stride]; tok_seq, tok_pos int32 [M]; out bf16 [M, n_q_heads * D]. */
+HYP_API int hyp_op_attn_prefill(const hyp_attn_shape* shape, int32_t M, const void* q, int32_t q_stride,
+                                const void* kv_pages, const int32_t* block_table, int32_t max_pages_per_seq,
+                                const int32_t* tok_seq, const int32_t* tok_pos, void* out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HYPERION_OPS_H */

@@ -57,7 +57,7 @@ attn_decode_partial_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfl
   // query heads kvh*G .. kvh*G+G-1 of row b, pre-scaled by 1/sqrt(D)
   const float scale = rsqrtf((float)D);
   float q[G][8];
-  const __nv_bfloat16* qrow = qkv + (size_t)bm.cu_q[b] * d.qkv_rows + (size_t)kvh * G * D;
+  const __nv_bfloat16* qrow = qkv + (size_t)b * d.qkv_rows + (size_t)kvh * G * D;  // decode: row b is sequence b
 #pragma unroll
   for (int gq = 0; gq < G; ++gq) {
     const uint4 v = *reinterpret_cast<const uint4*>(qrow + gq * D + dl);

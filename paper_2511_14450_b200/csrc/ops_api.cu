@@ -1,0 +1,104 @@
+// Single-kernel C entry points: argument checks, then the same launchers the stage runtime uses.
+#include "common.cuh"
+#include "gemm_tc.cuh"
+#include "hyperion_ops.h"
+
+using namespace hyp;
+
+namespace {
+
+bool attn_shape_ok(const hyp_attn_shape* s) {
+  if (!s || s->n_kv_heads < 1 || s->n_q_heads < s->n_kv_heads || s->n_q_heads % s->n_kv_heads) return false;
+  const int G = s->n_q_heads / s->n_kv_heads;
+  return (G == 1 || G == 2 || G == 4 || G == 8) && (s->head_dim == 64 || s->head_dim == 128);
+}
+
+ModelDims attn_dims(const hyp_attn_shape* s, int q_stride) {
+  ModelDims d{};
+  d.Hq = s->n_q_heads; d.Hkv = s->n_kv_heads; d.D = s->head_dim;
+  d.qkv_rows = q_stride;
+  d.page_tokens = 16;
+  return d;
+}
+
+int finish(int rc) {
+  if (rc < 0) return rc;
+  cudaError_t e = cudaPeekAtLastError();
+  if (e != cudaSuccess) {
+    set_last_cuda_error((int)e);
+    return HYP_ECUDA;
+  }
+  return HYP_OK;
+}
+
+}  // namespace
+
+extern "C" int hyp_op_rmsnorm(const float* x, const void* g, void* out, int32_t M, int32_t H, float eps, void* stream) {
+  if (!x || !g || !out || M < 1 || H < 8 || H % 8 || !(eps > 0.f)) return HYP_EINVAL;
+  return finish(launch_rmsnorm(x, (const __nv_bfloat16*)g, (__nv_bfloat16*)out, M, H, eps, nullptr, (cudaStream_t)stream));
+}
+
+extern "C" int hyp_op_gemm(const void* a, const void* w, int32_t M, int32_t N, int32_t K, int32_t epilogue, void* out,
+                           int32_t ldo, void* stream) {
+  if (!a || !w || !out || M < 1 || N < 1 || K < 8 || K % 8 || ldo < N) return HYP_EINVAL;
+  if (epilogue < HYP_EPI_STORE_BF16 || epilogue > HYP_EPI_STORE_F32) return HYP_EINVAL;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (M <= 32)
+    return finish(launch_gemm_skinny((const __nv_bfloat16*)a, K, (const __nv_bfloat16*)w, N, K, M, epilogue, out, ldo, st));
+  if (N % 16 || ldo % 8) return HYP_EINVAL;
+  int rc = tc_prepare();
+  if (rc) return rc;
+  TcAct ta;
+  TcWeight tw;
+  rc = tc_make_act(&ta, (const __nv_bfloat16*)a, M, K);
+  if (rc) return rc;
+  rc = tc_make_weight(&tw, (const __nv_bfloat16*)w, epilogue == HYP_EPI_SWIGLU_BF16 ? 2 * N : N, K);
+  if (rc) return rc;
+  return finish(launch_gemm_tc(ta, tw, M, N, K, epilogue, out, ldo, st));
+}
+
+extern "C" int hyp_op_attn_decode_splits(int32_t n_seqs, int32_t n_kv_heads, int32_t max_ctx) {
+  if (n_seqs < 1 || n_kv_heads < 1 || max_ctx < 1) return HYP_EINVAL;
+  return attn_decode_splits(n_seqs, n_kv_heads, max_ctx);
+}
+
+extern "C" size_t hyp_op_attn_decode_scratch_bytes(int32_t n_seqs, int32_t n_q_heads, int32_t head_dim,
+                                                   int32_t n_splits) {
+  if (n_seqs < 1 || n_q_heads < 1 || head_dim < 1 || n_splits < 1) return 0;
+  return attn_decode_scratch_bytes(n_seqs, n_q_heads, head_dim, n_splits);
+}
+
+extern "C" int hyp_op_attn_decode(const hyp_attn_shape* shape, int32_t n_seqs, const void* q, int32_t q_stride,
+                                  const void* kv_pages, const int32_t* block_table, int32_t max_pages_per_seq,
+                                  const int32_t* ctx_lens, int32_t n_splits, float* scratch, size_t scratch_bytes,
+                                  void* out, void* stream) {
+  if (!attn_shape_ok(shape) || !q || !kv_pages || !block_table || !ctx_lens || !scratch || !out) return HYP_EINVAL;
+  if (n_seqs < 1 || n_seqs > 65535 || max_pages_per_seq < 1 || n_splits < 1 || n_splits > 32) return HYP_EINVAL;
+  if (q_stride < shape->n_q_heads * shape->head_dim || q_stride % 8) return HYP_EINVAL;
+  if (scratch_bytes < attn_decode_scratch_bytes(n_seqs, shape->n_q_heads, shape->head_dim, n_splits)) return HYP_ECAPACITY;
+  BatchMeta bm{};
+  bm.n_seqs = n_seqs;
+  bm.n_tokens = n_seqs;
+  bm.max_pages_per_seq = max_pages_per_seq;
+  bm.ctx_lens = ctx_lens;
+  bm.block_table = block_table;
+  const ModelDims d = attn_dims(shape, q_stride);
+  return finish(launch_attn_decode((const __nv_bfloat16*)q, (const __nv_bfloat16*)kv_pages, (__nv_bfloat16*)out, scratch,
+                                   n_splits, bm, d, (cudaStream_t)stream));
+}
+
+extern "C" int hyp_op_attn_prefill(const hyp_attn_shape* shape, int32_t M, const void* q, int32_t q_stride,
+                                   const void* kv_pages, const int32_t* block_table, int32_t max_pages_per_seq,
+                                   const int32_t* tok_seq, const int32_t* tok_pos, void* out, void* stream) {
+  if (!attn_shape_ok(shape) || !q || !kv_pages || !block_table || !tok_seq || !tok_pos || !out) return HYP_EINVAL;
+  if (M < 1 || max_pages_per_seq < 1 || q_stride < shape->n_q_heads * shape->head_dim || q_stride % 8) return HYP_EINVAL;
+  BatchMeta bm{};
+  bm.n_tokens = M;
+  bm.max_pages_per_seq = max_pages_per_seq;
+  bm.tok_seq = tok_seq;
+  bm.tok_pos = tok_pos;
+  bm.block_table = block_table;
+  const ModelDims d = attn_dims(shape, q_stride);
+  return finish(launch_attn_prefill((const __nv_bfloat16*)q, (const __nv_bfloat16*)kv_pages, (__nv_bfloat16*)out, bm, d,
+                                    (cudaStream_t)stream));
+}

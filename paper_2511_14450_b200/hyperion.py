@@ -38,6 +38,10 @@ class hyp_node_state(C.Structure):
                 ("available", C.c_int32)]
 
 
+class hyp_attn_shape(C.Structure):
+    _fields_ = [("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32)]
+
+
 class HyperionError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
@@ -70,6 +74,16 @@ SIGNATURES = {
                                C.POINTER(C.c_double), C.POINTER(C.c_double), C.c_double, C.POINTER(C.c_int32),
                                C.POINTER(C.c_double)]),
     "hyp_sched_rt": (C.c_int, [C.c_double, C.c_double, C.POINTER(hyp_node_state), C.c_int32, C.POINTER(C.c_int32)]),
+    "hyp_op_rmsnorm": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_void_p]),
+    "hyp_op_gemm": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                              C.c_int32, C.c_void_p]),
+    "hyp_op_attn_decode_splits": (C.c_int, [C.c_int32, C.c_int32, C.c_int32]),
+    "hyp_op_attn_decode_scratch_bytes": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
+    "hyp_op_attn_decode": (C.c_int, [C.POINTER(hyp_attn_shape), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
+                                     C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t,
+                                     C.c_void_p, C.c_void_p]),
+    "hyp_op_attn_prefill": (C.c_int, [C.POINTER(hyp_attn_shape), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
+                                      C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "hyp_strerror": (C.c_char_p, [C.c_int]),
     "hyp_last_cuda_error": (C.c_int, []),
 }
@@ -235,6 +249,47 @@ def hyp_sched_rt(F_new: float, m_act: float, nodes) -> int:
     k = C.c_int32(-1)
     _check(lib().hyp_sched_rt(F_new, m_act, arr, len(nodes), C.byref(k)), "hyp_sched_rt")
     return k.value
+
+
+# --------------------------------------------------------------------------------------------
+# single-kernel entry points (hyperion_ops.h)
+# --------------------------------------------------------------------------------------------
+HYP_EPI_STORE_BF16, HYP_EPI_RESID_F32, HYP_EPI_SWIGLU_BF16, HYP_EPI_STORE_F32 = range(4)
+
+
+def hyp_op_rmsnorm(x, g, out, eps: float, stream=None):
+    M, H = x.shape
+    _check(lib().hyp_op_rmsnorm(_ptr(x), _ptr(g), _ptr(out), M, H, eps, _stream_handle(stream)), "hyp_op_rmsnorm")
+
+
+def hyp_op_gemm(a, w, N: int, epilogue: int, out, stream=None):
+    M, K = a.shape
+    _check(lib().hyp_op_gemm(_ptr(a), _ptr(w), M, N, K, epilogue, _ptr(out), out.stride(0), _stream_handle(stream)),
+           "hyp_op_gemm")
+
+
+def hyp_op_attn_decode_splits(n_seqs: int, n_kv_heads: int, max_ctx: int) -> int:
+    return lib().hyp_op_attn_decode_splits(n_seqs, n_kv_heads, max_ctx)
+
+
+def hyp_op_attn_decode_scratch_bytes(n_seqs: int, n_q_heads: int, head_dim: int, n_splits: int) -> int:
+    return lib().hyp_op_attn_decode_scratch_bytes(n_seqs, n_q_heads, head_dim, n_splits)
+
+
+def hyp_op_attn_decode(shape3, q, kv_pages, block_table, ctx_lens, n_splits, scratch, out, stream=None):
+    """shape3 = (n_q_heads, n_kv_heads, head_dim); tensors are CUDA tensors laid out as the header says."""
+    sh = hyp_attn_shape(*shape3)
+    _check(lib().hyp_op_attn_decode(C.byref(sh), q.shape[0], _ptr(q), q.stride(0), _ptr(kv_pages), _ptr(block_table),
+                                    block_table.stride(0), _ptr(ctx_lens), n_splits, _ptr(scratch),
+                                    scratch.numel() * scratch.element_size(), _ptr(out), _stream_handle(stream)),
+           "hyp_op_attn_decode")
+
+
+def hyp_op_attn_prefill(shape3, q, kv_pages, block_table, tok_seq, tok_pos, out, stream=None):
+    sh = hyp_attn_shape(*shape3)
+    _check(lib().hyp_op_attn_prefill(C.byref(sh), q.shape[0], _ptr(q), q.stride(0), _ptr(kv_pages), _ptr(block_table),
+                                     block_table.stride(0), _ptr(tok_seq), _ptr(tok_pos), _ptr(out),
+                                     _stream_handle(stream)), "hyp_op_attn_prefill")
 
 
 # --------------------------------------------------------------------------------------------

@@ -1,0 +1,135 @@
+"""Single-kernel parity: each kernel through its C entry point against the oracle's matching function,
+on small and ragged shapes (tile tails, page boundaries, shuffled block tables) and one full-size case."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import decoder as od
+from paper_2511_14450_b200 import hyperion as hyp
+from paper_2511_14450_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def f64(t):
+    return t.detach().cpu().to(torch.float64).numpy()
+
+
+def bf16_normal(stream, shape, std=1.0):
+    return inputs.normal_bf16(11, stream, shape, std=std, device="cuda")
+
+
+@pytest.mark.parametrize("M,H", [(1, 256), (7, 5120), (33, 1000)])
+def test_rmsnorm(M, H):
+    x = bf16_normal(1, (M, H)).float() * 3.0
+    g = inputs.uniform_bf16(11, 2, (H,), 0.5, 1.5, device="cuda")
+    out = torch.empty(M, H, dtype=torch.bfloat16, device="cuda")
+    hyp.hyp_op_rmsnorm(x, g, out, 1e-5)
+    torch.cuda.synchronize()
+    want = od.rmsnorm(f64(x), f64(g), 1e-5)
+    assert np.max(np.abs(f64(out) - want) / (np.abs(want) + 1e-2)) < 6e-3      # bf16 rounding of the output
+
+
+GEMM_SHAPES = [  # (M, N, K)
+    (1, 256, 256), (8, 512, 256), (32, 256, 688), (5, 1024, 64),          # weight-streaming kernel, K tail
+    (33, 512, 256), (128, 256, 256), (200, 1024, 688), (129, 272, 328),   # tile kernel: M, N and K tails
+    (512, 7680, 5120),                                                     # QKV projection at full size
+]
+
+
+@pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
+@pytest.mark.parametrize("epi", [hyp.HYP_EPI_STORE_BF16, hyp.HYP_EPI_RESID_F32, hyp.HYP_EPI_SWIGLU_BF16,
+                                 hyp.HYP_EPI_STORE_F32])
+def test_gemm_all_epilogues(M, N, K, epi):
+    if M == 512 and epi not in (hyp.HYP_EPI_STORE_BF16, hyp.HYP_EPI_SWIGLU_BF16):
+        pytest.skip("full-size case runs the two bf16 epilogues only")
+    swiglu = epi == hyp.HYP_EPI_SWIGLU_BF16
+    a = bf16_normal(3, (M, K))
+    w = bf16_normal(4, ((2 * N if swiglu else N), K), std=1.0 / np.sqrt(K))
+    acc = f64(a) @ f64(w).T
+    if epi in (hyp.HYP_EPI_STORE_BF16, hyp.HYP_EPI_SWIGLU_BF16):
+        out = torch.full((M, N), 7.0, dtype=torch.bfloat16, device="cuda")
+        want = od.silu(acc[:, :N]) * acc[:, N:] if swiglu else acc
+        tol = 6e-3
+    else:
+        res = bf16_normal(5, (M, N)).float()
+        out = res.clone()
+        want = acc + (f64(res) if epi == hyp.HYP_EPI_RESID_F32 else 0.0)
+        tol = 2e-5 * np.sqrt(K)
+    hyp.hyp_op_gemm(a, w, N, epi, out)
+    torch.cuda.synchronize()
+    err = np.abs(f64(out) - want) / (np.abs(want) + 1.0)
+    assert np.max(err) < tol, (np.max(err), np.unravel_index(np.argmax(err), err.shape))
+
+
+def build_cache(seq_lens, Hkv, D, seed):
+    """Random rotated keys / values for each sequence, scattered into a shuffled page pool."""
+    n = len(seq_lens)
+    mpps = max((l + 15) // 16 for l in seq_lens) + 1
+    n_pages = n * mpps + 3
+    perm = torch.from_numpy(np.random.default_rng(seed).permutation(n_pages)).to(torch.int32)
+    pool = torch.zeros(n_pages, 2, Hkv, 16, D, dtype=torch.bfloat16, device="cuda")
+    table = torch.zeros(n, mpps, dtype=torch.int32)
+    ks, vs = [], []
+    for i, L in enumerate(seq_lens):
+        k = bf16_normal(100 + 2 * i + seed, (L, Hkv, D))
+        v = bf16_normal(101 + 2 * i + seed, (L, Hkv, D))
+        ks.append(k); vs.append(v)
+        for p in range((L + 15) // 16):
+            page = int(perm[i * mpps + p])
+            table[i, p] = page
+            t0, t1 = 16 * p, min(L, 16 * p + 16)
+            pool[page, 0, :, :t1 - t0] = k[t0:t1].permute(1, 0, 2)
+            pool[page, 1, :, :t1 - t0] = v[t0:t1].permute(1, 0, 2)
+    return pool, table.cuda(), ks, vs
+
+
+@pytest.mark.parametrize("Hq,Hkv,D", [(4, 2, 64), (40, 10, 128), (8, 8, 128), (8, 1, 64)])
+@pytest.mark.parametrize("n_splits", [1, 3, 8])
+def test_attn_decode(Hq, Hkv, D, n_splits):
+    lens = [1, 15, 16, 17, 100, 333]                      # tokens visible, new one included
+    pool, table, ks, vs = build_cache(lens, Hkv, D, seed=Hq)
+    n = len(lens)
+    q_stride = (Hq + 2 * Hkv) * D                         # query rows as they sit inside a fused qkv buffer
+    q = bf16_normal(50, (n, q_stride))
+    ctx = torch.tensor([l - 1 for l in lens], dtype=torch.int32, device="cuda")
+    nbytes = hyp.hyp_op_attn_decode_scratch_bytes(n, Hq, D, n_splits)
+    scratch = torch.full((nbytes // 4,), float("nan"), dtype=torch.float32, device="cuda")
+    out = torch.empty(n, Hq * D, dtype=torch.bfloat16, device="cuda")
+    hyp.hyp_op_attn_decode((Hq, Hkv, D), q, pool, table, ctx, n_splits, scratch, out)
+    torch.cuda.synchronize()
+    for i, L in enumerate(lens):
+        qi = f64(q[i, :Hq * D]).reshape(1, Hq, D)
+        want = od.attention(qi, f64(ks[i]), f64(vs[i]), q_pos0=L - 1).reshape(-1)
+        assert np.max(np.abs(f64(out[i]) - want)) < 1.5e-2, (i, L)
+
+
+def test_attn_decode_rejects_small_scratch():
+    pool, table, _, _ = build_cache([20], 2, 64, seed=1)
+    q = bf16_normal(51, (1, 256))
+    ctx = torch.tensor([19], dtype=torch.int32, device="cuda")
+    out = torch.empty(1, 256, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(hyp.HyperionError) as ei:
+        hyp.hyp_op_attn_decode((4, 2, 64), q, pool, table, ctx, 4, torch.empty(8, device="cuda"), out)
+    assert ei.value.code == hyp.HYP_ECAPACITY
+
+
+@pytest.mark.parametrize("Hq,Hkv,D", [(4, 2, 64), (40, 10, 128)])
+def test_attn_prefill(Hq, Hkv, D):
+    lens = [37, 5, 64]                                    # cached tokens per sequence (own k, v included)
+    new = [37, 2, 20]                                     # query rows: the last `new` positions of each
+    pool, table, ks, vs = build_cache(lens, Hkv, D, seed=3)
+    M = sum(new)
+    q = bf16_normal(60, (M, Hq * D))
+    tok_seq = torch.tensor([i for i, c in enumerate(new) for _ in range(c)], dtype=torch.int32, device="cuda")
+    tok_pos = torch.tensor([lens[i] - c + t for i, c in enumerate(new) for t in range(c)], dtype=torch.int32,
+                           device="cuda")
+    out = torch.empty(M, Hq * D, dtype=torch.bfloat16, device="cuda")
+    hyp.hyp_op_attn_prefill((Hq, Hkv, D), q, pool, table, tok_seq, tok_pos, out)
+    torch.cuda.synchronize()
+    row = 0
+    for i, c in enumerate(new):
+        qi = f64(q[row:row + c]).reshape(c, Hq, D)
+        want = od.attention(qi, f64(ks[i]), f64(vs[i]), q_pos0=lens[i] - c).reshape(c, -1)
+        assert np.max(np.abs(f64(out[row:row + c]) - want)) < 1.5e-2, i
+        row += c
