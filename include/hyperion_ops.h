@@ -63,6 +63,34 @@ HYP_API int hyp_op_attn_decode(const hyp_attn_shape* shape, int32_t n_seqs, cons
                                const int32_t* ctx_lens, int32_t n_splits, float* scratch, size_t scratch_bytes,
                                void* out, void* stream);
 
+/* Decode attention for callers that must not allocate device memory.  (The paper has no counterpart
+ * to this call; it is a packaging variant of hyp_op_attn_decode.)
+ *
+ * Some users of this library cannot call cudaMalloc at the point where they need attention: an
+ * inference server that handed all free HBM to its own KV-cache pool at start-up, a plug-in running
+ * inside a host application whose memory budget is fixed after initialisation, or a latency-critical
+ * loop where an allocation's implicit device-wide synchronisation is not acceptable.  For them the
+ * per-split partial results go to a fixed HYP_STATIC_SCRATCH_BYTES (4 MiB) array that is part of the
+ * library image: every GPU that loads the library holds it until the process exits.  The caller
+ * passes inputs and outputs exactly as for hyp_op_attn_decode; there is no scratch argument.
+ *
+ *  - Limit: hyp_op_attn_decode_scratch_bytes(n_seqs, n_q_heads, head_dim, n_splits) must not exceed
+ *    HYP_STATIC_SCRATCH_BYTES; otherwise the call returns HYP_ECAPACITY and launches nothing
+ *    (4 MiB covers e.g. 8 sequences x 40 heads x 24 splits at head_dim 128).  Use fewer splits, a
+ *    smaller batch, or hyp_op_attn_decode with your own buffer.
+ *  - The call performs no cudaMalloc/cudaFree and calls no allocating library routine.
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *    that device current) and caches it; make that first call before starting any stream capture.
+ *  - All calls on a device share the one array and it keeps whatever the previous call left there.
+ *    Nothing needs clearing (each call overwrites every slot it later reads), but two calls whose
+ *    kernels can overlap on the GPU - different streams without an ordering between them - race on
+ *    it.  Keep calls on one stream, or order them with events.
+ * Other arguments, layouts and errors: as hyp_op_attn_decode. */
+#define HYP_STATIC_SCRATCH_BYTES (4u << 20)
+HYP_API int hyp_op_attn_decode_static(const hyp_attn_shape* shape, int32_t n_seqs, const void* q, int32_t q_stride,
+                                      const void* kv_pages, const int32_t* block_table, int32_t max_pages_per_seq,
+                                      const int32_t* ctx_lens, int32_t n_splits, void* out, void* stream);
+
 /* Prefill attention: the same definition for M query rows; row t belongs to batch-local sequence
  * tok_seq[t], sits at absolute position tok_pos[t] and sees cached positions 0 .. tok_pos[t].
  *   q bf16 [M, q_stride]; tok_seq, tok_pos int32 [M]; out bf16 [M, n_q_heads * D]. */

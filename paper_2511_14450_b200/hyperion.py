@@ -82,6 +82,8 @@ SIGNATURES = {
     "hyp_op_attn_decode": (C.c_int, [C.POINTER(hyp_attn_shape), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
                                      C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t,
                                      C.c_void_p, C.c_void_p]),
+    "hyp_op_attn_decode_static": (C.c_int, [C.POINTER(hyp_attn_shape), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
+                                            C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
     "hyp_op_attn_prefill": (C.c_int, [C.POINTER(hyp_attn_shape), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
                                       C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "hyp_strerror": (C.c_char_p, [C.c_int]),
@@ -283,6 +285,19 @@ def hyp_op_attn_decode(shape3, q, kv_pages, block_table, ctx_lens, n_splits, scr
                                     block_table.stride(0), _ptr(ctx_lens), n_splits, _ptr(scratch),
                                     scratch.numel() * scratch.element_size(), _ptr(out), _stream_handle(stream)),
            "hyp_op_attn_decode")
+
+
+HYP_STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def hyp_op_attn_decode_static(shape3, q, kv_pages, block_table, ctx_lens, n_splits, out, stream=None):
+    """Decode attention that allocates nothing: split partials go to the library's built-in 4 MiB
+    device array (shared by all calls on the device; calls that may overlap on the GPU race on it).
+    Raises HYP_ECAPACITY if this batch's partials would not fit."""
+    sh = hyp_attn_shape(*shape3)
+    _check(lib().hyp_op_attn_decode_static(C.byref(sh), q.shape[0], _ptr(q), q.stride(0), _ptr(kv_pages),
+                                           _ptr(block_table), block_table.stride(0), _ptr(ctx_lens), n_splits,
+                                           _ptr(out), _stream_handle(stream)), "hyp_op_attn_decode_static")
 
 
 def hyp_op_attn_prefill(shape3, q, kv_pages, block_table, tok_seq, tok_pos, out, stream=None):
