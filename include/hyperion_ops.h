@@ -91,12 +91,16 @@ HYP_API int hyp_op_attn_decode_static(const hyp_attn_shape* shape, int32_t n_seq
                                       const void* kv_pages, const int32_t* block_table, int32_t max_pages_per_seq,
                                       const int32_t* ctx_lens, int32_t n_splits, void* out, void* stream);
 
-/* Prefill attention: the same definition for M query rows; row t belongs to batch-local sequence
- * tok_seq[t], sits at absolute position tok_pos[t] and sees cached positions 0 .. tok_pos[t].
- *   q bf16 [M, q_stride]; tok_seq, tok_pos int32 [M]; out bf16 [M, n_q_heads * D]. */
-HYP_API int hyp_op_attn_prefill(const hyp_attn_shape* shape, int32_t M, const void* q, int32_t q_stride,
-                                const void* kv_pages, const int32_t* block_table, int32_t max_pages_per_seq,
-                                const int32_t* tok_seq, const int32_t* tok_pos, void* out, void* stream);
+/* Prefill attention: the same definition for M query rows packed sequence by sequence.  Sequence i
+ * owns rows cu_q[i] .. cu_q[i+1]-1; its row r sits at absolute position ctx_lens[i] + (r - cu_q[i]) and
+ * sees cached positions 0 .. its own (all of the sequence's k, v, new rows included, must already be in
+ * the cache).
+ *   q bf16 [M, q_stride]; cu_q int32 [n_seqs + 1] (cu_q[n_seqs] = M); ctx_lens int32 [n_seqs];
+ *   block_table int32 [n_seqs, max_pages_per_seq]; out bf16 [M, n_q_heads * D]. */
+HYP_API int hyp_op_attn_prefill(const hyp_attn_shape* shape, int32_t n_seqs, int32_t M, const void* q,
+                                int32_t q_stride, const void* kv_pages, const int32_t* block_table,
+                                int32_t max_pages_per_seq, const int32_t* cu_q, const int32_t* ctx_lens, void* out,
+                                void* stream);
 
 #ifdef __cplusplus
 }

@@ -1,68 +1,249 @@
-// Prefill attention over the paged KV cache: causal, grouped-query, fp32 softmax.
-// Query row t of sequence s sits at absolute position tok_pos[t] and sees cached positions
-// 0 .. tok_pos[t] (its own k, v were appended by the RoPE/KV-write kernel beforehand).
+// Prefill attention over the paged KV cache: causal, grouped-query, fp32 online softmax.
+//
+// Flash-attention tiling on tensor cores: one CTA = 64 query rows of one sequence and one query head
+// (4 warps x 16 rows); keys/values stream through shared memory in 64-token tiles (4 pages) with
+// double-buffered cp.async; S = Q K^T and O += P V run on mma.sync.m16n8k16 (bf16 in, fp32 accumulate),
+// the probabilities never leave registers.  New rows of a sequence sit at positions
+// ctx_len .. ctx_len + q_len - 1 and see every cached position up to their own (their k, v were
+// appended by the RoPE / KV-write kernel beforehand), so chunked prefill needs no special case.
 #include "common.cuh"
 #include "hyperion.h"
 
 namespace hyp {
 
-// Simple kernel: one warp per (row, query head); lanes split the head dimension.
-template <int D>
-__global__ void attn_prefill_rowwarp_kernel(const __nv_bfloat16* __restrict__ qkv,
-                                            const __nv_bfloat16* __restrict__ kv_layer,
-                                            __nv_bfloat16* __restrict__ out, BatchMeta bm, ModelDims d) {
-  constexpr int EPL = D / 32;  // elements per lane
-  constexpr int PT = 16;
-  const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  if (warp_global >= bm.n_tokens * d.Hq) return;
-  const int t = warp_global / d.Hq, hq = warp_global % d.Hq;
-  const int kvh = hq / (d.Hq / d.Hkv);
-  const int pos = bm.tok_pos[t];
-  const int32_t* bt = bm.block_table + (size_t)bm.tok_seq[t] * bm.max_pages_per_seq;
-  const size_t page_elems = kv_page_elems(d.Hkv, PT, D);
-  const size_t v_off = (size_t)d.Hkv * PT * D;
-  const float scale = rsqrtf((float)D);
+namespace {
 
-  float q[EPL], acc[EPL];
-  const __nv_bfloat16* qp = qkv + (size_t)t * d.qkv_rows + (size_t)hq * D + lane * EPL;
-#pragma unroll
-  for (int e = 0; e < EPL; ++e) {
-    q[e] = __bfloat162float(qp[e]) * scale;
-    acc[e] = 0.f;
-  }
-  float m = -1e30f, l = 0.f;
-  for (int j = 0; j <= pos; ++j) {
-    const __nv_bfloat16* kp =
-        kv_layer + (size_t)bt[j / PT] * page_elems + ((size_t)kvh * PT + (j % PT)) * D + lane * EPL;
-    float s = 0.f;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) s += q[e] * __bfloat162float(kp[e]);
-    s = warp_sum(s);
-    const float m_new = fmaxf(m, s);
-    const float corr = __expf(m - m_new), p = __expf(s - m_new);
-    l = l * corr + p;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) acc[e] = acc[e] * corr + p * __bfloat162float(kp[v_off + e]);
-    m = m_new;
-  }
-  __nv_bfloat16* op = out + (size_t)t * d.Hq * D + (size_t)hq * D + lane * EPL;
-#pragma unroll
-  for (int e = 0; e < EPL; ++e) op[e] = __float2bfloat16_rn(acc[e] / l);
+constexpr int FA_BQ = 64, FA_BKV = 64, FA_THREADS = 128, PT = 16;
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
+  const int sz = valid ? 16 : 0;  // size 0 zero-fills the 16 destination bytes
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
 }
 
+// Byte offset of 16-byte chunk `c` of row `r` in a [64][D] bf16 tile; chunks are XOR-swizzled by the row
+// so that ldmatrix reads of 8 consecutive rows hit 8 different bank groups.
+template <int D>
+__device__ __forceinline__ uint32_t tile_off(int r, int c) {
+  return (uint32_t)(r * (D * 2) + ((c ^ (r & 7)) << 4));
+}
+
+template <int D>
+__global__ void __launch_bounds__(FA_THREADS)
+attn_prefill_fa_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfloat16* __restrict__ kv_layer,
+                       __nv_bfloat16* __restrict__ out, BatchMeta bm, ModelDims d) {
+  constexpr int KS = D / 16;       // k-steps of the QK^T contraction
+  constexpr int DN = D / 8;        // 8-wide output column tiles of O
+  constexpr int CPR = D / 8;       // 16-byte chunks per K/V row
+  constexpr int TILE_BYTES = FA_BKV * D * 2;
+  extern __shared__ __align__(128) uint8_t fa_smem[];
+  const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(fa_smem);
+  // layout: K[2] then V[2]
+  auto k_tile = [&](int buf) { return smem0 + buf * TILE_BYTES; };
+  auto v_tile = [&](int buf) { return smem0 + (2 + buf) * TILE_BYTES; };
+
+  // which (sequence, query tile) is this CTA?
+  int t = blockIdx.x, seq = -1, q0 = 0, q_len = 0;
+  for (int i = 0; i < bm.n_seqs; ++i) {
+    const int ql = bm.cu_q[i + 1] - bm.cu_q[i];
+    const int nt = (ql + FA_BQ - 1) / FA_BQ;
+    if (t < nt) { seq = i; q0 = t * FA_BQ; q_len = ql; break; }
+    t -= nt;
+  }
+  if (seq < 0) return;
+  const int hq = blockIdx.y;
+  const int kvh = hq / (d.Hq / d.Hkv);
+  const int ctx = bm.ctx_lens[seq];
+  const int row_base = bm.cu_q[seq] + q0;               // first packed row of this tile
+  const int rows_here = min(FA_BQ, q_len - q0);
+  const int kv_total = ctx + q0 + rows_here;             // keys this tile may need: positions < kv_total
+  const int n_kv_tiles = (kv_total + FA_BKV - 1) / FA_BKV;
+  const int32_t* bt = bm.block_table + (size_t)seq * bm.max_pages_per_seq;
+  const size_t page_elems = kv_page_elems(d.Hkv, PT, D);
+  const size_t v_off = (size_t)d.Hkv * PT * D;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, tq = lane & 3;
+
+  auto load_kv_tile = [&](int j, int buf) {
+    // 64 keys x CPR chunks for K and the same for V; 128 threads
+    for (int idx = threadIdx.x; idx < FA_BKV * CPR; idx += FA_THREADS) {
+      const int r = idx / CPR, c = idx % CPR;
+      const int key = j * FA_BKV + r;
+      const bool ok = key < kv_total;
+      const int kk = ok ? key : 0;
+      const __nv_bfloat16* src =
+          kv_layer + (size_t)bt[kk / PT] * page_elems + ((size_t)kvh * PT + (kk % PT)) * D + c * 8;
+      cp_async16(k_tile(buf) + tile_off<D>(r, c), src, ok);
+      cp_async16(v_tile(buf) + tile_off<D>(r, c), src + v_off, ok);
+    }
+  };
+
+  load_kv_tile(0, 0);
+  cp_async_commit();
+
+  // Q fragments of this warp's 16 rows, straight from global memory
+  uint32_t qf[KS][4];
+  {
+    const int r_lo = 16 * warp + g, r_hi = r_lo + 8;
+    const __nv_bfloat16* q_lo = qkv + (size_t)(row_base + r_lo) * d.qkv_rows + (size_t)hq * D;
+    const __nv_bfloat16* q_hi = qkv + (size_t)(row_base + r_hi) * d.qkv_rows + (size_t)hq * D;
+    const bool ok_lo = r_lo < rows_here, ok_hi = r_hi < rows_here;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      qf[ks][0] = ok_lo ? *reinterpret_cast<const uint32_t*>(q_lo + 16 * ks + 2 * tq) : 0u;
+      qf[ks][1] = ok_hi ? *reinterpret_cast<const uint32_t*>(q_hi + 16 * ks + 2 * tq) : 0u;
+      qf[ks][2] = ok_lo ? *reinterpret_cast<const uint32_t*>(q_lo + 16 * ks + 8 + 2 * tq) : 0u;
+      qf[ks][3] = ok_hi ? *reinterpret_cast<const uint32_t*>(q_hi + 16 * ks + 8 + 2 * tq) : 0u;
+    }
+  }
+
+  const float sl2 = rsqrtf((float)D) * 1.4426950408889634f;  // scores are kept in log2 units
+  // absolute positions of this thread's two rows (rows past the end are clamped: computed, never stored)
+  const int pos_lo = ctx + q0 + min(16 * warp + g, rows_here - 1);
+  const int pos_hi = ctx + q0 + min(16 * warp + g + 8, rows_here - 1);
+
+  float o[DN][4];
+#pragma unroll
+  for (int i = 0; i < DN; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+  float m_lo = -1e30f, m_hi = -1e30f, l_lo = 0.f, l_hi = 0.f;
+
+  for (int j = 0; j < n_kv_tiles; ++j) {
+    const int buf = j & 1;
+    if (j + 1 < n_kv_tiles) load_kv_tile(j + 1, buf ^ 1);
+    cp_async_commit();
+    cp_async_wait<1>();
+    __syncthreads();
+
+    // ---- S = Q K^T (16 rows x 64 keys per warp) ----
+    float s[8][4];
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) { s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f; }
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+      for (int np = 0; np < 4; ++np) {  // pairs of 8-key tiles
+        const int r = 16 * np + (lane & 7) + ((lane >> 4) << 3);
+        const int c = 2 * ks + ((lane >> 3) & 1);
+        uint32_t b0, b1, b2, b3;
+        ldsm_x4(k_tile(buf) + tile_off<D>(r, c), b0, b1, b2, b3);
+        mma_bf16_16816(s[2 * np], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b0, b1);
+        mma_bf16_16816(s[2 * np + 1], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b2, b3);
+      }
+    }
+
+    // ---- scale, causal mask, online softmax ----
+    const int key0 = j * FA_BKV;
+    const bool need_mask = key0 + FA_BKV - 1 > ctx + q0;  // some key of the tile may lie past a row's position
+    float mx_lo = m_lo, mx_hi = m_hi;
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float v = s[nt][e] * sl2;
+        if (need_mask) {
+          const int key = key0 + 8 * nt + 2 * tq + (e & 1);
+          if (key > ((e < 2) ? pos_lo : pos_hi)) v = -1e30f;
+        }
+        s[nt][e] = v;
+      }
+      mx_lo = fmaxf(mx_lo, fmaxf(s[nt][0], s[nt][1]));
+      mx_hi = fmaxf(mx_hi, fmaxf(s[nt][2], s[nt][3]));
+    }
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+    const float corr_lo = exp2f(m_lo - mx_lo), corr_hi = exp2f(m_hi - mx_hi);
+    m_lo = mx_lo;
+    m_hi = mx_hi;
+    float sum_lo = 0.f, sum_hi = 0.f;
+    uint32_t pf[8][2];  // probabilities as bf16 pairs: [key tile][row lo / hi]
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+      const float p0 = exp2f(s[nt][0] - mx_lo), p1 = exp2f(s[nt][1] - mx_lo);
+      const float p2 = exp2f(s[nt][2] - mx_hi), p3 = exp2f(s[nt][3] - mx_hi);
+      sum_lo += p0 + p1;
+      sum_hi += p2 + p3;
+      pf[nt][0] = pack_bf16(p0, p1);
+      pf[nt][1] = pack_bf16(p2, p3);
+    }
+    l_lo = l_lo * corr_lo + sum_lo;
+    l_hi = l_hi * corr_hi + sum_hi;
+#pragma unroll
+    for (int dn = 0; dn < DN; ++dn) {
+      o[dn][0] *= corr_lo; o[dn][1] *= corr_lo;
+      o[dn][2] *= corr_hi; o[dn][3] *= corr_hi;
+    }
+
+    // ---- O += P V ----
+#pragma unroll
+    for (int kk = 0; kk < FA_BKV / 16; ++kk) {
+#pragma unroll
+      for (int dp = 0; dp < DN / 2; ++dp) {  // pairs of 8-wide output column tiles
+        const int r = 16 * kk + (lane & 7) + (((lane >> 3) & 1) << 3);
+        const int c = 2 * dp + (lane >> 4);
+        uint32_t b0, b1, b2, b3;
+        ldsm_x4_t(v_tile(buf) + tile_off<D>(r, c), b0, b1, b2, b3);
+        mma_bf16_16816(o[2 * dp], pf[2 * kk][0], pf[2 * kk][1], pf[2 * kk + 1][0], pf[2 * kk + 1][1], b0, b1);
+        mma_bf16_16816(o[2 * dp + 1], pf[2 * kk][0], pf[2 * kk][1], pf[2 * kk + 1][0], pf[2 * kk + 1][1], b2, b3);
+      }
+    }
+    __syncthreads();  // everyone is done with `buf` before the next iteration's loads overwrite it
+  }
+  cp_async_wait<0>();
+
+  // row sums live spread over the 4 lanes of a quad
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+  const float inv_lo = 1.f / l_lo, inv_hi = 1.f / l_hi;
+  const int r_lo = 16 * warp + g, r_hi = r_lo + 8;
+  __nv_bfloat16* o_lo = out + (size_t)(row_base + r_lo) * d.Hq * D + (size_t)hq * D;
+  __nv_bfloat16* o_hi = out + (size_t)(row_base + r_hi) * d.Hq * D + (size_t)hq * D;
+#pragma unroll
+  for (int dn = 0; dn < DN; ++dn) {
+    if (r_lo < rows_here)
+      *reinterpret_cast<uint32_t*>(o_lo + 8 * dn + 2 * tq) = pack_bf16(o[dn][0] * inv_lo, o[dn][1] * inv_lo);
+    if (r_hi < rows_here)
+      *reinterpret_cast<uint32_t*>(o_hi + 8 * dn + 2 * tq) = pack_bf16(o[dn][2] * inv_hi, o[dn][3] * inv_hi);
+  }
+}
+
+template <int D>
+int launch_fa(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __nv_bfloat16* attn_out, const BatchMeta& bm,
+              const ModelDims& d, cudaStream_t st) {
+  static bool configured = false;
+  constexpr int smem = 4 * FA_BKV * D * 2;
+  if (!configured) {
+    HYP_CUDA_TRY(cudaFuncSetAttribute(attn_prefill_fa_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    configured = true;
+  }
+  // every sequence adds at most one ragged tile on top of floor(rows / 64)
+  const int max_tiles = bm.n_tokens / FA_BQ + bm.n_seqs;
+  attn_prefill_fa_kernel<D><<<dim3(max_tiles, d.Hq), FA_THREADS, smem, st>>>(qkv, kv_layer, attn_out, bm, d);
+  return 1;
+}
+
+}  // namespace
+
+// Needs bm.cu_q, bm.ctx_lens, bm.block_table, bm.n_seqs, bm.n_tokens.
 int launch_attn_prefill(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __nv_bfloat16* attn_out,
                         const BatchMeta& bm, const ModelDims& d, cudaStream_t st) {
-  const long warps = (long)bm.n_tokens * d.Hq;
-  const int block = 128;
-  const int grid = (int)((warps * 32 + block - 1) / block);
-  if (d.D == 128)
-    attn_prefill_rowwarp_kernel<128><<<grid, block, 0, st>>>(qkv, kv_layer, attn_out, bm, d);
-  else if (d.D == 64)
-    attn_prefill_rowwarp_kernel<64><<<grid, block, 0, st>>>(qkv, kv_layer, attn_out, bm, d);
-  else
-    return HYP_EINVAL;
-  return 1;
+  if (d.D == 128) return launch_fa<128>(qkv, kv_layer, attn_out, bm, d, st);
+  if (d.D == 64) return launch_fa<64>(qkv, kv_layer, attn_out, bm, d, st);
+  return HYP_EINVAL;
 }
 
 }  // namespace hyp

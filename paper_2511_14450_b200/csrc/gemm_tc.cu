@@ -9,6 +9,11 @@
 //            SiLU(gate) * up, fp32 store) straight to global memory.
 // For the SwiGLU epilogue the 256 accumulator columns are 128 gate columns and the 128 matching up
 // columns (two weight boxes per stage), so gate and up never leave the chip.
+// Work split: for the bf16 / fp32-store epilogues each CTA takes whole output tiles.  For the residual
+// epilogue (out += acc) the k-blocks of all tiles form one list that is cut into equal contiguous
+// ranges, one per CTA ("stream-K"); a CTA that holds only part of a tile's k range adds its partial
+// sum with fp32 reductions, so 80 tiles still keep 148 SMs busy (used up to 2048 rows).  The order of
+// those additions is not fixed, so the last bits of a split tile can differ between runs.
 // Every mbarrier wait is bounded: on expiry the kernel records an error code and unwinds.
 #include <cuda.h>
 
@@ -104,9 +109,61 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 256.
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
+// Walks the work of one CTA as a sequence of (tile, k-block range) segments.  All three roles of a CTA
+// run the same walk, so they agree on the order without communicating.
+//
+// Stream-K mode: CTAs form teams of `team` members; member j of a team owns M-tile (group * team + j).
+// The list of (M-tile group, N-tile, k-block) columns is cut into equal contiguous ranges, one per team,
+// so the members of a team walk the same weight k-blocks at the same time (one HBM fetch, the rest L2
+// hits) and every CTA gets the same number of k-blocks.
+struct Segments {
+  long u, u_end;  // stream-K: position in the column list
+  int tile, n_tiles, stride, KB, tiles_m, tiles_n, team, member;
+  bool streamk;
+  __device__ Segments(bool sk, int tiles_m_, int tiles_n_, int KB_, int team_)
+      : n_tiles(tiles_m_ * tiles_n_), KB(KB_), tiles_m(tiles_m_), tiles_n(tiles_n_), team(team_), streamk(sk) {
+    if (sk) {
+      const int n_teams = gridDim.x / team_;
+      const int my_team = blockIdx.x / team_;
+      member = blockIdx.x % team_;
+      const long total = (long)(tiles_m_ / team_) * tiles_n_ * KB_;
+      u = total * my_team / n_teams;
+      u_end = total * (my_team + 1) / n_teams;
+    } else {
+      tile = blockIdx.x;
+      stride = gridDim.x;
+    }
+  }
+  __device__ bool next(int& t, int& kb0, int& kb1) {
+    if (streamk) {
+      if (u >= u_end) return false;
+      const long per_group = (long)tiles_n * KB;
+      const int mg = (int)(u / per_group);
+      const long rem = u % per_group;
+      const int nt = (int)(rem / KB);
+      kb0 = (int)(rem % KB);
+      const long room = u_end - u;
+      kb1 = (KB - kb0 < room) ? KB : kb0 + (int)room;
+      u += kb1 - kb0;
+      t = nt * tiles_m + mg * team + member;
+      return true;
+    }
+    if (tile >= n_tiles) return false;
+    t = tile;
+    kb0 = 0;
+    kb1 = KB;
+    tile += stride;
+    return true;
+  }
+};
+
+__device__ __forceinline__ void red_add_f32x4(float* p, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
 template <int EPI>
 __device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[16], const uint32_t (&v2)[16], void* out, int ldo,
-                                               int row, int col, int N) {
+                                               int row, int col, int N, bool partial) {
   const size_t o = (size_t)row * ldo + col;
   const bool full = col + 16 <= N;
   if (EPI == EPI_STORE_BF16 || EPI == EPI_SWIGLU_BF16) {
@@ -130,7 +187,19 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[16], const ui
     }
   } else {
     float* p = reinterpret_cast<float*>(out) + o;
-    if (full) {
+    if (EPI == EPI_RESID_F32 && partial) {
+      // this CTA holds only part of the tile's k range: add, never overwrite
+      if (full) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          red_add_f32x4(p + 4 * i, __uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                        __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+      } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          if (col + i < N) atomicAdd(p + i, __uint_as_float(v[i]));
+      }
+    } else if (full) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         float4 a = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
@@ -152,8 +221,9 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[16], const ui
 template <int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int M, int N, int K,
-               void* __restrict__ out, int ldo, int* __restrict__ err) {
+               void* __restrict__ out, int ldo, int team, int* __restrict__ err) {
   constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
+  const bool STREAMK = EPI == EPI_RESID_F32 && team > 0;
   constexpr int BN_OUT = SWIGLU ? BN / 2 : BN;  // output columns per tile
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -170,7 +240,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN_OUT - 1) / BN_OUT;
-  const int n_tiles = tiles_m * tiles_n;
   const int KB = (K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
@@ -200,11 +269,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      Segments seg(STREAMK, tiles_m, tiles_n, KB, team);
+      int tile, kb0, kb1;
+      while (ok && seg.next(tile, kb0, kb1)) {
         const int m0 = (tile % tiles_m) * BM;
         const int n0 = (tile / tiles_m) * BN_OUT;
         const int rb0 = n0, rb1 = SWIGLU ? N + n0 : n0 + 128;
-        for (int kb = 0; kb < KB; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) { ok = false; break; }
           const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
           mbar_expect_tx(full_bar(stage), STAGE_BYTES);
@@ -225,11 +296,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      Segments seg(STREAMK, tiles_m, tiles_n, KB, team);
+      int tile, kb0, kb1;
+      while (ok && seg.next(tile, kb0, kb1)) {
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = 0; kb < KB; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
@@ -237,7 +310,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k)
             tc_mma(d_tmem, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), IDESC,
-                   (kb | k) != 0 ? 1u : 0u);
+                   (kb > kb0 || k > 0) ? 1u : 0u);
           tc_commit(empty_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -257,9 +330,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+    Segments seg(STREAMK, tiles_m, tiles_n, KB, team);
+    int tile, kb0, kb1;
+    while (ok && seg.next(tile, kb0, kb1)) {
       const int m0 = (tile % tiles_m) * BM;
       const int n0 = (tile / tiles_m) * BN_OUT;
+      const bool partial = kb0 != 0 || kb1 != KB;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int row = m0 + 32 * q + lane;
@@ -271,7 +347,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         tmem_ld16(t0 + c, v);
         if (SWIGLU) tmem_ld16(t0 + BN / 2 + c, v2);
         tmem_ld_wait();
-        if (row < M) epilogue_chunk<EPI>(v, v2, out, ldo, row, n0 + c, N);
+        if (row < M) epilogue_chunk<EPI>(v, v2, out, ldo, row, n0 + c, N, partial);
       }
       tc_fence_before();
       mbar_arrive(tempty_bar(acc));
@@ -344,9 +420,27 @@ int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
     configured = true;
   }
   constexpr int BN_OUT = EPI == EPI_SWIGLU_BF16 ? BN / 2 : BN;
-  const int tiles = ((M + BM - 1) / BM) * ((N + BN_OUT - 1) / BN_OUT);
-  const int grid = tiles < num_sms ? tiles : num_sms;
-  gemm_tc_kernel<EPI><<<grid, TC_THREADS, SMEM_BYTES, st>>>(act.map, w.map, M, N, K, out, ldo, g_err_flag);
+  const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN_OUT - 1) / BN_OUT;
+  int grid, team = 0;  // team 0 = whole tiles per CTA
+  if (EPI == EPI_RESID_F32 && tiles_m <= 16) {
+    // stream-K (up to 2048 rows; beyond that whole tiles already balance and reuse A better): pick the team size (a divisor of tiles_m) that keeps most SMs busy, larger teams preferred
+    double best = -1.0;
+    team = 1;
+    for (int ts = 1; ts <= tiles_m && ts <= num_sms; ++ts) {
+      if (tiles_m % ts) continue;
+      const int teams = num_sms / ts;
+      const double score = (double)(teams * ts) / num_sms + 0.003 * ts;
+      if (score > best) { best = score; team = ts; }
+    }
+    long teams = num_sms / team;
+    const long cols = (long)(tiles_m / team) * tiles_n * ((K + BK - 1) / BK);
+    if (teams > cols) teams = cols;
+    grid = (int)teams * team;
+  } else {
+    const long tiles = (long)tiles_m * tiles_n;
+    grid = (int)(tiles < num_sms ? tiles : num_sms);
+  }
+  gemm_tc_kernel<EPI><<<grid, TC_THREADS, SMEM_BYTES, st>>>(act.map, w.map, M, N, K, out, ldo, team, g_err_flag);
   return 1;
 }
 

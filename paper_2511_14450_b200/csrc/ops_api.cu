@@ -87,16 +87,19 @@ extern "C" int hyp_op_attn_decode(const hyp_attn_shape* shape, int32_t n_seqs, c
                                    n_splits, bm, d, (cudaStream_t)stream));
 }
 
-extern "C" int hyp_op_attn_prefill(const hyp_attn_shape* shape, int32_t M, const void* q, int32_t q_stride,
-                                   const void* kv_pages, const int32_t* block_table, int32_t max_pages_per_seq,
-                                   const int32_t* tok_seq, const int32_t* tok_pos, void* out, void* stream) {
-  if (!attn_shape_ok(shape) || !q || !kv_pages || !block_table || !tok_seq || !tok_pos || !out) return HYP_EINVAL;
-  if (M < 1 || max_pages_per_seq < 1 || q_stride < shape->n_q_heads * shape->head_dim || q_stride % 8) return HYP_EINVAL;
+extern "C" int hyp_op_attn_prefill(const hyp_attn_shape* shape, int32_t n_seqs, int32_t M, const void* q,
+                                   int32_t q_stride, const void* kv_pages, const int32_t* block_table,
+                                   int32_t max_pages_per_seq, const int32_t* cu_q, const int32_t* ctx_lens, void* out,
+                                   void* stream) {
+  if (!attn_shape_ok(shape) || !q || !kv_pages || !block_table || !cu_q || !ctx_lens || !out) return HYP_EINVAL;
+  if (n_seqs < 1 || M < n_seqs || max_pages_per_seq < 1) return HYP_EINVAL;
+  if (q_stride < shape->n_q_heads * shape->head_dim || q_stride % 8) return HYP_EINVAL;
   BatchMeta bm{};
+  bm.n_seqs = n_seqs;
   bm.n_tokens = M;
   bm.max_pages_per_seq = max_pages_per_seq;
-  bm.tok_seq = tok_seq;
-  bm.tok_pos = tok_pos;
+  bm.cu_q = cu_q;
+  bm.ctx_lens = ctx_lens;
   bm.block_table = block_table;
   const ModelDims d = attn_dims(shape, q_stride);
   return finish(launch_attn_prefill((const __nv_bfloat16*)q, (const __nv_bfloat16*)kv_pages, (__nv_bfloat16*)out, bm, d,

@@ -84,8 +84,9 @@ SIGNATURES = {
                                      C.c_void_p, C.c_void_p]),
     "hyp_op_attn_decode_static": (C.c_int, [C.POINTER(hyp_attn_shape), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
                                             C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
-    "hyp_op_attn_prefill": (C.c_int, [C.POINTER(hyp_attn_shape), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
-                                      C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "hyp_op_attn_prefill": (C.c_int, [C.POINTER(hyp_attn_shape), C.c_int32, C.c_int32, C.c_void_p, C.c_int32,
+                                      C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                      C.c_void_p]),
     "hyp_strerror": (C.c_char_p, [C.c_int]),
     "hyp_last_cuda_error": (C.c_int, []),
 }
@@ -300,10 +301,10 @@ def hyp_op_attn_decode_static(shape3, q, kv_pages, block_table, ctx_lens, n_spli
                                            _ptr(out), _stream_handle(stream)), "hyp_op_attn_decode_static")
 
 
-def hyp_op_attn_prefill(shape3, q, kv_pages, block_table, tok_seq, tok_pos, out, stream=None):
+def hyp_op_attn_prefill(shape3, q, kv_pages, block_table, cu_q, ctx_lens, out, stream=None):
     sh = hyp_attn_shape(*shape3)
-    _check(lib().hyp_op_attn_prefill(C.byref(sh), q.shape[0], _ptr(q), q.stride(0), _ptr(kv_pages), _ptr(block_table),
-                                     block_table.stride(0), _ptr(tok_seq), _ptr(tok_pos), _ptr(out),
+    _check(lib().hyp_op_attn_prefill(C.byref(sh), ctx_lens.shape[0], q.shape[0], _ptr(q), q.stride(0), _ptr(kv_pages),
+                                     _ptr(block_table), block_table.stride(0), _ptr(cu_q), _ptr(ctx_lens), _ptr(out),
                                      _stream_handle(stream)), "hyp_op_attn_prefill")
 
 

@@ -114,22 +114,22 @@ def test_attn_decode_rejects_small_scratch():
     assert ei.value.code == hyp.HYP_ECAPACITY
 
 
-@pytest.mark.parametrize("Hq,Hkv,D", [(4, 2, 64), (40, 10, 128)])
-def test_attn_prefill(Hq, Hkv, D):
-    lens = [37, 5, 64]                                    # cached tokens per sequence (own k, v included)
-    new = [37, 2, 20]                                     # query rows: the last `new` positions of each
+@pytest.mark.parametrize("Hq,Hkv,D", [(4, 2, 64), (40, 10, 128), (8, 8, 64)])
+@pytest.mark.parametrize("lens,new", [([37, 5, 64], [37, 2, 20]), ([300, 129, 1, 64], [300, 65, 1, 64])])
+def test_attn_prefill(Hq, Hkv, D, lens, new):
+    # lens: cached tokens per sequence (own k, v included); new: query rows = the last `new` positions
     pool, table, ks, vs = build_cache(lens, Hkv, D, seed=3)
     M = sum(new)
     q = bf16_normal(60, (M, Hq * D))
-    tok_seq = torch.tensor([i for i, c in enumerate(new) for _ in range(c)], dtype=torch.int32, device="cuda")
-    tok_pos = torch.tensor([lens[i] - c + t for i, c in enumerate(new) for t in range(c)], dtype=torch.int32,
-                           device="cuda")
-    out = torch.empty(M, Hq * D, dtype=torch.bfloat16, device="cuda")
-    hyp.hyp_op_attn_prefill((Hq, Hkv, D), q, pool, table, tok_seq, tok_pos, out)
+    cu = np.concatenate([[0], np.cumsum(new)]).astype(np.int32)
+    cu_q = torch.from_numpy(cu).cuda()
+    ctx = torch.tensor([l - c for l, c in zip(lens, new)], dtype=torch.int32, device="cuda")
+    out = torch.full((M, Hq * D), 5.0, dtype=torch.bfloat16, device="cuda")
+    hyp.hyp_op_attn_prefill((Hq, Hkv, D), q, pool, table, cu_q, ctx, out)
     torch.cuda.synchronize()
     row = 0
     for i, c in enumerate(new):
         qi = f64(q[row:row + c]).reshape(c, Hq, D)
         want = od.attention(qi, f64(ks[i]), f64(vs[i]), q_pos0=lens[i] - c).reshape(c, -1)
-        assert np.max(np.abs(f64(out[row:row + c]) - want)) < 1.5e-2, i
+        assert np.max(np.abs(f64(out[row:row + c]) - want)) < 2e-2, i
         row += c
