@@ -1,21 +1,24 @@
 // Decode attention: one query row per sequence against its paged KV cache, split along the
 // context so that a small batch still fills the GPU, followed by a log-sum-exp merge.
 //
-//   partial kernel: grid (n_splits, Hkv, n_seqs).  A CTA streams its context slice of one KV head
-//   once with 128-bit loads and serves all G = Hq/Hkv query heads that share it.  Each group of
-//   D/8 lanes owns one token per iteration; the dot product is finished with warp shuffles and a
-//   running (max, sum, weighted V) state is kept in fp32 per lane group, then combined in shared
-//   memory.
+//   partial kernel: grid (n_splits, Hkv, n_seqs), 4 warps.  A CTA streams its context slice of one KV
+//   head through shared memory in 64-token tiles (double-buffered cp.async, 128-bit, each byte read
+//   once) and serves the G = Hq/Hkv query heads that share the head as the rows of one
+//   mma.sync.m16n8k16 operand (rows >= G are padding).  Warp w owns keys 16w..16w+15 of every tile:
+//   it forms their scores, keeps its own online-softmax state and its own O += P V partial, so there is
+//   no cross-warp traffic inside the loop; the four warps are combined once at the end.  Tensor cores
+//   are used because the scalar version needs ~130 instructions per KB of cache and is issue-bound at
+//   HBM speed; the roofline of this kernel is HBM.
 //   merge kernel: grid (n_seqs * Hq).  Combines the split partials and writes bf16.
 //
 // Scratch layout (fp32): acc [n_seqs][Hq][n_splits][D], then ml [n_seqs][Hq][n_splits][2].
-#include "common.cuh"
+#include "attn_common.cuh"
 #include "hyperion.h"
 
 namespace hyp {
 
 constexpr int AD_WARPS = 4;
-constexpr int AD_UNROLL = 4;
+constexpr int AD_TILE = 64;
 constexpr float AD_NEG = -1e30f;
 
 size_t attn_decode_scratch_bytes(int max_seqs, int Hq, int D, int max_splits) {
@@ -23,8 +26,8 @@ size_t attn_decode_scratch_bytes(int max_seqs, int Hq, int D, int max_splits) {
 }
 
 int attn_decode_splits(int n_seqs, int Hkv, int max_ctx) {
-  int want = (4 * 148 + n_seqs * Hkv - 1) / (n_seqs * Hkv);
-  int cap = (max_ctx + 63) / 64;
+  int want = (3 * 148 + n_seqs * Hkv - 1) / (n_seqs * Hkv);
+  int cap = (max_ctx + 2 * AD_TILE - 1) / (2 * AD_TILE);  // at least two tiles per split
   if (want > cap) want = cap;
   if (want > 32) want = 32;
   if (want < 1) want = 1;
@@ -36,127 +39,157 @@ __global__ void __launch_bounds__(AD_WARPS * 32)
 attn_decode_partial_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfloat16* __restrict__ kv_layer,
                            float* __restrict__ part_acc, float* __restrict__ part_ml, int n_splits,
                            BatchMeta bm, ModelDims d) {
-  constexpr int LPT = D / 8;          // lanes per token
-  constexpr int TPW = 32 / LPT;       // tokens per warp iteration
-  constexpr int GROUPS = AD_WARPS * TPW;
-  constexpr int PT = 16;              // tokens per page
-  __shared__ float sm_m[GROUPS][G], sm_l[GROUPS][G];
-  __shared__ float sm_acc[GROUPS][G][D];
+  constexpr int KS = D / 16, DN = D / 8, CPR = D / 8, PT = 16;
+  constexpr int TILE_BYTES = AD_TILE * D * 2;
+  extern __shared__ __align__(128) uint8_t ad_smem[];
+  const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(ad_smem);
+  auto k_tile = [&](int buf) { return smem0 + buf * TILE_BYTES; };
+  auto v_tile = [&](int buf) { return smem0 + (2 + buf) * TILE_BYTES; };
 
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int sub = lane / LPT, dl = (lane % LPT) * 8;
-  const int grp = warp * TPW + sub;
+  const int g = lane >> 2, tq = lane & 3;
 
   const int ctx_total = bm.ctx_lens[b] + 1;  // the new token's k, v are already in the cache
   int tps = (ctx_total + n_splits - 1) / n_splits;
-  tps = ((tps + PT - 1) / PT) * PT;
+  tps = ((tps + AD_TILE - 1) / AD_TILE) * AD_TILE;
   const int t_begin = split * tps;
   const int t_end = min(ctx_total, t_begin + tps);
-
-  // query heads kvh*G .. kvh*G+G-1 of row b, pre-scaled by 1/sqrt(D)
-  const float scale = rsqrtf((float)D);
-  float q[G][8];
-  const __nv_bfloat16* qrow = qkv + (size_t)b * d.qkv_rows + (size_t)kvh * G * D;  // decode: row b is sequence b
-#pragma unroll
-  for (int gq = 0; gq < G; ++gq) {
-    const uint4 v = *reinterpret_cast<const uint4*>(qrow + gq * D + dl);
-    q[gq][0] = bf16_lo(v.x) * scale; q[gq][1] = bf16_hi(v.x) * scale;
-    q[gq][2] = bf16_lo(v.y) * scale; q[gq][3] = bf16_hi(v.y) * scale;
-    q[gq][4] = bf16_lo(v.z) * scale; q[gq][5] = bf16_hi(v.z) * scale;
-    q[gq][6] = bf16_lo(v.w) * scale; q[gq][7] = bf16_hi(v.w) * scale;
-  }
-
-  float m_run[G], l_run[G], acc[G][8];
-#pragma unroll
-  for (int gq = 0; gq < G; ++gq) {
-    m_run[gq] = AD_NEG;
-    l_run[gq] = 0.f;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) acc[gq][e] = 0.f;
-  }
+  const int n_tiles = t_begin < t_end ? (t_end - t_begin + AD_TILE - 1) / AD_TILE : 0;
 
   const int32_t* bt = bm.block_table + (size_t)b * bm.max_pages_per_seq;
   const size_t page_elems = kv_page_elems(d.Hkv, PT, D);
   const size_t v_off = (size_t)d.Hkv * PT * D;
 
-  for (int base = t_begin; base < t_end; base += GROUPS * AD_UNROLL) {
-    uint4 kreg[AD_UNROLL], vreg[AD_UNROLL];
-    bool ok[AD_UNROLL];
-#pragma unroll
-    for (int u = 0; u < AD_UNROLL; ++u) {
-      const int tok = base + u * GROUPS + grp;
-      ok[u] = tok < t_end;
-      const int tk = ok[u] ? tok : t_begin;
-      const int page = bt[tk / PT];
-      const __nv_bfloat16* kp = kv_layer + (size_t)page * page_elems + ((size_t)kvh * PT + (tk % PT)) * D + dl;
-      kreg[u] = ldg_stream(kp);
-      vreg[u] = ldg_stream(kp + v_off);
+  auto load_tile = [&](int j, int buf) {
+    for (int idx = threadIdx.x; idx < AD_TILE * CPR; idx += AD_WARPS * 32) {
+      const int r = idx / CPR, c = idx % CPR;
+      const int key = t_begin + j * AD_TILE + r;
+      const bool ok = key < t_end;
+      const int kk = ok ? key : t_begin;
+      const __nv_bfloat16* src =
+          kv_layer + (size_t)bt[kk / PT] * page_elems + ((size_t)kvh * PT + (kk % PT)) * D + c * 8;
+      cp_async16(k_tile(buf) + tile_off<D>(r, c), src, ok);
+      cp_async16(v_tile(buf) + tile_off<D>(r, c), src + v_off, ok);
     }
-    float s[AD_UNROLL][G];
+  };
+  if (n_tiles > 0) load_tile(0, 0);
+  cp_async_commit();
+
+  // query heads kvh*G .. kvh*G+G-1 of row b as operand rows 0..G-1 (rows G..15 are zero)
+  uint32_t qf[KS][2];  // [k step][k half]; only the "row g" halves of the fragment are non-zero
+  {
+    const __nv_bfloat16* qrow = qkv + (size_t)b * d.qkv_rows + (size_t)(kvh * G + (g < G ? g : 0)) * D;
 #pragma unroll
-    for (int u = 0; u < AD_UNROLL; ++u) {
-      const float k0 = bf16_lo(kreg[u].x), k1 = bf16_hi(kreg[u].x), k2 = bf16_lo(kreg[u].y), k3 = bf16_hi(kreg[u].y);
-      const float k4 = bf16_lo(kreg[u].z), k5 = bf16_hi(kreg[u].z), k6 = bf16_lo(kreg[u].w), k7 = bf16_hi(kreg[u].w);
-#pragma unroll
-      for (int gq = 0; gq < G; ++gq) {
-        float p = q[gq][0] * k0 + q[gq][1] * k1 + q[gq][2] * k2 + q[gq][3] * k3 + q[gq][4] * k4 + q[gq][5] * k5 +
-                  q[gq][6] * k6 + q[gq][7] * k7;
-#pragma unroll
-        for (int o = LPT / 2; o > 0; o >>= 1) p += __shfl_xor_sync(0xffffffffu, p, o);
-        s[u][gq] = ok[u] ? p : AD_NEG;
-      }
-    }
-#pragma unroll
-    for (int gq = 0; gq < G; ++gq) {
-      float m_new = m_run[gq];
-#pragma unroll
-      for (int u = 0; u < AD_UNROLL; ++u) m_new = fmaxf(m_new, s[u][gq]);
-      const float corr = __expf(m_run[gq] - m_new);
-      m_run[gq] = m_new;
-      l_run[gq] *= corr;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) acc[gq][e] *= corr;
-#pragma unroll
-      for (int u = 0; u < AD_UNROLL; ++u) {
-        const float p = ok[u] ? __expf(s[u][gq] - m_new) : 0.f;
-        l_run[gq] += p;
-        acc[gq][0] += p * bf16_lo(vreg[u].x); acc[gq][1] += p * bf16_hi(vreg[u].x);
-        acc[gq][2] += p * bf16_lo(vreg[u].y); acc[gq][3] += p * bf16_hi(vreg[u].y);
-        acc[gq][4] += p * bf16_lo(vreg[u].z); acc[gq][5] += p * bf16_hi(vreg[u].z);
-        acc[gq][6] += p * bf16_lo(vreg[u].w); acc[gq][7] += p * bf16_hi(vreg[u].w);
-      }
+    for (int ks = 0; ks < KS; ++ks) {
+      qf[ks][0] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * tq) : 0u;
+      qf[ks][1] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * tq) : 0u;
     }
   }
+  const float sl2 = rsqrtf((float)D) * 1.4426950408889634f;
 
-  // combine the lane groups of the CTA
+  float o[DN][2];  // row g of each 8-wide output column tile (rows 8..15 are padding and dropped)
 #pragma unroll
-  for (int gq = 0; gq < G; ++gq) {
-    if ((lane % LPT) == 0) {
-      sm_m[grp][gq] = m_run[gq];
-      sm_l[grp][gq] = l_run[gq];
+  for (int i = 0; i < DN; ++i) o[i][0] = o[i][1] = 0.f;
+  float m_run = AD_NEG, l_run = 0.f;
+
+  for (int j = 0; j < n_tiles; ++j) {
+    const int buf = j & 1;
+    if (j + 1 < n_tiles) load_tile(j + 1, buf ^ 1);
+    cp_async_commit();
+    cp_async_wait<1>();
+    __syncthreads();
+
+    // scores of this warp's 16 keys: two 8-key column tiles
+    float s[2][4];
+    s[0][0] = s[0][1] = s[0][2] = s[0][3] = 0.f;
+    s[1][0] = s[1][1] = s[1][2] = s[1][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      const int r = 16 * warp + (lane & 7) + ((lane >> 4) << 3);
+      const int c = 2 * ks + ((lane >> 3) & 1);
+      uint32_t b0, b1, b2, b3;
+      ldsm_x4(k_tile(buf) + tile_off<D>(r, c), b0, b1, b2, b3);
+      mma_bf16_16816(s[0], qf[ks][0], 0u, qf[ks][1], 0u, b0, b1);
+      mma_bf16_16816(s[1], qf[ks][0], 0u, qf[ks][1], 0u, b2, b3);
+    }
+    const int key0 = t_begin + j * AD_TILE + 16 * warp + 2 * tq;
+    float mx = m_run;
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const float v = (key0 + 8 * nt + e < t_end) ? s[nt][e] * sl2 : AD_NEG;
+        s[nt][e] = v;
+        mx = fmaxf(mx, v);
+      }
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    const float corr = exp2f(m_run - mx);
+    m_run = mx;
+    float p[2][2];
+    float sum = 0.f;
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        p[nt][e] = (key0 + 8 * nt + e < t_end) ? exp2f(s[nt][e] - mx) : 0.f;
+        sum += p[nt][e];
+      }
+    l_run = l_run * corr + sum;
+    const uint32_t pa0 = pack_bf16(p[0][0], p[0][1]), pa2 = pack_bf16(p[1][0], p[1][1]);
+#pragma unroll
+    for (int dp = 0; dp < DN / 2; ++dp) {
+      const int r = 16 * warp + (lane & 7) + (((lane >> 3) & 1) << 3);
+      const int c = 2 * dp + (lane >> 4);
+      uint32_t b0, b1, b2, b3;
+      ldsm_x4_t(v_tile(buf) + tile_off<D>(r, c), b0, b1, b2, b3);
+      float c0[4] = {o[2 * dp][0] * corr, o[2 * dp][1] * corr, 0.f, 0.f};
+      float c1[4] = {o[2 * dp + 1][0] * corr, o[2 * dp + 1][1] * corr, 0.f, 0.f};
+      mma_bf16_16816(c0, pa0, 0u, pa2, 0u, b0, b1);
+      mma_bf16_16816(c1, pa0, 0u, pa2, 0u, b2, b3);
+      o[2 * dp][0] = c0[0]; o[2 * dp][1] = c0[1];
+      o[2 * dp + 1][0] = c1[0]; o[2 * dp + 1][1] = c1[1];
+    }
+    __syncthreads();
+  }
+  cp_async_wait<0>();
+  __syncthreads();  // the staging buffers are reused below
+
+  // combine the four warps: (m, l) per head, then rescaled O
+  l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+  l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+  float* sm_m = reinterpret_cast<float*>(ad_smem);                 // [AD_WARPS][8]
+  float* sm_l = sm_m + AD_WARPS * 8;                               // [AD_WARPS][8]
+  float* sm_o = sm_l + AD_WARPS * 8;                               // [AD_WARPS][G][D]
+  if (g < G) {
+    if (tq == 0) {
+      sm_m[warp * 8 + g] = m_run;
+      sm_l[warp * 8 + g] = l_run;
     }
 #pragma unroll
-    for (int e = 0; e < 8; ++e) sm_acc[grp][gq][dl + e] = acc[gq][e];
+    for (int dn = 0; dn < DN; ++dn) {
+      sm_o[(warp * G + g) * D + 8 * dn + 2 * tq] = o[dn][0];
+      sm_o[(warp * G + g) * D + 8 * dn + 2 * tq + 1] = o[dn][1];
+    }
   }
   __syncthreads();
-  for (int o = threadIdx.x; o < G * D; o += AD_WARPS * 32) {
-    const int gq = o / D, dd = o % D;
+  for (int e = threadIdx.x; e < G * D; e += AD_WARPS * 32) {
+    const int gq = e / D, dd = e % D;
     float mx = AD_NEG;
 #pragma unroll
-    for (int r = 0; r < GROUPS; ++r) mx = fmaxf(mx, sm_m[r][gq]);
+    for (int w = 0; w < AD_WARPS; ++w) mx = fmaxf(mx, sm_m[w * 8 + gq]);
     float l = 0.f, a = 0.f;
 #pragma unroll
-    for (int r = 0; r < GROUPS; ++r) {
-      const float wgt = __expf(sm_m[r][gq] - mx);
-      l += wgt * sm_l[r][gq];
-      a += wgt * sm_acc[r][gq][dd];
+    for (int w = 0; w < AD_WARPS; ++w) {
+      const float wgt = exp2f(sm_m[w * 8 + gq] - mx);
+      l += wgt * sm_l[w * 8 + gq];
+      a += wgt * sm_o[(w * G + gq) * D + dd];
     }
-    const int hq = kvh * G + gq;
-    const size_t slot = ((size_t)b * d.Hq + hq) * n_splits + split;
+    const size_t slot = ((size_t)b * d.Hq + kvh * G + gq) * n_splits + split;
     part_acc[slot * D + dd] = a;
     if (dd == 0) {
-      part_ml[slot * 2] = mx;
+      part_ml[slot * 2] = mx;  // log2 units
       part_ml[slot * 2 + 1] = l;
     }
   }
@@ -172,7 +205,7 @@ __global__ void attn_decode_merge_kernel(const float* __restrict__ part_acc, con
   float l = 0.f, a = 0.f;
   for (int s = 0; s < n_splits; ++s) {
     const size_t slot = (size_t)bh * n_splits + s;
-    const float wgt = __expf(part_ml[slot * 2] - mx);
+    const float wgt = exp2f(part_ml[slot * 2] - mx);
     l += wgt * part_ml[slot * 2 + 1];
     a += wgt * part_acc[slot * D + dd];
   }
@@ -182,9 +215,16 @@ __global__ void attn_decode_merge_kernel(const float* __restrict__ part_acc, con
 template <int D, int G>
 static int launch_dg(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __nv_bfloat16* attn_out,
                      float* scratch, int n_splits, const BatchMeta& bm, const ModelDims& d, cudaStream_t st) {
+  static bool configured = false;
+  constexpr int smem = 4 * AD_TILE * D * 2;  // K[2] + V[2]; also covers the end-of-kernel combine buffers
+  static_assert(smem >= (int)((2 * AD_WARPS * 8 + AD_WARPS * G * D) * sizeof(float)), "combine buffers must fit");
+  if (!configured) {
+    HYP_CUDA_TRY(cudaFuncSetAttribute(attn_decode_partial_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    configured = true;
+  }
   float* part_acc = scratch;
   float* part_ml = scratch + (size_t)bm.n_seqs * d.Hq * n_splits * D;
-  attn_decode_partial_kernel<D, G><<<dim3(n_splits, d.Hkv, bm.n_seqs), AD_WARPS * 32, 0, st>>>(
+  attn_decode_partial_kernel<D, G><<<dim3(n_splits, d.Hkv, bm.n_seqs), AD_WARPS * 32, smem, st>>>(
       qkv, kv_layer, part_acc, part_ml, n_splits, bm, d);
   attn_decode_merge_kernel<D><<<bm.n_seqs * d.Hq, D, 0, st>>>(part_acc, part_ml, attn_out, n_splits, d.Hq);
   return 2;
