@@ -18,6 +18,7 @@
 #include <cuda.h>
 
 #include "gemm_tc.cuh"
+#include "sm100_common.cuh"
 #include "hyperion.h"
 
 namespace hyp {
@@ -28,52 +29,7 @@ constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
 constexpr int TC_THREADS = 192;
-constexpr uint64_t WAIT_LIMIT_NS = 4000000000ull;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ uint64_t globaltimer() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false after WAIT_LIMIT_NS or once another role has raised `abort_flag`.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (int i = 0; i < 64; ++i)
-    if (mbar_try(bar, parity)) return true;
-  const uint64_t t0 = globaltimer();
-  while (true) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (globaltimer() - t0 > WAIT_LIMIT_NS) return false;
-  }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
-      : "memory");
-}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -384,19 +340,15 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-int make_map(TcOperand* op, const __nv_bfloat16* ptr, int rows, int K) {
-  op->ptr = ptr;
-  op->rows = rows;
-  op->K = K;
-  op->box_rows = 128;
+int encode_map(CUtensorMap* map, const __nv_bfloat16* ptr, int rows, int K, int box_rows) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return HYP_ECUDA;
   if ((K % 8) != 0 || ((uintptr_t)ptr & 15) != 0) return HYP_EINVAL;
   const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)BK, 128u};
+  const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1u, 1u};
-  CUresult r = enc(&op->map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)ptr, dims, strides, box, estr,
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)ptr, dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
@@ -446,8 +398,24 @@ int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
 
 }  // namespace
 
-int tc_make_weight(TcWeight* w, const __nv_bfloat16* ptr, int rows, int K) { return make_map(w, ptr, rows, K); }
-int tc_make_act(TcAct* a, const __nv_bfloat16* ptr, int rows, int K) { return make_map(a, ptr, rows, K); }
+// Weights: 128-row boxes for the tile kernel, 16- and 32-row boxes for the weight-streaming kernel.
+int tc_make_weight(TcWeight* w, const __nv_bfloat16* ptr, int rows, int K) {
+  w->ptr = ptr; w->rows = rows; w->K = K;
+  int rc = encode_map(&w->map, ptr, rows, K, 128);
+  if (rc) return rc;
+  rc = encode_map(&w->map_small[0], ptr, rows, K, 16);
+  if (rc) return rc;
+  return encode_map(&w->map_small[1], ptr, rows, K, 32);
+}
+// Activations: 128-row boxes for the tile kernel, 8/16/24/32-row boxes for the weight-streaming kernel.
+int tc_make_act(TcAct* a, const __nv_bfloat16* ptr, int rows, int K) {
+  a->ptr = ptr; a->rows = rows; a->K = K;
+  int rc = encode_map(&a->map, ptr, rows, K, 128);
+  for (int nb = 1; nb <= 4 && !rc; ++nb) rc = encode_map(&a->map_small[nb - 1], ptr, rows, K, 8 * nb);
+  return rc;
+}
+
+int* tc_err_flag_ptr() { return g_err_flag; }
 
 int tc_prepare() {
   if (!g_err_flag) {

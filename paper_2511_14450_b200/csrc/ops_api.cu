@@ -43,9 +43,7 @@ extern "C" int hyp_op_gemm(const void* a, const void* w, int32_t M, int32_t N, i
   if (!a || !w || !out || M < 1 || N < 1 || K < 8 || K % 8 || ldo < N) return HYP_EINVAL;
   if (epilogue < HYP_EPI_STORE_BF16 || epilogue > HYP_EPI_STORE_F32) return HYP_EINVAL;
   cudaStream_t st = (cudaStream_t)stream;
-  if (M <= 32)
-    return finish(launch_gemm_skinny((const __nv_bfloat16*)a, K, (const __nv_bfloat16*)w, N, K, M, epilogue, out, ldo, st));
-  if (N % 16 || ldo % 8) return HYP_EINVAL;
+  if (M > 32 && (N % 16 || ldo % 8)) return HYP_EINVAL;
   int rc = tc_prepare();
   if (rc) return rc;
   TcAct ta;
@@ -54,6 +52,7 @@ extern "C" int hyp_op_gemm(const void* a, const void* w, int32_t M, int32_t N, i
   if (rc) return rc;
   rc = tc_make_weight(&tw, (const __nv_bfloat16*)w, epilogue == HYP_EPI_SWIGLU_BF16 ? 2 * N : N, K);
   if (rc) return rc;
+  if (M <= 32) return finish(launch_gemm_stream(ta, tw, M, N, K, epilogue, out, ldo, st));
   return finish(launch_gemm_tc(ta, tw, M, N, K, epilogue, out, ldo, st));
 }
 

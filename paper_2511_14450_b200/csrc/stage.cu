@@ -234,7 +234,8 @@ int check_ready(const hyp_stage* s) {
 // out[m, n] (+)= a[m, :] . w[n, :] with the kernel family chosen by the row count.
 int project(hyp_stage* s, const TcAct& act, const bf16* a, int lda, const TcWeight& tw, const bf16* w, int N, int K,
             int M, int epi, void* out, int ldo, cudaStream_t st) {
-  if (M <= 32) return launch_gemm_skinny(a, lda, w, N, K, M, epi, out, ldo, st);
+  (void)a; (void)lda; (void)w;
+  if (M <= 32) return launch_gemm_stream(act, tw, M, N, K, epi, out, ldo, st);
   return launch_gemm_tc(act, tw, M, N, K, epi, out, ldo, st);
 }
 
