@@ -49,6 +49,7 @@ attn_decode_partial_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfl
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, tq = lane & 3;
+  pdl_wait();  // the cache pages, the query row and the metadata all come from earlier kernels / copies
 
   const int ctx_total = bm.ctx_lens[b] + 1;  // the new token's k, v are already in the cache
   int tps = (ctx_total + n_splits - 1) / n_splits;
@@ -154,6 +155,7 @@ attn_decode_partial_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfl
     __syncthreads();
   }
   cp_async_wait<0>();
+  pdl_trigger();
   __syncthreads();  // the staging buffers are reused below
 
   // combine the four warps: (m, l) per head, then rescaled O
@@ -200,6 +202,8 @@ __global__ void attn_decode_merge_kernel(const float* __restrict__ part_acc, con
                                          __nv_bfloat16* __restrict__ out, int n_splits, int Hq) {
   const int bh = blockIdx.x;  // b * Hq + hq
   const int dd = threadIdx.x;
+  pdl_trigger();
+  pdl_wait();
   float mx = AD_NEG;
   for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, part_ml[((size_t)bh * n_splits + s) * 2]);
   float l = 0.f, a = 0.f;
@@ -224,9 +228,10 @@ static int launch_dg(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __
   }
   float* part_acc = scratch;
   float* part_ml = scratch + (size_t)bm.n_seqs * d.Hq * n_splits * D;
-  attn_decode_partial_kernel<D, G><<<dim3(n_splits, d.Hkv, bm.n_seqs), AD_WARPS * 32, smem, st>>>(
-      qkv, kv_layer, part_acc, part_ml, n_splits, bm, d);
-  attn_decode_merge_kernel<D><<<bm.n_seqs * d.Hq, D, 0, st>>>(part_acc, part_ml, attn_out, n_splits, d.Hq);
+  HYP_CUDA_TRY(launch_pdl(attn_decode_partial_kernel<D, G>, dim3(n_splits, d.Hkv, bm.n_seqs), dim3(AD_WARPS * 32), smem,
+                          st, qkv, kv_layer, part_acc, part_ml, n_splits, bm, d));
+  HYP_CUDA_TRY(launch_pdl(attn_decode_merge_kernel<D>, dim3(bm.n_seqs * d.Hq), dim3(D), 0, st, part_acc, part_ml,
+                          attn_out, n_splits, d.Hq));
   return 2;
 }
 

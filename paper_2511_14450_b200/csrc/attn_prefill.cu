@@ -29,6 +29,8 @@ attn_prefill_fa_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfloat1
   auto k_tile = [&](int buf) { return smem0 + buf * TILE_BYTES; };
   auto v_tile = [&](int buf) { return smem0 + (2 + buf) * TILE_BYTES; };
 
+  pdl_trigger();
+  pdl_wait();
   // which (sequence, query tile) is this CTA?
   int t = blockIdx.x, seq = -1, q0 = 0, q_len = 0;
   for (int i = 0; i < bm.n_seqs; ++i) {
@@ -209,7 +211,8 @@ int launch_fa(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __nv_bflo
   }
   // every sequence adds at most one ragged tile on top of floor(rows / 64)
   const int max_tiles = bm.n_tokens / FA_BQ + bm.n_seqs;
-  attn_prefill_fa_kernel<D><<<dim3(max_tiles, d.Hq), FA_THREADS, smem, st>>>(qkv, kv_layer, attn_out, bm, d);
+  HYP_CUDA_TRY(launch_pdl(attn_prefill_fa_kernel<D>, dim3(max_tiles, d.Hq), dim3(FA_THREADS), smem, st, qkv, kv_layer,
+                          attn_out, bm, d));
   return 1;
 }
 

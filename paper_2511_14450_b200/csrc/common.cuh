@@ -56,6 +56,40 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
 }
 
 // ---------------------------------------------------------------------------------------------
+// programmatic dependent launch: every kernel of the block sequence can be launched so that it may start
+// while its predecessor drains.  A kernel calls pdl_trigger() when its successor may be scheduled and
+// pdl_wait() before the first access to memory its predecessor writes or reads; everything before
+// pdl_wait() - barrier set-up, weight prefetch - then overlaps the predecessor's tail.  Without the
+// launch attribute both are no-ops.  Measured on B200 the overlap made the decode step slower (2.55 ms
+// against 2.14 ms for the 14-block stage: successors that become resident early add copies in flight
+// beyond the point where HBM throughput peaks), so the attribute is off by default.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Process-wide switch for the launch attribute (see above for why it defaults to off).
+inline bool& pdl_enabled() {
+  static bool on = false;
+  return on;
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// ---------------------------------------------------------------------------------------------
 // per-call batch metadata as the kernels see it (all DEVICE pointers, int32)
 // ---------------------------------------------------------------------------------------------
 struct BatchMeta {
@@ -100,11 +134,6 @@ int launch_rmsnorm(const float* x, const __nv_bfloat16* g, __nv_bfloat16* h, int
                    const int32_t* row_index /* optional gather of rows, may be null */, cudaStream_t st);
 int launch_rope_kv_write(__nv_bfloat16* qkv, __nv_bfloat16* kv_layer, const float2* rope_table,
                          const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
-// out[m, n] = sum_k a[m, k] * w[n, k] for M <= 32 rows (weight-streaming, HBM-bound)
-int launch_gemm_skinny(const __nv_bfloat16* a, int lda, const __nv_bfloat16* w, int N, int K, int M,
-                       int epi, void* out, int ldo, cudaStream_t st);
-// any M, tensor-core tiles (tcgen05); tensor maps are prepared by the caller
-struct GemmPlan;
 int launch_attn_prefill(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __nv_bfloat16* attn_out,
                         const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
 // decode attention: one query row per sequence; `scratch` holds split partials

@@ -8,6 +8,8 @@ namespace hyp {
 // cannot validate device-resident ids without a sync).
 __global__ void embed_kernel(const int32_t* __restrict__ ids, const __nv_bfloat16* __restrict__ E,
                              float* __restrict__ x, int H, int V) {
+  pdl_trigger();
+  pdl_wait();
   const int t = blockIdx.x;
   int id = ids[t];
   id = id < 0 ? 0 : (id >= V ? V - 1 : id);
@@ -21,11 +23,13 @@ __global__ void embed_kernel(const int32_t* __restrict__ ids, const __nv_bfloat1
 }
 
 int launch_embed(const int32_t* ids, const __nv_bfloat16* E, float* x, int M, int H, int V, cudaStream_t st) {
-  embed_kernel<<<M, 128, 0, st>>>(ids, E, x, H, V);
+  HYP_CUDA_TRY(launch_pdl(embed_kernel, dim3(M), dim3(128), 0, st, ids, E, x, H, V));
   return 1;
 }
 
 __global__ void copy_f32_kernel(const float4* __restrict__ src, float4* __restrict__ dst, size_t n4) {
+  pdl_trigger();
+  pdl_wait();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x)
     dst[i] = src[i];
 }
@@ -35,7 +39,8 @@ int launch_copy_f32(const float* src, float* dst, size_t n, cudaStream_t st) {
   int blocks = (int)((n4 + 255) / 256);
   if (blocks > 148 * 8) blocks = 148 * 8;
   if (blocks < 1) blocks = 1;
-  copy_f32_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(src), reinterpret_cast<float4*>(dst), n4);
+  HYP_CUDA_TRY(launch_pdl(copy_f32_kernel, dim3(blocks), dim3(256), 0, st, reinterpret_cast<const float4*>(src),
+                          reinterpret_cast<float4*>(dst), n4));
   return 1;
 }
 
@@ -46,6 +51,8 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16*
                                __nv_bfloat16* __restrict__ h, int H, float eps,
                                const int32_t* __restrict__ row_index) {
   __shared__ float red[THREADS / 32];
+  pdl_trigger();
+  pdl_wait();
   const int r = blockIdx.x;
   const int row = row_index ? row_index[r] : r;
   const float4* xr = reinterpret_cast<const float4*>(x + (size_t)row * H);
@@ -76,7 +83,7 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16*
 
 int launch_rmsnorm(const float* x, const __nv_bfloat16* g, __nv_bfloat16* h, int M, int H, float eps,
                    const int32_t* row_index, cudaStream_t st) {
-  rmsnorm_kernel<256><<<M, 256, 0, st>>>(x, g, h, H, eps, row_index);
+  HYP_CUDA_TRY(launch_pdl(rmsnorm_kernel<256>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
   return 1;
 }
 
@@ -85,6 +92,8 @@ int launch_rmsnorm(const float* x, const __nv_bfloat16* g, __nv_bfloat16* h, int
 // One thread handles 8 rotation pairs (i .. i+7, i+D/2 .. i+D/2+7) of one head of one row.
 __global__ void rope_kv_write_kernel(__nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ kv_layer,
                                      const float2* __restrict__ rope_table, BatchMeta bm, ModelDims d) {
+  pdl_trigger();
+  pdl_wait();
   const int t = blockIdx.x;
   const int vec_per_head = d.D / 16;
   const int n_heads = d.Hq + 2 * d.Hkv;
@@ -137,7 +146,7 @@ int launch_rope_kv_write(__nv_bfloat16* qkv, __nv_bfloat16* kv_layer, const floa
   const int work = (d.Hq + 2 * d.Hkv) * (d.D / 16);
   int threads = ((work + 31) / 32) * 32;
   if (threads > 512) threads = 512;
-  rope_kv_write_kernel<<<bm.n_tokens, threads, 0, st>>>(qkv, kv_layer, rope_table, bm, d);
+  HYP_CUDA_TRY(launch_pdl(rope_kv_write_kernel, dim3(bm.n_tokens), dim3(threads), 0, st, qkv, kv_layer, rope_table, bm, d));
   return 1;
 }
 

@@ -53,33 +53,38 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   const int KB = (K + GS_BK - 1) / GS_BK;
   const uint32_t my_bars = smem_u32(bars) + 8u * (warp * GS_MAX_SLOTS);
   const uint32_t my_ring = base + (uint32_t)(warp * S) * STAGE_BYTES;
-  const int row1 = SWIGLU ? N + n0 : n0 + 16;
+  const int row1 = N + n0;  // SwiGLU: the up rows that pair with this CTA's gate rows
 
   // one k-block into one of this warp's slots (lane 0 only).  CTAs walk K from staggered starting points
   // (a fixed rotation per CTA, so the summation order stays reproducible): otherwise every resident CTA
   // would ask for the same activation slice and the same column offsets of its rows at the same moment.
   const int rot = (int)((blockIdx.x * 13u) % (unsigned)KB);
-  auto issue = [&](int kb_logical, int slot) {
+  // weights: never written by any kernel, may be fetched before the predecessor has finished
+  auto issue_w = [&](int kb_logical, int slot) {
     int kb = kb_logical + rot;
     if (kb >= KB) kb -= KB;
     const uint32_t dst = my_ring + slot * STAGE_BYTES, bar = my_bars + 8u * slot;
     mbar_expect_tx(bar, STAGE_BYTES);
-    if (TILES == 2 && !SWIGLU) {
-      tma_load_2d(dst, &tm_w, kb * GS_BK, n0, bar);  // one 32-row box
-    } else {
-      tma_load_2d(dst, &tm_w, kb * GS_BK, n0, bar);
-      if (TILES == 2) tma_load_2d(dst + W_TILE_BYTES, &tm_w, kb * GS_BK, row1, bar);
-    }
-    tma_load_2d(dst + TILES * W_TILE_BYTES, &tm_a, kb * GS_BK, 0, bar);
+    tma_load_2d(dst, &tm_w, kb * GS_BK, n0, bar);  // 16 rows, or one 32-row box
+    if (SWIGLU) tma_load_2d(dst + W_TILE_BYTES, &tm_w, kb * GS_BK, row1, bar);
+  };
+  // activations: produced by the predecessor
+  auto issue_a = [&](int kb_logical, int slot) {
+    int kb = kb_logical + rot;
+    if (kb >= KB) kb -= KB;
+    tma_load_2d(my_ring + slot * STAGE_BYTES + TILES * W_TILE_BYTES, &tm_a, kb * GS_BK, 0, my_bars + 8u * slot);
   };
 
   if (lane == 0) {
     for (int sl = 0; sl < S; ++sl) mbar_init(my_bars + 8u * sl, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    for (int sl = 0; sl < S; ++sl) {
-      const int kb = warp + GS_WARPS * sl;
-      if (kb < KB) issue(kb, sl);
-    }
+    for (int sl = 0; sl < S; ++sl)
+      if (warp + GS_WARPS * sl < KB) issue_w(warp + GS_WARPS * sl, sl);
+  }
+  pdl_wait();
+  if (lane == 0) {
+    for (int sl = 0; sl < S; ++sl)
+      if (warp + GS_WARPS * sl < KB) issue_a(warp + GS_WARPS * sl, sl);
   }
   __syncwarp();
 
@@ -118,10 +123,14 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
     __syncwarp();
     if (lane == 0) {
       const int next = kb + GS_WARPS * S;
-      if (next < KB) issue(next, slot);
+      if (next < KB) {
+        issue_w(next, slot);
+        issue_a(next, slot);
+      }
     }
     if (++slot == S) { slot = 0; phase ^= 1u; }
   }
+  pdl_trigger();  // this warp has no more copies to issue: the successor may begin its own prefetch
   if (!ok) {
     // a copy never landed: record it and let whatever is still in flight arrive (bounded) before leaving
     if (lane == 0) atomicCAS(err, 0, 4);
@@ -197,9 +206,9 @@ int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
   if (slots < 2) slots = 2;
   while (slots > 1 && GS_WARPS * slots * STAGE_BYTES + 1024 > MAX_DYN) --slots;
   const int smem = GS_WARPS * slots * STAGE_BYTES + 1024;
-  gemm_stream_kernel<NB, EPI, TILES><<<n_ctas, GS_THREADS, smem, st>>>(
-      (TILES == 2 && !SWIGLU) ? w.map_small[1] : w.map_small[0], act.map_small[NB - 1], N, K, M, out, ldo, slots,
-      tc_err_flag_ptr());
+  HYP_CUDA_TRY(launch_pdl(gemm_stream_kernel<NB, EPI, TILES>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
+                          (TILES == 2 && !SWIGLU) ? w.map_small[1] : w.map_small[0], act.map_small[NB - 1], N, K, M, out,
+                          ldo, slots, tc_err_flag_ptr()));
   return 1;
 }
 

@@ -218,6 +218,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_trigger();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -225,6 +226,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      pdl_wait();  // the activation operand is the predecessor's output
       Segments seg(STREAMK, tiles_m, tiles_n, KB, team);
       int tile, kb0, kb1;
       while (ok && seg.next(tile, kb0, kb1)) {
@@ -283,6 +285,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   } else {
     // ---------------- epilogue warps ----------------
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
+    pdl_wait();              // the output buffer may still be in use by the predecessor
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
@@ -392,7 +395,8 @@ int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
     const long tiles = (long)tiles_m * tiles_n;
     grid = (int)(tiles < num_sms ? tiles : num_sms);
   }
-  gemm_tc_kernel<EPI><<<grid, TC_THREADS, SMEM_BYTES, st>>>(act.map, w.map, M, N, K, out, ldo, team, g_err_flag);
+  HYP_CUDA_TRY(launch_pdl(gemm_tc_kernel<EPI>, dim3(grid), dim3(TC_THREADS), (size_t)SMEM_BYTES, st, act.map, w.map, M, N,
+                          K, out, ldo, team, g_err_flag));
   return 1;
 }
 

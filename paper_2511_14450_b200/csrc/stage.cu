@@ -67,6 +67,16 @@ struct hyp_stage {
   void *io_in = nullptr, *io_out = nullptr;
   size_t io_in_bytes = 0, io_out_bytes = 0;
   int64_t launches = 0;
+  // decode steps replay a captured CUDA graph (one per batch size and attention split count); the graph
+  // reads its input from g_in and leaves its result in g_out
+  struct DecodeGraph {
+    int n = 0, n_splits = 0, n_launches = 0;
+    cudaGraphExec_t exec = nullptr;  // null until the second use of the key (the first runs eagerly)
+  };
+  std::vector<DecodeGraph> graphs;
+  bool graphs_ok = true;
+  cudaStream_t cap_stream = nullptr;
+  void *g_in = nullptr, *g_out = nullptr;
   // optional per-launch timing of one kernel class
   int time_cls = -1;
   std::vector<cudaEvent_t> time_ev;
@@ -268,7 +278,79 @@ int run_blocks(hyp_stage* s, const BatchMeta& bm, bool decode, int n_splits, cud
   return HYP_OK;
 }
 
-int run_stage(hyp_stage* s, const hyp_batch* b, const void* in, void* out, cudaStream_t st, bool decode) {
+// Enqueue [embedding gather | input copy] -> blocks -> [final norm + LM head | output copy] on `st`.
+int enqueue_stage(hyp_stage* s, const BatchMeta& bm, int n_seqs, bool decode, bool all_rows, int n_splits,
+                  const void* in, void* out, cudaStream_t st) {
+  const ModelDims& d = s->dims;
+  const int M = bm.n_tokens;
+  if (s->first)
+    HYP_LAUNCH(launch_embed((const int32_t*)in, s->embed, s->x, M, d.H, d.V, st));
+  else
+    HYP_LAUNCH(launch_copy_f32((const float*)in, s->x, (size_t)M * d.H, st));
+  int rc = run_blocks(s, bm, decode, n_splits, st, nullptr);
+  if (rc) return rc;
+  if (s->last) {
+    const int rows = all_rows ? M : n_seqs;
+    HYP_LAUNCH(launch_rmsnorm(s->x, s->gf, s->h, rows, d.H, d.eps, all_rows ? nullptr : bm.last_row, st));
+    HYP_LAUNCH_T(HYP_K_LM_HEAD,
+                 project(s, s->tc_h, s->h, d.H, s->tc_lm, s->wlm, d.V, d.H, rows, EPI_STORE_F32, out, d.V, st));
+  } else {
+    HYP_LAUNCH(launch_copy_f32(s->x, (float*)out, (size_t)M * d.H, st));
+  }
+  return HYP_OK;
+}
+
+// Decode through a captured graph.  `in` / `out` may be device or host memory (the copies around the
+// graph take either).  Returns HYP_OK, an error, or 1 if the caller should run the step eagerly.
+int decode_with_graph(hyp_stage* s, const BatchMeta& bm, int n, int n_splits, const void* in, void* out,
+                      cudaStream_t st) {
+  const ModelDims& d = s->dims;
+  hyp_stage::DecodeGraph* g = nullptr;
+  for (auto& e : s->graphs)
+    if (e.n == n && e.n_splits == n_splits) g = &e;
+  if (!g) {  // first use of this key: run eagerly (also completes one-time kernel configuration)
+    hyp_stage::DecodeGraph e;
+    e.n = n;
+    e.n_splits = n_splits;
+    s->graphs.push_back(e);
+    return 1;
+  }
+  if (!g->exec) {
+    const int64_t before = s->launches;
+    if (cudaStreamBeginCapture(s->cap_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+      cudaGetLastError();
+      s->graphs_ok = false;
+      return 1;
+    }
+    const int rc = enqueue_stage(s, bm, n, true, true, n_splits, s->g_in, s->g_out, s->cap_stream);
+    cudaGraph_t graph = nullptr;
+    const cudaError_t e1 = cudaStreamEndCapture(s->cap_stream, &graph);
+    g->n_launches = (int)(s->launches - before);
+    s->launches = before;
+    cudaError_t e2 = cudaErrorUnknown;
+    if (rc == HYP_OK && e1 == cudaSuccess && graph) e2 = cudaGraphInstantiate(&g->exec, graph, 0);
+    if (graph) cudaGraphDestroy(graph);
+    if (e2 != cudaSuccess) {
+      cudaGetLastError();
+      g->exec = nullptr;
+      if (pdl_enabled())
+        pdl_enabled() = false;  // retry on the next step without programmatic launches
+      else
+        s->graphs_ok = false;   // this driver cannot capture the sequence: stay on the eager path
+      return 1;
+    }
+  }
+  const size_t in_bytes = s->first ? (size_t)n * sizeof(int32_t) : (size_t)n * d.H * sizeof(float);
+  const size_t out_bytes = (size_t)n * (s->last ? d.V : d.H) * sizeof(float);
+  HYP_CUDA_TRY(cudaMemcpyAsync(s->g_in, in, in_bytes, cudaMemcpyDefault, st));
+  HYP_CUDA_TRY(cudaGraphLaunch(g->exec, st));
+  s->launches += g->n_launches;
+  HYP_CUDA_TRY(cudaMemcpyAsync(out, s->g_out, out_bytes, cudaMemcpyDefault, st));
+  return HYP_OK;
+}
+
+int run_stage(hyp_stage* s, const hyp_batch* b, const void* in, void* out, cudaStream_t st, bool decode,
+              bool io_on_host = false) {
   if (!s || !in || !out) return HYP_EINVAL;
   int rc = check_ready(s);
   if (rc) return rc;
@@ -279,12 +361,6 @@ int run_stage(hyp_stage* s, const hyp_batch* b, const void* in, void* out, cudaS
   if (rc) return rc;
   const BatchMeta bm = device_meta(s, hb);
   const ModelDims& d = s->dims;
-  const int M = hb.M;
-
-  if (s->first)
-    HYP_LAUNCH(launch_embed((const int32_t*)in, s->embed, s->x, M, d.H, d.V, st));
-  else
-    HYP_LAUNCH(launch_copy_f32((const float*)in, s->x, (size_t)M * d.H, st));
 
   int n_splits = 1;
   if (decode) {
@@ -292,18 +368,21 @@ int run_stage(hyp_stage* s, const hyp_batch* b, const void* in, void* out, cudaS
     for (int i = 0; i < hb.n; ++i) max_ctx = std::max(max_ctx, b->ctx_lens[i] + 1);
     n_splits = std::min(s->max_splits, attn_decode_splits(hb.n, d.Hkv, max_ctx));
   }
-  rc = run_blocks(s, bm, decode, n_splits, st, nullptr);
-  if (rc) return rc;
-
-  if (s->last) {
-    const bool all = (b->flags & HYP_BATCH_ALL_LOGITS) != 0 || decode;
-    const int rows = all ? M : hb.n;
-    HYP_LAUNCH(launch_rmsnorm(s->x, s->gf, s->h, rows, d.H, d.eps, all ? nullptr : bm.last_row, st));
-    HYP_LAUNCH_T(HYP_K_LM_HEAD,
-                 project(s, s->tc_h, s->h, d.H, s->tc_lm, s->wlm, d.V, d.H, rows, EPI_STORE_F32, out, d.V, st));
-  } else {
-    HYP_LAUNCH(launch_copy_f32(s->x, (float*)out, (size_t)M * d.H, st));
+  const bool all = (b->flags & HYP_BATCH_ALL_LOGITS) != 0 || decode;
+  rc = 1;
+  if (decode && s->graphs_ok && s->time_cls < 0) rc = decode_with_graph(s, bm, hb.n, n_splits, in, out, st);
+  if (rc == 1) {
+    if (io_on_host) {  // eager kernels need device buffers: stage through the I/O buffers
+      const size_t in_bytes = s->first ? (size_t)hb.M * sizeof(int32_t) : (size_t)hb.M * d.H * sizeof(float);
+      const size_t out_bytes = (size_t)(all ? hb.M : hb.n) * (s->last ? d.V : d.H) * sizeof(float);
+      HYP_CUDA_TRY(cudaMemcpyAsync(s->io_in, in, in_bytes, cudaMemcpyHostToDevice, st));
+      rc = enqueue_stage(s, bm, hb.n, decode, all, n_splits, s->io_in, s->io_out, st);
+      if (rc == HYP_OK) HYP_CUDA_TRY(cudaMemcpyAsync(out, s->io_out, out_bytes, cudaMemcpyDeviceToHost, st));
+    } else {
+      rc = enqueue_stage(s, bm, hb.n, decode, all, n_splits, in, out, st);
+    }
   }
+  if (rc) return rc;
   cudaError_t e = cudaPeekAtLastError();
   if (e != cudaSuccess) {
     set_last_cuda_error((int)e);
@@ -338,10 +417,8 @@ int run_stage_host(hyp_stage* s, const hyp_batch* b, const void* in, void* out, 
     s->free_pages.swap(freep);
     if (rc) return rc;
   }
-  HYP_CUDA_TRY(cudaMemcpyAsync(s->io_in, in, in_bytes, cudaMemcpyHostToDevice, st));
-  int rc = run_stage(s, b, s->io_in, s->io_out, st, decode);
+  int rc = run_stage(s, b, in, out, st, decode, /*io_on_host=*/true);
   if (rc) return rc;
-  HYP_CUDA_TRY(cudaMemcpyAsync(out, s->io_out, out_bytes, cudaMemcpyDeviceToHost, st));
   HYP_CUDA_TRY(cudaStreamSynchronize(st));
   int dev_err = 0;
   rc = tc_error_flag(&dev_err);
@@ -391,6 +468,10 @@ extern "C" void hyp_stage_destroy(hyp_stage* s) {
     if (s->meta_ev[i]) cudaEventDestroy(s->meta_ev[i]);
   }
   for (cudaEvent_t e : s->time_ev) cudaEventDestroy(e);
+  for (auto& g : s->graphs)
+    if (g.exec) cudaGraphExecDestroy(g.exec);
+  if (s->cap_stream) cudaStreamDestroy(s->cap_stream);
+  cudaFree(s->g_in); cudaFree(s->g_out);
   delete s;
 }
 
@@ -488,6 +569,9 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
                             : (size_t)s->max_rows * d.H * sizeof(float);
   TRY_CUDA(cudaMalloc(&s->io_in, s->io_in_bytes));
   TRY_CUDA(cudaMalloc(&s->io_out, s->io_out_bytes));
+  TRY_CUDA(cudaMalloc(&s->g_in, (size_t)HYP_MAX_DECODE_BATCH * std::max((size_t)d.H * sizeof(float), sizeof(int32_t))));
+  TRY_CUDA(cudaMalloc(&s->g_out, (size_t)HYP_MAX_DECODE_BATCH * std::max(d.H, d.V) * sizeof(float)));
+  TRY_CUDA(cudaStreamCreateWithFlags(&s->cap_stream, cudaStreamNonBlocking));
   // tensor-core operand descriptors over the fixed workspace buffers
   TRY(tc_prepare());
   TRY(tc_make_act(&s->tc_h, s->h, (int)rows_pad, d.H));
