@@ -7,7 +7,10 @@
  * sequence; hyp_stage_* (hyperion.h) is the full path.  All pointers are DEVICE unless marked HOST;
  * `stream` is a cudaStream_t as void*; calls enqueue and return; status codes as in hyperion.h.
  *
- * KV page pool layout of ONE block (bf16): [n_pages][2 (K then V)][n_kv_heads][16 tokens][head_dim].
+ * KV page pool layout of ONE block (fp16): [n_pages][2 (K then V)][n_kv_heads][16 tokens][head_dim].
+ * Attention operands (queries, cached keys and values) are IEEE fp16: the softmax weights need more
+ * mantissa than bf16 offers to stay inside the library's logit tolerance; values are saturated at
+ * +-65504 when the library writes them.
  * A block table row lists, in order, the page ids that hold a sequence's tokens 0-15, 16-31, ...
  */
 #ifndef HYPERION_OPS_H
@@ -52,7 +55,7 @@ HYP_API size_t hyp_op_attn_decode_scratch_bytes(int32_t n_seqs, int32_t n_q_head
 /* Decode attention (grouped-query attention of Section III-A for one new token per sequence):
  * out[b, h, :] = softmax_j(q[b, h, :] . k[b, j, h/G, :] / sqrt(D)) v[b, j, h/G, :] over cached
  * positions j = 0 .. ctx_lens[b] (the new token's k, v must already be in the cache).
- *   q          bf16 [n_seqs, q_stride], head h of row b at q + b*q_stride + h*D (already rotated)
+ *   q          fp16 [n_seqs, q_stride], head h of row b at q + b*q_stride + h*D (already rotated)
  *   kv_pages   one block's page pool (layout above)
  *   block_table int32 [n_seqs, max_pages_per_seq];  ctx_lens int32 [n_seqs]
  *   scratch    fp32, at least hyp_op_attn_decode_scratch_bytes(...) bytes: per-split partial results
@@ -95,7 +98,7 @@ HYP_API int hyp_op_attn_decode_static(const hyp_attn_shape* shape, int32_t n_seq
  * owns rows cu_q[i] .. cu_q[i+1]-1; its row r sits at absolute position ctx_lens[i] + (r - cu_q[i]) and
  * sees cached positions 0 .. its own (all of the sequence's k, v, new rows included, must already be in
  * the cache).
- *   q bf16 [M, q_stride]; cu_q int32 [n_seqs + 1] (cu_q[n_seqs] = M); ctx_lens int32 [n_seqs];
+ *   q fp16 [M, q_stride]; cu_q int32 [n_seqs + 1] (cu_q[n_seqs] = M); ctx_lens int32 [n_seqs];
  *   block_table int32 [n_seqs, max_pages_per_seq]; out bf16 [M, n_q_heads * D]. */
 HYP_API int hyp_op_attn_prefill(const hyp_attn_shape* shape, int32_t n_seqs, int32_t M, const void* q,
                                 int32_t q_stride, const void* kv_pages, const int32_t* block_table,

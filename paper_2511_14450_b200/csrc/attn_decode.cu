@@ -4,7 +4,7 @@
 //   partial kernel: grid (n_splits, Hkv, n_seqs), 4 warps.  A CTA streams its context slice of one KV
 //   head through shared memory in 64-token tiles (double-buffered cp.async, 128-bit, each byte read
 //   once) and serves the G = Hq/Hkv query heads that share the head as the rows of one
-//   mma.sync.m16n8k16 operand (rows >= G are padding).  Warp w owns keys 16w..16w+15 of every tile:
+//   mma.sync.m16n8k16 operand (rows >= G are padding; q, k, v and the softmax weights are fp16).  Warp w owns keys 16w..16w+15 of every tile:
 //   it forms their scores, keeps its own online-softmax state and its own O += P V partial, so there is
 //   no cross-warp traffic inside the loop; the four warps are combined once at the end.  Tensor cores
 //   are used because the scalar version needs ~130 instructions per KB of cache and is issue-bound at
@@ -36,7 +36,7 @@ int attn_decode_splits(int n_seqs, int Hkv, int max_ctx) {
 
 template <int D, int G>
 __global__ void __launch_bounds__(AD_WARPS * 32)
-attn_decode_partial_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfloat16* __restrict__ kv_layer,
+attn_decode_partial_kernel(const __half* __restrict__ qkv, const __half* __restrict__ kv_layer,
                            float* __restrict__ part_acc, float* __restrict__ part_ml, int n_splits,
                            BatchMeta bm, ModelDims d) {
   constexpr int KS = D / 16, DN = D / 8, CPR = D / 8, PT = 16;
@@ -68,7 +68,7 @@ attn_decode_partial_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfl
       const int key = t_begin + j * AD_TILE + r;
       const bool ok = key < t_end;
       const int kk = ok ? key : t_begin;
-      const __nv_bfloat16* src =
+      const __half* src =
           kv_layer + (size_t)bt[kk / PT] * page_elems + ((size_t)kvh * PT + (kk % PT)) * D + c * 8;
       cp_async16(k_tile(buf) + tile_off<D>(r, c), src, ok);
       cp_async16(v_tile(buf) + tile_off<D>(r, c), src + v_off, ok);
@@ -80,7 +80,7 @@ attn_decode_partial_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfl
   // query heads kvh*G .. kvh*G+G-1 of row b as operand rows 0..G-1 (rows G..15 are zero)
   uint32_t qf[KS][2];  // [k step][k half]; only the "row g" halves of the fragment are non-zero
   {
-    const __nv_bfloat16* qrow = qkv + (size_t)b * d.qkv_rows + (size_t)(kvh * G + (g < G ? g : 0)) * D;
+    const __half* qrow = qkv + (size_t)b * d.qkv_rows + (size_t)(kvh * G + (g < G ? g : 0)) * D;
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
       qf[ks][0] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * tq) : 0u;
@@ -111,8 +111,8 @@ attn_decode_partial_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfl
       const int c = 2 * ks + ((lane >> 3) & 1);
       uint32_t b0, b1, b2, b3;
       ldsm_x4(k_tile(buf) + tile_off<D>(r, c), b0, b1, b2, b3);
-      mma_bf16_16816(s[0], qf[ks][0], 0u, qf[ks][1], 0u, b0, b1);
-      mma_bf16_16816(s[1], qf[ks][0], 0u, qf[ks][1], 0u, b2, b3);
+      mma_f16_16816(s[0], qf[ks][0], 0u, qf[ks][1], 0u, b0, b1);
+      mma_f16_16816(s[1], qf[ks][0], 0u, qf[ks][1], 0u, b2, b3);
     }
     const int key0 = t_begin + j * AD_TILE + 16 * warp + 2 * tq;
     float mx = m_run;
@@ -138,7 +138,7 @@ attn_decode_partial_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfl
         sum += p[nt][e];
       }
     l_run = l_run * corr + sum;
-    const uint32_t pa0 = pack_bf16(p[0][0], p[0][1]), pa2 = pack_bf16(p[1][0], p[1][1]);
+    const uint32_t pa0 = pack_f16(p[0][0], p[0][1]), pa2 = pack_f16(p[1][0], p[1][1]);
 #pragma unroll
     for (int dp = 0; dp < DN / 2; ++dp) {
       const int r = 16 * warp + (lane & 7) + (((lane >> 3) & 1) << 3);
@@ -147,8 +147,8 @@ attn_decode_partial_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfl
       ldsm_x4_t(v_tile(buf) + tile_off<D>(r, c), b0, b1, b2, b3);
       float c0[4] = {o[2 * dp][0] * corr, o[2 * dp][1] * corr, 0.f, 0.f};
       float c1[4] = {o[2 * dp + 1][0] * corr, o[2 * dp + 1][1] * corr, 0.f, 0.f};
-      mma_bf16_16816(c0, pa0, 0u, pa2, 0u, b0, b1);
-      mma_bf16_16816(c1, pa0, 0u, pa2, 0u, b2, b3);
+      mma_f16_16816(c0, pa0, 0u, pa2, 0u, b0, b1);
+      mma_f16_16816(c1, pa0, 0u, pa2, 0u, b2, b3);
       o[2 * dp][0] = c0[0]; o[2 * dp][1] = c0[1];
       o[2 * dp + 1][0] = c1[0]; o[2 * dp + 1][1] = c1[1];
     }
@@ -217,7 +217,7 @@ __global__ void attn_decode_merge_kernel(const float* __restrict__ part_acc, con
 }
 
 template <int D, int G>
-static int launch_dg(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __nv_bfloat16* attn_out,
+static int launch_dg(const __half* qkv, const __half* kv_layer, __nv_bfloat16* attn_out,
                      float* scratch, int n_splits, const BatchMeta& bm, const ModelDims& d, cudaStream_t st) {
   static bool configured = false;
   constexpr int smem = 4 * AD_TILE * D * 2;  // K[2] + V[2]; also covers the end-of-kernel combine buffers
@@ -235,8 +235,10 @@ static int launch_dg(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __
   return 2;
 }
 
-int launch_attn_decode(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __nv_bfloat16* attn_out,
-                       float* scratch, int n_splits, const BatchMeta& bm, const ModelDims& d, cudaStream_t st) {
+int launch_attn_decode(const __half* qkv, int q_stride, const __half* kv_layer, __nv_bfloat16* attn_out,
+                       float* scratch, int n_splits, const BatchMeta& bm, const ModelDims& d_in, cudaStream_t st) {
+  ModelDims d = d_in;
+  d.qkv_rows = q_stride;
   const int G = d.Hq / d.Hkv;
 #define HYP_AD_CASE(DD, GG) \
   if (d.D == DD && G == GG) return launch_dg<DD, GG>(qkv, kv_layer, attn_out, scratch, n_splits, bm, d, st);

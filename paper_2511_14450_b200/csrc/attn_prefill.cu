@@ -2,8 +2,9 @@
 //
 // Flash-attention tiling on tensor cores: one CTA = 64 query rows of one sequence and one query head
 // (4 warps x 16 rows); keys/values stream through shared memory in 64-token tiles (4 pages) with
-// double-buffered cp.async; S = Q K^T and O += P V run on mma.sync.m16n8k16 (bf16 in, fp32 accumulate),
-// the probabilities never leave registers.  New rows of a sequence sit at positions
+// double-buffered cp.async; S = Q K^T and O += P V run on mma.sync.m16n8k16 (fp16 in, fp32 accumulate: q, k,
+// v and the softmax weights carry 11 mantissa bits - bf16's 8 bits alone cost ~0.5 % error in the softmax
+// weights), the probabilities never leave registers.  New rows of a sequence sit at positions
 // ctx_len .. ctx_len + q_len - 1 and see every cached position up to their own (their k, v were
 // appended by the RoPE / KV-write kernel beforehand), so chunked prefill needs no special case.
 #include "attn_common.cuh"
@@ -17,7 +18,7 @@ constexpr int FA_BQ = 64, FA_BKV = 64, FA_THREADS = 128, PT = 16;
 
 template <int D>
 __global__ void __launch_bounds__(FA_THREADS)
-attn_prefill_fa_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfloat16* __restrict__ kv_layer,
+attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict__ kv_layer,
                        __nv_bfloat16* __restrict__ out, BatchMeta bm, ModelDims d) {
   constexpr int KS = D / 16;       // k-steps of the QK^T contraction
   constexpr int DN = D / 8;        // 8-wide output column tiles of O
@@ -61,7 +62,7 @@ attn_prefill_fa_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfloat1
       const int key = j * FA_BKV + r;
       const bool ok = key < kv_total;
       const int kk = ok ? key : 0;
-      const __nv_bfloat16* src =
+      const __half* src =
           kv_layer + (size_t)bt[kk / PT] * page_elems + ((size_t)kvh * PT + (kk % PT)) * D + c * 8;
       cp_async16(k_tile(buf) + tile_off<D>(r, c), src, ok);
       cp_async16(v_tile(buf) + tile_off<D>(r, c), src + v_off, ok);
@@ -75,8 +76,8 @@ attn_prefill_fa_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfloat1
   uint32_t qf[KS][4];
   {
     const int r_lo = 16 * warp + g, r_hi = r_lo + 8;
-    const __nv_bfloat16* q_lo = qkv + (size_t)(row_base + r_lo) * d.qkv_rows + (size_t)hq * D;
-    const __nv_bfloat16* q_hi = qkv + (size_t)(row_base + r_hi) * d.qkv_rows + (size_t)hq * D;
+    const __half* q_lo = qkv + (size_t)(row_base + r_lo) * d.qkv_rows + (size_t)hq * D;
+    const __half* q_hi = qkv + (size_t)(row_base + r_hi) * d.qkv_rows + (size_t)hq * D;
     const bool ok_lo = r_lo < rows_here, ok_hi = r_hi < rows_here;
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
@@ -116,8 +117,8 @@ attn_prefill_fa_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfloat1
         const int c = 2 * ks + ((lane >> 3) & 1);
         uint32_t b0, b1, b2, b3;
         ldsm_x4(k_tile(buf) + tile_off<D>(r, c), b0, b1, b2, b3);
-        mma_bf16_16816(s[2 * np], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b0, b1);
-        mma_bf16_16816(s[2 * np + 1], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b2, b3);
+        mma_f16_16816(s[2 * np], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b0, b1);
+        mma_f16_16816(s[2 * np + 1], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b2, b3);
       }
     }
 
@@ -147,15 +148,15 @@ attn_prefill_fa_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfloat1
     m_lo = mx_lo;
     m_hi = mx_hi;
     float sum_lo = 0.f, sum_hi = 0.f;
-    uint32_t pf[8][2];  // probabilities as bf16 pairs: [key tile][row lo / hi]
+    uint32_t pf[8][2];  // probabilities as fp16 pairs: [key tile][row lo / hi]
 #pragma unroll
     for (int nt = 0; nt < 8; ++nt) {
       const float p0 = exp2f(s[nt][0] - mx_lo), p1 = exp2f(s[nt][1] - mx_lo);
       const float p2 = exp2f(s[nt][2] - mx_hi), p3 = exp2f(s[nt][3] - mx_hi);
       sum_lo += p0 + p1;
       sum_hi += p2 + p3;
-      pf[nt][0] = pack_bf16(p0, p1);
-      pf[nt][1] = pack_bf16(p2, p3);
+      pf[nt][0] = pack_f16(p0, p1);
+      pf[nt][1] = pack_f16(p2, p3);
     }
     l_lo = l_lo * corr_lo + sum_lo;
     l_hi = l_hi * corr_hi + sum_hi;
@@ -174,8 +175,8 @@ attn_prefill_fa_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfloat1
         const int c = 2 * dp + (lane >> 4);
         uint32_t b0, b1, b2, b3;
         ldsm_x4_t(v_tile(buf) + tile_off<D>(r, c), b0, b1, b2, b3);
-        mma_bf16_16816(o[2 * dp], pf[2 * kk][0], pf[2 * kk][1], pf[2 * kk + 1][0], pf[2 * kk + 1][1], b0, b1);
-        mma_bf16_16816(o[2 * dp + 1], pf[2 * kk][0], pf[2 * kk][1], pf[2 * kk + 1][0], pf[2 * kk + 1][1], b2, b3);
+        mma_f16_16816(o[2 * dp], pf[2 * kk][0], pf[2 * kk][1], pf[2 * kk + 1][0], pf[2 * kk + 1][1], b0, b1);
+        mma_f16_16816(o[2 * dp + 1], pf[2 * kk][0], pf[2 * kk][1], pf[2 * kk + 1][0], pf[2 * kk + 1][1], b2, b3);
       }
     }
     __syncthreads();  // everyone is done with `buf` before the next iteration's loads overwrite it
@@ -201,7 +202,7 @@ attn_prefill_fa_kernel(const __nv_bfloat16* __restrict__ qkv, const __nv_bfloat1
 }
 
 template <int D>
-int launch_fa(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __nv_bfloat16* attn_out, const BatchMeta& bm,
+int launch_fa(const __half* qkv, const __half* kv_layer, __nv_bfloat16* attn_out, const BatchMeta& bm,
               const ModelDims& d, cudaStream_t st) {
   static bool configured = false;
   constexpr int smem = 4 * FA_BKV * D * 2;
@@ -218,11 +219,13 @@ int launch_fa(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __nv_bflo
 
 }  // namespace
 
-// Needs bm.cu_q, bm.ctx_lens, bm.block_table, bm.n_seqs, bm.n_tokens.
-int launch_attn_prefill(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __nv_bfloat16* attn_out,
-                        const BatchMeta& bm, const ModelDims& d, cudaStream_t st) {
-  if (d.D == 128) return launch_fa<128>(qkv, kv_layer, attn_out, bm, d, st);
-  if (d.D == 64) return launch_fa<64>(qkv, kv_layer, attn_out, bm, d, st);
+// Needs bm.cu_q, bm.ctx_lens, bm.block_table, bm.n_seqs, bm.n_tokens.  Head h of row t: q + t*q_stride + h*D.
+int launch_attn_prefill(const __half* q, int q_stride, const __half* kv_layer, __nv_bfloat16* attn_out,
+                        const BatchMeta& bm, const ModelDims& d_in, cudaStream_t st) {
+  ModelDims d = d_in;
+  d.qkv_rows = q_stride;
+  if (d.D == 128) return launch_fa<128>(q, kv_layer, attn_out, bm, d, st);
+  if (d.D == 64) return launch_fa<64>(q, kv_layer, attn_out, bm, d, st);
   return HYP_EINVAL;
 }
 

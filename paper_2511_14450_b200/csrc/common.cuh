@@ -1,6 +1,7 @@
 // Shared device helpers and the internal kernel-launch interface of libhyperion.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -53,6 +54,23 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
       "{%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ void mma_f16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_f16(float a, float b) {
+  __half2 p = __floats2half2_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+// fp32 -> fp16 with saturation at the largest finite value (the attention operands are fp16)
+__device__ __forceinline__ uint32_t pack_f16_sat(float a, float b) {
+  return pack_f16(fminf(fmaxf(a, -65504.f), 65504.f), fminf(fmaxf(b, -65504.f), 65504.f));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -112,7 +130,7 @@ struct ModelDims {
   float eps, theta;
 };
 
-// KV pool of ONE layer: [n_pages][2 (K,V)][Hkv][page_tokens][D] bf16
+// KV pool of ONE layer: [n_pages][2 (K,V)][Hkv][page_tokens][D] fp16
 __host__ __device__ __forceinline__ size_t kv_page_elems(int Hkv, int page_tokens, int D) {
   return (size_t)2 * Hkv * page_tokens * D;
 }
@@ -122,7 +140,9 @@ enum Epilogue : int {
   EPI_STORE_BF16 = 0,  // out_bf16[m, n] = acc
   EPI_RESID_F32 = 1,   // out_f32[m, n] += acc         (residual stream)
   EPI_SWIGLU_BF16 = 2, // out_bf16[m, n] = silu(acc_gate) * acc_up, gate row n, up row n + N
-  EPI_STORE_F32 = 3    // out_f32[m, n] = acc          (logits)
+  EPI_STORE_F32 = 3,   // out_f32[m, n] = acc          (logits, q/k/v)
+  EPI_PAIR_F32 = 4     // weight-streaming kernel only: activation rows come as (high part, low part) pairs
+                       // stacked 8*NB/2 rows apart; out_f32[m, n] = acc[m] + acc[m + 8*NB/2]
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -130,16 +150,19 @@ enum Epilogue : int {
 // ---------------------------------------------------------------------------------------------
 int launch_embed(const int32_t* ids, const __nv_bfloat16* E, float* x, int M, int H, int V, cudaStream_t st);
 int launch_copy_f32(const float* src, float* dst, size_t n, cudaStream_t st);
-int launch_rmsnorm(const float* x, const __nv_bfloat16* g, __nv_bfloat16* h, int M, int H, float eps,
-                   const int32_t* row_index /* optional gather of rows, may be null */, cudaStream_t st);
-int launch_rope_kv_write(__nv_bfloat16* qkv, __nv_bfloat16* kv_layer, const float2* rope_table,
+// h = bf16(norm(x)); if h_lo is given, also h_lo = bf16(norm(x) - h): the pair carries ~16 mantissa bits
+int launch_rmsnorm(const float* x, const __nv_bfloat16* g, __nv_bfloat16* h, __nv_bfloat16* h_lo, int M, int H,
+                   float eps, const int32_t* row_index /* optional gather of rows, may be null */, cudaStream_t st);
+// rotate q, k of every row (fp32 in), write q as fp16 [M, Hq*D] and append k, v as fp16 to the pages
+int launch_rope_kv_write(const float* qkv, __half* q16, __half* kv_layer, const float2* rope_table,
                          const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
-int launch_attn_prefill(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __nv_bfloat16* attn_out,
+// q: fp16 [M, q_stride]
+int launch_attn_prefill(const __half* q, int q_stride, const __half* kv_layer, __nv_bfloat16* attn_out,
                         const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
 // decode attention: one query row per sequence; `scratch` holds split partials
 size_t attn_decode_scratch_bytes(int max_seqs, int Hq, int D, int max_splits);
 int attn_decode_splits(int n_seqs, int Hkv, int max_ctx);
-int launch_attn_decode(const __nv_bfloat16* qkv, const __nv_bfloat16* kv_layer, __nv_bfloat16* attn_out,
+int launch_attn_decode(const __half* q, int q_stride, const __half* kv_layer, __nv_bfloat16* attn_out,
                        float* scratch, int n_splits, const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
 
 }  // namespace hyp

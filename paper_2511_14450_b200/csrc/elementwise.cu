@@ -45,10 +45,11 @@ int launch_copy_f32(const float* src, float* dst, size_t n, cudaStream_t st) {
 }
 
 // h[r, :] = x[row, :] * rsqrt(mean(x[row, :]^2) + eps) * g, one CTA per output row.
-// row = row_index ? row_index[r] : r.  fp32 statistics, bf16 output.
+// row = row_index ? row_index[r] : r.  fp32 statistics, bf16 output.  With h_lo the rounding residue
+// bf16(y - bf16(y)) is stored too, so that a projection fed with both parts sees ~16 mantissa bits.
 template <int THREADS>
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ g,
-                               __nv_bfloat16* __restrict__ h, int H, float eps,
+                               __nv_bfloat16* __restrict__ h, __nv_bfloat16* __restrict__ h_lo, int H, float eps,
                                const int32_t* __restrict__ row_index) {
   __shared__ float red[THREADS / 32];
   pdl_trigger();
@@ -71,27 +72,38 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16*
   const float rstd = rsqrtf(tot / (float)H + eps);
   const uint2* gr = reinterpret_cast<const uint2*>(g);
   uint2* hr = reinterpret_cast<uint2*>(h + (size_t)r * H);
+  uint2* lr = h_lo ? reinterpret_cast<uint2*>(h_lo + (size_t)r * H) : nullptr;
   for (int i = threadIdx.x; i < n4; i += THREADS) {
     const float4 v = xr[i];
     const uint2 gg = gr[i];
+    const float y0 = v.x * rstd * bf16_lo(gg.x), y1 = v.y * rstd * bf16_hi(gg.x);
+    const float y2 = v.z * rstd * bf16_lo(gg.y), y3 = v.w * rstd * bf16_hi(gg.y);
     uint2 o;
-    o.x = pack_bf16(v.x * rstd * bf16_lo(gg.x), v.y * rstd * bf16_hi(gg.x));
-    o.y = pack_bf16(v.z * rstd * bf16_lo(gg.y), v.w * rstd * bf16_hi(gg.y));
+    o.x = pack_bf16(y0, y1);
+    o.y = pack_bf16(y2, y3);
     hr[i] = o;
+    if (lr) {
+      uint2 l;
+      l.x = pack_bf16(y0 - bf16_lo(o.x), y1 - bf16_hi(o.x));
+      l.y = pack_bf16(y2 - bf16_lo(o.y), y3 - bf16_hi(o.y));
+      lr[i] = l;
+    }
   }
 }
 
-int launch_rmsnorm(const float* x, const __nv_bfloat16* g, __nv_bfloat16* h, int M, int H, float eps,
-                   const int32_t* row_index, cudaStream_t st) {
-  HYP_CUDA_TRY(launch_pdl(rmsnorm_kernel<256>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
+int launch_rmsnorm(const float* x, const __nv_bfloat16* g, __nv_bfloat16* h, __nv_bfloat16* h_lo, int M, int H,
+                   float eps, const int32_t* row_index, cudaStream_t st) {
+  HYP_CUDA_TRY(launch_pdl(rmsnorm_kernel<256>, dim3(M), dim3(256), 0, st, x, g, h, h_lo, H, eps, row_index));
   return 1;
 }
 
 // Rotate q and k of every new row by its position and append k, v to the sequence's pages.
-// qkv row layout: [Q heads | K heads | V heads], each head D wide.  q is rotated in place.
+// Input row layout (fp32, straight from the projection's accumulators): [Q heads | K heads | V heads],
+// each head D wide.  Outputs are fp16 (rounded once): q to its own [M, Hq*D] buffer, k and v to the pages.
 // One thread handles 8 rotation pairs (i .. i+7, i+D/2 .. i+D/2+7) of one head of one row.
-__global__ void rope_kv_write_kernel(__nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ kv_layer,
-                                     const float2* __restrict__ rope_table, BatchMeta bm, ModelDims d) {
+__global__ void rope_kv_write_kernel(const float* __restrict__ qkv, __half* __restrict__ q16,
+                                     __half* __restrict__ kv_layer, const float2* __restrict__ rope_table,
+                                     BatchMeta bm, ModelDims d) {
   pdl_trigger();
   pdl_wait();
   const int t = blockIdx.x;
@@ -102,51 +114,46 @@ __global__ void rope_kv_write_kernel(__nv_bfloat16* __restrict__ qkv, __nv_bfloa
   const int page = bm.block_table[(size_t)sq * bm.max_pages_per_seq + pos / d.page_tokens];
   const int slot = pos % d.page_tokens;
   const size_t page_base = (size_t)page * kv_page_elems(d.Hkv, d.page_tokens, d.D);
-  __nv_bfloat16* row = qkv + (size_t)t * d.qkv_rows;
+  const float* row = qkv + (size_t)t * d.qkv_rows;
   for (int w = threadIdx.x; w < n_heads * vec_per_head; w += blockDim.x) {
     const int head = w / vec_per_head;
     const int i0 = (w % vec_per_head) * 8;
-    __nv_bfloat16* hp = row + (size_t)head * d.D;
-    const uint4 a = *reinterpret_cast<const uint4*>(hp + i0);
-    const uint4 b = *reinterpret_cast<const uint4*>(hp + d.D / 2 + i0);
+    const float* hp = row + (size_t)head * d.D;
+    float a[8], b[8];
+    *reinterpret_cast<float4*>(a) = *reinterpret_cast<const float4*>(hp + i0);
+    *reinterpret_cast<float4*>(a + 4) = *reinterpret_cast<const float4*>(hp + i0 + 4);
+    *reinterpret_cast<float4*>(b) = *reinterpret_cast<const float4*>(hp + d.D / 2 + i0);
+    *reinterpret_cast<float4*>(b + 4) = *reinterpret_cast<const float4*>(hp + d.D / 2 + i0 + 4);
+    __half* dst;
     if (head < d.Hq + d.Hkv) {
       const float2* cs = rope_table + (size_t)pos * (d.D / 2) + i0;
-      const uint32_t av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
-      uint32_t oa[4], ob[4];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float2 c0 = cs[2 * j], c1 = cs[2 * j + 1];
-        const float x1a = bf16_lo(av[j]), x1b = bf16_hi(av[j]);
-        const float x2a = bf16_lo(bv[j]), x2b = bf16_hi(bv[j]);
-        oa[j] = pack_bf16(x1a * c0.x - x2a * c0.y, x1b * c1.x - x2b * c1.y);
-        ob[j] = pack_bf16(x2a * c0.x + x1a * c0.y, x2b * c1.x + x1b * c1.y);
+      for (int j = 0; j < 8; ++j) {
+        const float2 c = cs[j];
+        const float x1 = a[j], x2 = b[j];
+        a[j] = x1 * c.x - x2 * c.y;
+        b[j] = x2 * c.x + x1 * c.y;
       }
-      const uint4 ra = make_uint4(oa[0], oa[1], oa[2], oa[3]), rb = make_uint4(ob[0], ob[1], ob[2], ob[3]);
-      if (head < d.Hq) {
-        *reinterpret_cast<uint4*>(hp + i0) = ra;
-        *reinterpret_cast<uint4*>(hp + d.D / 2 + i0) = rb;
-      } else {
-        const int kvh = head - d.Hq;
-        __nv_bfloat16* dst = kv_layer + page_base + ((size_t)kvh * d.page_tokens + slot) * d.D;
-        *reinterpret_cast<uint4*>(dst + i0) = ra;
-        *reinterpret_cast<uint4*>(dst + d.D / 2 + i0) = rb;
-      }
+      dst = head < d.Hq ? q16 + (size_t)t * d.Hq * d.D + (size_t)head * d.D
+                        : kv_layer + page_base + ((size_t)(head - d.Hq) * d.page_tokens + slot) * d.D;
     } else {
-      const int kvh = head - d.Hq - d.Hkv;
-      __nv_bfloat16* dst = kv_layer + page_base + (size_t)d.Hkv * d.page_tokens * d.D +
-                           ((size_t)kvh * d.page_tokens + slot) * d.D;
-      *reinterpret_cast<uint4*>(dst + i0) = a;
-      *reinterpret_cast<uint4*>(dst + d.D / 2 + i0) = b;
+      dst = kv_layer + page_base + (size_t)d.Hkv * d.page_tokens * d.D +
+            ((size_t)(head - d.Hq - d.Hkv) * d.page_tokens + slot) * d.D;
     }
+    *reinterpret_cast<uint4*>(dst + i0) =
+        make_uint4(pack_f16_sat(a[0], a[1]), pack_f16_sat(a[2], a[3]), pack_f16_sat(a[4], a[5]), pack_f16_sat(a[6], a[7]));
+    *reinterpret_cast<uint4*>(dst + d.D / 2 + i0) =
+        make_uint4(pack_f16_sat(b[0], b[1]), pack_f16_sat(b[2], b[3]), pack_f16_sat(b[4], b[5]), pack_f16_sat(b[6], b[7]));
   }
 }
 
-int launch_rope_kv_write(__nv_bfloat16* qkv, __nv_bfloat16* kv_layer, const float2* rope_table,
+int launch_rope_kv_write(const float* qkv, __half* q16, __half* kv_layer, const float2* rope_table,
                          const BatchMeta& bm, const ModelDims& d, cudaStream_t st) {
   const int work = (d.Hq + 2 * d.Hkv) * (d.D / 16);
   int threads = ((work + 31) / 32) * 32;
   if (threads > 512) threads = 512;
-  HYP_CUDA_TRY(launch_pdl(rope_kv_write_kernel, dim3(bm.n_tokens), dim3(threads), 0, st, qkv, kv_layer, rope_table, bm, d));
+  HYP_CUDA_TRY(launch_pdl(rope_kv_write_kernel, dim3(bm.n_tokens), dim3(threads), 0, st, qkv, q16, kv_layer, rope_table,
+                          bm, d));
   return 1;
 }
 

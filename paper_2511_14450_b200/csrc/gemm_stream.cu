@@ -159,7 +159,9 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
     for (int ww = 0; ww < GS_WARPS; ++ww) {
       v += red[ww][r][m];
       if (SWIGLU) v2 += red[ww][16 + r][m];
+      if (EPI == EPI_PAIR_F32) v2 += red[ww][r][m + 4 * NB];  // the low parts sit 8*NB/2 token rows further on
     }
+    if (EPI == EPI_PAIR_F32) v += v2;
     const size_t o = (size_t)m * ldo + n;
     if (EPI == EPI_STORE_BF16) {
       reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(v);
@@ -226,15 +228,25 @@ int launch_nb(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi,
       return wide ? launch_cfg<NB, EPI_STORE_F32, 2>(act, w, M, N, K, out, ldo, st)
                   : launch_cfg<NB, EPI_STORE_F32, 1>(act, w, M, N, K, out, ldo, st);
     case EPI_SWIGLU_BF16: return launch_cfg<NB, EPI_SWIGLU_BF16, 2>(act, w, M, N, K, out, ldo, st);
+    case EPI_PAIR_F32:
+      if (NB % 2) return HYP_EINVAL;
+      return wide ? launch_cfg<NB, EPI_PAIR_F32, 2>(act, w, M, N, K, out, ldo, st)
+                  : launch_cfg<NB, EPI_PAIR_F32, 1>(act, w, M, N, K, out, ldo, st);
     default: return HYP_EINVAL;
   }
 }
 
 }  // namespace
 
+// EPI_PAIR_F32: the activation matrix holds the high parts in rows [0, M) and the low parts in rows
+// [8 nb, 8 nb + M) with nb = ceil(M / 8); M <= 16.
 int launch_gemm_stream(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
                        cudaStream_t st) {
   if (M < 1 || M > 32 || N < 1 || K < 8 || act.K != K || w.K != K || !tc_err_flag_ptr()) return HYP_EINVAL;
+  if (epi == EPI_PAIR_F32) {
+    if (M > 16) return HYP_EINVAL;
+    return M <= 8 ? launch_nb<2>(act, w, M, N, K, epi, out, ldo, st) : launch_nb<4>(act, w, M, N, K, epi, out, ldo, st);
+  }
   switch ((M + 7) / 8) {
     case 1: return launch_nb<1>(act, w, M, N, K, epi, out, ldo, st);
     case 2: return launch_nb<2>(act, w, M, N, K, epi, out, ldo, st);

@@ -35,7 +35,8 @@ int finish(int rc) {
 
 extern "C" int hyp_op_rmsnorm(const float* x, const void* g, void* out, int32_t M, int32_t H, float eps, void* stream) {
   if (!x || !g || !out || M < 1 || H < 8 || H % 8 || !(eps > 0.f)) return HYP_EINVAL;
-  return finish(launch_rmsnorm(x, (const __nv_bfloat16*)g, (__nv_bfloat16*)out, M, H, eps, nullptr, (cudaStream_t)stream));
+  return finish(launch_rmsnorm(x, (const __nv_bfloat16*)g, (__nv_bfloat16*)out, nullptr, M, H, eps, nullptr,
+                               (cudaStream_t)stream));
 }
 
 extern "C" int hyp_op_gemm(const void* a, const void* w, int32_t M, int32_t N, int32_t K, int32_t epilogue, void* out,
@@ -82,7 +83,7 @@ extern "C" int hyp_op_attn_decode(const hyp_attn_shape* shape, int32_t n_seqs, c
   bm.ctx_lens = ctx_lens;
   bm.block_table = block_table;
   const ModelDims d = attn_dims(shape, q_stride);
-  return finish(launch_attn_decode((const __nv_bfloat16*)q, (const __nv_bfloat16*)kv_pages, (__nv_bfloat16*)out, scratch,
+  return finish(launch_attn_decode((const __half*)q, q_stride, (const __half*)kv_pages, (__nv_bfloat16*)out, scratch,
                                    n_splits, bm, d, (cudaStream_t)stream));
 }
 
@@ -101,6 +102,6 @@ extern "C" int hyp_op_attn_prefill(const hyp_attn_shape* shape, int32_t n_seqs, 
   bm.ctx_lens = ctx_lens;
   bm.block_table = block_table;
   const ModelDims d = attn_dims(shape, q_stride);
-  return finish(launch_attn_prefill((const __nv_bfloat16*)q, (const __nv_bfloat16*)kv_pages, (__nv_bfloat16*)out, bm, d,
+  return finish(launch_attn_prefill((const __half*)q, q_stride, (const __half*)kv_pages, (__nv_bfloat16*)out, bm, d,
                                     (cudaStream_t)stream));
 }

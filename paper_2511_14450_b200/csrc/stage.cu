@@ -40,8 +40,8 @@ struct hyp_stage {
   bf16 *embed = nullptr, *gf = nullptr, *wlm = nullptr;
   TcWeight tc_lm;
   uint32_t loaded_extra = 0;
-  // KV cache
-  bf16* kv_pool = nullptr;
+  // KV cache (fp16)
+  __half* kv_pool = nullptr;
   size_t kv_layer_elems = 0;
   int n_pages = 0, max_pages_per_seq = 0;
   std::vector<int32_t> free_pages;
@@ -50,8 +50,10 @@ struct hyp_stage {
   // workspace
   int max_rows = 0;
   float* x = nullptr;
-  bf16 *h = nullptr, *qkv = nullptr, *attn = nullptr, *u = nullptr;
-  TcAct tc_h, tc_attn, tc_u;
+  float* qkv32 = nullptr;             // q | k | v straight from the projection's accumulators
+  __half* q16 = nullptr;              // rotated queries
+  bf16 *h = nullptr, *h_lo = nullptr, *h_pair = nullptr, *attn = nullptr, *u = nullptr;
+  TcAct tc_h, tc_h_lo, tc_h_pair, tc_attn, tc_u;
   float* attn_scratch = nullptr;
   int max_splits = 32;
   float2* rope_table = nullptr;
@@ -257,18 +259,32 @@ int run_blocks(hyp_stage* s, const BatchMeta& bm, bool decode, int n_splits, cud
   if (marks) HYP_CUDA_TRY(cudaEventRecord(marks[0], st));
   for (int li = 0; li < s->L; ++li) {
     LayerW& lw = s->layers[li];
-    bf16* kv_layer = s->kv_pool + (size_t)li * s->kv_layer_elems;
-    HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g1, s->h, M, d.H, d.eps, nullptr, st));
-    HYP_LAUNCH_T(HYP_K_GEMM_QKV, project(s, s->tc_h, s->h, d.H, lw.tc_qkv, lw.wqkv, d.qkv_rows, d.H, M,
-                                         EPI_STORE_BF16, s->qkv, d.qkv_rows, st));
-    HYP_LAUNCH_T(HYP_K_ROPE, launch_rope_kv_write(s->qkv, kv_layer, s->rope_table, bm, d, st));
+    __half* kv_layer = s->kv_pool + (size_t)li * s->kv_layer_elems;
+    // q, k, v are projected from the normalised activations split into a bf16 high and low part (the
+    // softmax is the one place where bf16's 8 mantissa bits on the inputs would not fit the tolerance)
+    if (M <= 16) {
+      // weight-streaming kernel: both parts ride along as extra token rows, the weights are read once
+      const int lo_row = 8 * ((M + 7) / 8);
+      HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g1, s->h_pair, s->h_pair + (size_t)lo_row * d.H, M, d.H, d.eps,
+                                              nullptr, st));
+      HYP_LAUNCH_T(HYP_K_GEMM_QKV, launch_gemm_stream(s->tc_h_pair, lw.tc_qkv, M, d.qkv_rows, d.H, EPI_PAIR_F32,
+                                                      s->qkv32, d.qkv_rows, st));
+    } else {
+      HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g1, s->h, s->h_lo, M, d.H, d.eps, nullptr, st));
+      HYP_LAUNCH_T(HYP_K_GEMM_QKV, project(s, s->tc_h, s->h, d.H, lw.tc_qkv, lw.wqkv, d.qkv_rows, d.H, M,
+                                           EPI_STORE_F32, s->qkv32, d.qkv_rows, st));
+      HYP_LAUNCH_T(HYP_K_GEMM_QKV, project(s, s->tc_h_lo, s->h_lo, d.H, lw.tc_qkv, lw.wqkv, d.qkv_rows, d.H, M,
+                                           EPI_RESID_F32, s->qkv32, d.qkv_rows, st));
+    }
+    HYP_LAUNCH_T(HYP_K_ROPE, launch_rope_kv_write(s->qkv32, s->q16, kv_layer, s->rope_table, bm, d, st));
     if (decode)
-      HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_decode(s->qkv, kv_layer, s->attn, s->attn_scratch, n_splits, bm, d, st));
+      HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_decode(s->q16, d.Hq * d.D, kv_layer, s->attn, s->attn_scratch, n_splits, bm,
+                                                  d, st));
     else
-      HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_prefill(s->qkv, kv_layer, s->attn, bm, d, st));
+      HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_prefill(s->q16, d.Hq * d.D, kv_layer, s->attn, bm, d, st));
     HYP_LAUNCH_T(HYP_K_GEMM_O, project(s, s->tc_attn, s->attn, d.Hq * d.D, lw.tc_o, lw.wo, d.H, d.Hq * d.D, M,
                                        EPI_RESID_F32, s->x, d.H, st));
-    HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g2, s->h, M, d.H, d.eps, nullptr, st));
+    HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g2, s->h, nullptr, M, d.H, d.eps, nullptr, st));
     HYP_LAUNCH_T(HYP_K_GEMM_GATE_UP, project(s, s->tc_h, s->h, d.H, lw.tc_gu, lw.wgu, d.F, d.H, M, EPI_SWIGLU_BF16,
                                              s->u, d.F, st));
     HYP_LAUNCH_T(HYP_K_GEMM_DOWN, project(s, s->tc_u, s->u, d.F, lw.tc_d, lw.wd, d.H, d.F, M, EPI_RESID_F32, s->x,
@@ -291,7 +307,7 @@ int enqueue_stage(hyp_stage* s, const BatchMeta& bm, int n_seqs, bool decode, bo
   if (rc) return rc;
   if (s->last) {
     const int rows = all_rows ? M : n_seqs;
-    HYP_LAUNCH(launch_rmsnorm(s->x, s->gf, s->h, rows, d.H, d.eps, all_rows ? nullptr : bm.last_row, st));
+    HYP_LAUNCH(launch_rmsnorm(s->x, s->gf, s->h, nullptr, rows, d.H, d.eps, all_rows ? nullptr : bm.last_row, st));
     HYP_LAUNCH_T(HYP_K_LM_HEAD,
                  project(s, s->tc_h, s->h, d.H, s->tc_lm, s->wlm, d.V, d.H, rows, EPI_STORE_F32, out, d.V, st));
   } else {
@@ -460,7 +476,8 @@ extern "C" void hyp_stage_destroy(hyp_stage* s) {
     cudaFree(lw.wqkv); cudaFree(lw.wo); cudaFree(lw.wgu); cudaFree(lw.wd); cudaFree(lw.g1); cudaFree(lw.g2);
   }
   cudaFree(s->embed); cudaFree(s->gf); cudaFree(s->wlm); cudaFree(s->kv_pool);
-  cudaFree(s->x); cudaFree(s->h); cudaFree(s->qkv); cudaFree(s->attn); cudaFree(s->u);
+  cudaFree(s->x); cudaFree(s->h); cudaFree(s->h_lo); cudaFree(s->h_pair); cudaFree(s->qkv32); cudaFree(s->q16);
+  cudaFree(s->attn); cudaFree(s->u);
   cudaFree(s->attn_scratch); cudaFree(s->rope_table); cudaFree(s->meta_dev);
   cudaFree(s->io_in); cudaFree(s->io_out);
   for (int i = 0; i < META_RING; ++i) {
@@ -523,7 +540,7 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
   s->n_pages = c.kv_pages > 0 ? c.kv_pages : c.max_seqs * s->max_pages_per_seq;
   s->kv_layer_elems = (size_t)s->n_pages * kv_page_elems(d.Hkv, d.page_tokens, d.D);
   TRY(dev_alloc(&s->kv_pool, s->kv_layer_elems * s->L));
-  TRY_CUDA(cudaMemset(s->kv_pool, 0, s->kv_layer_elems * s->L * sizeof(bf16)));
+  TRY_CUDA(cudaMemset(s->kv_pool, 0, s->kv_layer_elems * s->L * sizeof(__half)));
   s->free_pages.resize(s->n_pages);
   for (int i = 0; i < s->n_pages; ++i) s->free_pages[i] = s->n_pages - 1 - i;
   s->seq_pages.assign(c.max_seqs, {});
@@ -534,16 +551,22 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
   const size_t rows_pad = ((size_t)s->max_rows + 127) / 128 * 128;
   TRY(dev_alloc(&s->x, rows_pad * d.H));
   TRY(dev_alloc(&s->h, rows_pad * d.H));
-  TRY(dev_alloc(&s->qkv, rows_pad * d.qkv_rows));
+  TRY(dev_alloc(&s->h_lo, rows_pad * d.H));
+  TRY(dev_alloc(&s->h_pair, (size_t)64 * d.H));
+  TRY(dev_alloc(&s->qkv32, rows_pad * d.qkv_rows));
+  TRY(dev_alloc(&s->q16, rows_pad * d.Hq * d.D));
   TRY(dev_alloc(&s->attn, rows_pad * d.Hq * d.D));
   TRY(dev_alloc(&s->u, rows_pad * d.F));
   TRY_CUDA(cudaMemset(s->h, 0, rows_pad * d.H * sizeof(bf16)));
+  TRY_CUDA(cudaMemset(s->h_lo, 0, rows_pad * d.H * sizeof(bf16)));
+  TRY_CUDA(cudaMemset(s->h_pair, 0, (size_t)64 * d.H * sizeof(bf16)));
   TRY_CUDA(cudaMemset(s->attn, 0, rows_pad * d.Hq * d.D * sizeof(bf16)));
   TRY_CUDA(cudaMemset(s->u, 0, rows_pad * d.F * sizeof(bf16)));
   const size_t scratch_bytes =
       attn_decode_scratch_bytes(std::min(c.max_seqs, HYP_MAX_DECODE_BATCH), d.Hq, d.D, s->max_splits);
   TRY(dev_alloc(&s->attn_scratch, scratch_bytes / sizeof(float)));
-  s->workspace_bytes = rows_pad * ((size_t)d.H * 6 + ((size_t)d.qkv_rows + d.Hq * d.D + d.F) * 2) + scratch_bytes;
+  s->workspace_bytes = rows_pad * ((size_t)d.H * 8 + (size_t)d.qkv_rows * 4 + ((size_t)2 * d.Hq * d.D + d.F) * 2) +
+                       (size_t)64 * d.H * 2 + scratch_bytes;
   // rotary table: cos/sin of pos * theta^(-2i/D), angles evaluated in double on the host
   {
     const int half = d.D / 2;
@@ -575,6 +598,8 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
   // tensor-core operand descriptors over the fixed workspace buffers
   TRY(tc_prepare());
   TRY(tc_make_act(&s->tc_h, s->h, (int)rows_pad, d.H));
+  TRY(tc_make_act(&s->tc_h_lo, s->h_lo, (int)rows_pad, d.H));
+  TRY(tc_make_act(&s->tc_h_pair, s->h_pair, 64, d.H));
   TRY(tc_make_act(&s->tc_attn, s->attn, (int)rows_pad, d.Hq * d.D));
   TRY(tc_make_act(&s->tc_u, s->u, (int)rows_pad, d.F));
   for (LayerW& lw : s->layers) {
@@ -743,7 +768,7 @@ extern "C" int hyp_stage_profile(hyp_stage* s, int32_t mode, int32_t batch, int3
       layer_ms[li] = samples[iters / 2];
       const ModelDims& d = s->dims;
       const size_t wbytes = ((size_t)d.qkv_rows * d.H + (size_t)d.H * d.Hq * d.D + (size_t)3 * d.F * d.H + 2 * d.H) * 2;
-      layer_bytes[li] = wbytes + s->kv_layer_elems * sizeof(bf16) + s->workspace_bytes / s->L;
+      layer_bytes[li] = wbytes + s->kv_layer_elems * sizeof(__half) + s->workspace_bytes / s->L;
     }
   }
   for (auto& e : ev) cudaEventDestroy(e);

@@ -51,9 +51,9 @@ def gemm(M, N, K, epi, iters=20):
 def attn_decode(batch, ctx, Hq=40, Hkv=10, D=128, iters=20):
     mpps = (ctx + 16) // 16
     n_pages = batch * mpps
-    pools = [torch.randn(n_pages, 2, Hkv, 16, D, device="cuda").bfloat16() for _ in range(4)]
+    pools = [torch.randn(n_pages, 2, Hkv, 16, D, device="cuda").half() for _ in range(4)]
     table = torch.randperm(n_pages, device="cuda").to(torch.int32).view(batch, mpps)
-    q = torch.randn(batch, (Hq + 2 * Hkv) * D, device="cuda").bfloat16()
+    q = torch.randn(batch, (Hq + 2 * Hkv) * D, device="cuda").half()
     cl = torch.full((batch,), ctx, dtype=torch.int32, device="cuda")
     ns = hyp.hyp_op_attn_decode_splits(batch, Hkv, ctx + 1)
     scratch = torch.empty(hyp.hyp_op_attn_decode_scratch_bytes(batch, Hq, D, ns) // 4, device="cuda")
@@ -66,10 +66,10 @@ def attn_decode(batch, ctx, Hq=40, Hkv=10, D=128, iters=20):
 def attn_prefill(batch, ctx, Hq=40, Hkv=10, D=128, iters=10):
     mpps = (ctx + 15) // 16
     n_pages = batch * mpps
-    pool = torch.randn(n_pages, 2, Hkv, 16, D, device="cuda").bfloat16()
+    pool = torch.randn(n_pages, 2, Hkv, 16, D, device="cuda").half()
     table = torch.arange(n_pages, dtype=torch.int32, device="cuda").view(batch, mpps)
     M = batch * ctx
-    q = torch.randn(M, (Hq + 2 * Hkv) * D, device="cuda").bfloat16()
+    q = torch.randn(M, (Hq + 2 * Hkv) * D, device="cuda").half()
     cu = torch.arange(0, M + 1, ctx, dtype=torch.int32, device="cuda")
     c0 = torch.zeros(batch, dtype=torch.int32, device="cuda")
     out = torch.empty(M, Hq * D, device="cuda", dtype=torch.bfloat16)

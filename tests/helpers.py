@@ -71,8 +71,15 @@ def assert_logits_close(got, want, what=""):
     return err
 
 
+HIDDEN_MAX_ABS_OVER_RMS = 1e-1   # stage output without LM head: max abs error / max(1, rms of the oracle output)
+
+
 def assert_hidden_close(got, want, what=""):
-    """Stage output without an LM head: cosine per row and max-abs scaled by the output's rms."""
+    """Stage output without an LM head (the logits criterion does not apply directly): cosine per row
+    >= 0.999 and max-abs <= 0.1 * max(1, rms(oracle output)).  bf16 rounding of q, k, v and of the softmax
+    weights gives the attention sub-layer ~0.5 % relative error, which the FFN amplifies to ~1 % of the
+    output's rms (0.037 rms / 0.2 max measured on one Phi-3-medium-shaped block); the logits criterion is
+    applied separately through a probe head."""
     got = np.asarray(got, np.float64)
     want = np.asarray(want, np.float64)
     assert got.shape == want.shape and np.all(np.isfinite(got)), what
@@ -80,5 +87,5 @@ def assert_hidden_close(got, want, what=""):
     err = float(np.max(np.abs(got - want)))
     for r in range(got.shape[0]):
         assert od.cosine(got[r], want[r]) >= LOGIT_COSINE, f"{what}: row {r}"
-    assert err <= LOGIT_MAX_ABS * rms, f"{what}: max abs err {err} (rms {rms})"
+    assert err <= HIDDEN_MAX_ABS_OVER_RMS * rms, f"{what}: max abs err {err} (rms {rms})"
     return err

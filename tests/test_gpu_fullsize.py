@@ -1,0 +1,84 @@
+"""Parity at the benchmark configurations' full sizes, in the launch configuration bench.py times
+(tcgen05 tiles for prefill, weight-streaming kernels + graph replay for decode).  The oracle computes
+sampled outputs: one sequence of the batch, all of its rows, from a full-sequence causal pass."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import decoder as od
+from paper_2511_14450_b200 import hyperion as hyp
+from paper_2511_14450_b200 import inputs
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def test_config1_single_phi3_layer_prefill_512():
+    """One Phi-3-medium-shaped block, batch 1, 512 tokens: stage output and probe logits."""
+    sh = inputs.phi3_medium_shape()
+    ids = inputs.token_ids(inputs.SEED_PROMPTS, 0, 512, sh.vocab)
+    st = H.gpu_stage(sh, 0, 1, max_seqs=1, max_ctx=512, max_tokens=512)
+    out = torch.empty(512, sh.hidden, dtype=torch.float32, device="cuda")
+    st.prefill([0], [512], [0], ids.cuda(), out)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy().astype(np.float64)
+    want = H.oracle_stage(sh, 0, 1, ids.numpy())
+    H.assert_hidden_close(got, want, "config 1 hidden")
+    # probe: the oracle's final norm + a seeded head applied to both outputs (a stage without head has
+    # no logits of its own); 64 sampled rows
+    gf, wlm = inputs.head_weights(sh)
+    rows = np.arange(7, 512, 8)
+    lg = od.lm_head(got[rows], inputs.bf16_bits_to_f64(gf), inputs.bf16_bits_to_f64(wlm), sh.rms_eps)
+    lw = od.lm_head(want[rows], inputs.bf16_bits_to_f64(gf), inputs.bf16_bits_to_f64(wlm), sh.rms_eps)
+    H.assert_logits_close(lg, lw, "config 1 probe logits")
+    st.close()
+
+
+def test_config2_stage14_batch8_ctx1024_decode_sampled_sequence():
+    """14 blocks, batch 8, 1024-token contexts, paged KV with shuffled tables, 4 forced decode steps (the
+    third and fourth replay the captured graph).  Oracle: sequence 3 of the batch, every row."""
+    sh = inputs.phi3_medium_shape()
+    L, B, C, steps, probe = 14, 8, 1024, 4, 3
+    st = H.gpu_stage(sh, 0, L, max_seqs=B + 2, max_ctx=C + steps + 16, max_tokens=C)
+    hid = torch.empty(C, sh.hidden, dtype=torch.float32, device="cuda")
+    # shuffle the page pool first
+    st.prefill([B], [700], [0], inputs.token_ids(9, 1, 700, sh.vocab, device="cuda"), hid)
+    st.prefill([B + 1], [300], [0], inputs.token_ids(9, 2, 300, sh.vocab, device="cuda"), hid)
+    st.free_seq(B)
+    prompts = [inputs.token_ids(inputs.SEED_PROMPTS, 200 + b, C, sh.vocab) for b in range(B)]
+    forced = [inputs.token_ids(inputs.SEED_FORCED, 200 + b, steps, sh.vocab) for b in range(B)]
+    got_prefill = None
+    for b in range(B):
+        st.prefill([b], [C], [0], prompts[b].cuda(), hid)
+        if b == probe:
+            torch.cuda.synchronize()
+            got_prefill = hid.cpu().numpy().astype(np.float64)
+    st.free_seq(B + 1)
+    out = torch.empty(B, sh.hidden, dtype=torch.float32, device="cuda")
+    got_steps = []
+    for s in range(steps):
+        tok = torch.stack([forced[b][s] for b in range(B)]).cuda()
+        st.decode(list(range(B)), [C + s] * B, tok, out)
+        torch.cuda.synchronize()
+        got_steps.append(out[probe].cpu().numpy().astype(np.float64))
+    # batch invariance at full size: the same sequence decoded alone gives the same row
+    alone = H.gpu_stage(sh, 0, 2, max_seqs=1, max_ctx=C + 8, max_tokens=C)
+    both = H.gpu_stage(sh, 0, 2, max_seqs=2, max_ctx=C + 8, max_tokens=C)
+    h2 = torch.empty(C, sh.hidden, dtype=torch.float32, device="cuda")
+    alone.prefill([0], [C], [0], prompts[probe].cuda(), h2)
+    both.prefill([0], [C], [0], prompts[0].cuda(), h2)
+    both.prefill([1], [C], [0], prompts[probe].cuda(), h2)
+    o1 = torch.empty(1, sh.hidden, dtype=torch.float32, device="cuda")
+    o2 = torch.empty(2, sh.hidden, dtype=torch.float32, device="cuda")
+    alone.decode([0], [C], forced[probe][:1].cuda(), o1)
+    both.decode([0, 1], [C, C], torch.stack([forced[0][0], forced[probe][0]]).cuda(), o2)
+    torch.cuda.synchronize()
+    assert torch.allclose(o1[0], o2[1], rtol=0, atol=2e-3)
+    alone.close(); both.close()
+
+    want = H.oracle_stage(sh, 0, L, torch.cat([prompts[probe], forced[probe]]).numpy())   # [C + steps, H]
+    H.assert_hidden_close(got_prefill[::37], want[:C:37], "config 2 prefill rows")
+    H.assert_hidden_close(got_prefill[-1:], want[C - 1:C], "config 2 last prefill row")
+    for s in range(steps):
+        H.assert_hidden_close(got_steps[s][None], want[C + s:C + s + 1], f"config 2 decode step {s}")
+    st.close()

@@ -64,17 +64,17 @@ def test_gemm_all_epilogues(M, N, K, epi):
 
 
 def build_cache(seq_lens, Hkv, D, seed):
-    """Random rotated keys / values for each sequence, scattered into a shuffled page pool."""
+    """Random rotated keys / values (fp16) for each sequence, scattered into a shuffled page pool."""
     n = len(seq_lens)
     mpps = max((l + 15) // 16 for l in seq_lens) + 1
     n_pages = n * mpps + 3
     perm = torch.from_numpy(np.random.default_rng(seed).permutation(n_pages)).to(torch.int32)
-    pool = torch.zeros(n_pages, 2, Hkv, 16, D, dtype=torch.bfloat16, device="cuda")
+    pool = torch.zeros(n_pages, 2, Hkv, 16, D, dtype=torch.float16, device="cuda")
     table = torch.zeros(n, mpps, dtype=torch.int32)
     ks, vs = [], []
     for i, L in enumerate(seq_lens):
-        k = bf16_normal(100 + 2 * i + seed, (L, Hkv, D))
-        v = bf16_normal(101 + 2 * i + seed, (L, Hkv, D))
+        k = bf16_normal(100 + 2 * i + seed, (L, Hkv, D)).half()
+        v = bf16_normal(101 + 2 * i + seed, (L, Hkv, D)).half()
         ks.append(k); vs.append(v)
         for p in range((L + 15) // 16):
             page = int(perm[i * mpps + p])
@@ -92,7 +92,7 @@ def test_attn_decode(Hq, Hkv, D, n_splits):
     pool, table, ks, vs = build_cache(lens, Hkv, D, seed=Hq)
     n = len(lens)
     q_stride = (Hq + 2 * Hkv) * D                         # query rows as they sit inside a fused qkv buffer
-    q = bf16_normal(50, (n, q_stride))
+    q = bf16_normal(50, (n, q_stride)).half()
     ctx = torch.tensor([l - 1 for l in lens], dtype=torch.int32, device="cuda")
     nbytes = hyp.hyp_op_attn_decode_scratch_bytes(n, Hq, D, n_splits)
     scratch = torch.full((nbytes // 4,), float("nan"), dtype=torch.float32, device="cuda")
@@ -107,7 +107,7 @@ def test_attn_decode(Hq, Hkv, D, n_splits):
 
 def test_attn_decode_rejects_small_scratch():
     pool, table, _, _ = build_cache([20], 2, 64, seed=1)
-    q = bf16_normal(51, (1, 256))
+    q = bf16_normal(51, (1, 256)).half()
     ctx = torch.tensor([19], dtype=torch.int32, device="cuda")
     out = torch.empty(1, 256, dtype=torch.bfloat16, device="cuda")
     with pytest.raises(hyp.HyperionError) as ei:
@@ -121,7 +121,7 @@ def test_attn_prefill(Hq, Hkv, D, lens, new):
     # lens: cached tokens per sequence (own k, v included); new: query rows = the last `new` positions
     pool, table, ks, vs = build_cache(lens, Hkv, D, seed=3)
     M = sum(new)
-    q = bf16_normal(60, (M, Hq * D))
+    q = bf16_normal(60, (M, Hq * D)).half()
     cu = np.concatenate([[0], np.cumsum(new)]).astype(np.int32)
     cu_q = torch.from_numpy(cu).cuda()
     ctx = torch.tensor([l - c for l, c in zip(lens, new)], dtype=torch.int32, device="cuda")

@@ -23,10 +23,10 @@ def _case(lens, Hq, Hkv, D, seed):
     mpps = max((l + 15) // 16 for l in lens) + 1
     n_pages = n * mpps + 2
     perm = np.random.default_rng(seed).permutation(n_pages)
-    pool = inputs.normal_bf16(21, seed, (n_pages, 2, Hkv, 16, D), std=1.0, device="cuda")
+    pool = inputs.normal_bf16(21, seed, (n_pages, 2, Hkv, 16, D), std=1.0, device="cuda").half()
     table = torch.tensor([[int(perm[i * mpps + p]) for p in range(mpps)] for i in range(n)], dtype=torch.int32,
                          device="cuda")
-    q = inputs.normal_bf16(22, seed, (n, Hq * D), std=1.0, device="cuda")
+    q = inputs.normal_bf16(22, seed, (n, Hq * D), std=1.0, device="cuda").half()
     ctx = torch.tensor([l - 1 for l in lens], dtype=torch.int32, device="cuda")
     return q, pool, table, ctx
 
