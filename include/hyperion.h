@@ -24,6 +24,14 @@
  *    hyp_strerror are pure host functions, thread-safe, and never touch a GPU.
  *  - Activations crossing a stage boundary are fp32, row-major [M, hidden], rows packed in batch
  *    order (all rows of sequence 0, then sequence 1, ...).
+ *  - Precision.  The residual stream, all accumulation, softmax and norms are fp32.  The O, gate/up,
+ *    down and LM-head projections take bf16 inputs.  The q/k/v projection takes fp16 inputs and writes
+ *    fp32; q, k are rotated in fp32 and q, k, v rounded once to fp16; the KV cache and the softmax
+ *    weights are fp16 (values saturate at +-65504).  With bf16 there instead, the softmax weights alone
+ *    carry ~0.5 % error and per-step logits of the 5120-wide model miss the 5e-2 tolerance.
+ *  - Prefill rows: the residual projections split K across CTAs for row counts up to 2048 and add
+ *    partial sums with floating-point atomics, so the last bits of a prefill result may differ from
+ *    run to run; decode is bit-reproducible.
  */
 #ifndef HYPERION_H
 #define HYPERION_H
@@ -79,7 +87,9 @@ typedef struct {
 
 /* Weight tensor ids for hyp_stage_load.  Every matrix is bf16, row-major [out, in] (y = x W^T). */
 enum {
-  HYP_W_QKV = 0,     /* [(Hq + 2 Hkv) D, H]: rows = Q heads, then K heads, then V heads            */
+  HYP_W_QKV = 0,     /* [(Hq + 2 Hkv) D, H]: rows = Q heads, then K heads, then V heads.  The library   */
+                     /* keeps this one as fp16 (exact for |w| >= 2^-17, else off by < 3e-8), because   */
+                     /* q/k/v are projected from fp16 activations: see "Precision" below              */
   HYP_W_O = 1,       /* [H, Hq D]                                                                   */
   HYP_W_GATE_UP = 2, /* [2 F, H]: rows = gate (F) then up (F)                                       */
   HYP_W_DOWN = 3,    /* [H, F]                                                                      */

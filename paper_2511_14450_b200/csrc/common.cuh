@@ -140,9 +140,7 @@ enum Epilogue : int {
   EPI_STORE_BF16 = 0,  // out_bf16[m, n] = acc
   EPI_RESID_F32 = 1,   // out_f32[m, n] += acc         (residual stream)
   EPI_SWIGLU_BF16 = 2, // out_bf16[m, n] = silu(acc_gate) * acc_up, gate row n, up row n + N
-  EPI_STORE_F32 = 3,   // out_f32[m, n] = acc          (logits, q/k/v)
-  EPI_PAIR_F32 = 4     // weight-streaming kernel only: activation rows come as (high part, low part) pairs
-                       // stacked 8*NB/2 rows apart; out_f32[m, n] = acc[m] + acc[m + 8*NB/2]
+  EPI_STORE_F32 = 3    // out_f32[m, n] = acc          (logits, q/k/v)
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -150,9 +148,11 @@ enum Epilogue : int {
 // ---------------------------------------------------------------------------------------------
 int launch_embed(const int32_t* ids, const __nv_bfloat16* E, float* x, int M, int H, int V, cudaStream_t st);
 int launch_copy_f32(const float* src, float* dst, size_t n, cudaStream_t st);
-// h = bf16(norm(x)); if h_lo is given, also h_lo = bf16(norm(x) - h): the pair carries ~16 mantissa bits
-int launch_rmsnorm(const float* x, const __nv_bfloat16* g, __nv_bfloat16* h, __nv_bfloat16* h_lo, int M, int H,
-                   float eps, const int32_t* row_index /* optional gather of rows, may be null */, cudaStream_t st);
+// h = norm(x) as bf16, or as fp16 when out_f16 (h then points to __half storage)
+int launch_rmsnorm(const float* x, const __nv_bfloat16* g, void* h, bool out_f16, int M, int H, float eps,
+                   const int32_t* row_index /* optional gather of rows, may be null */, cudaStream_t st);
+// dst[i] = fp16(src[i]) (exact for |x| >= 2^-17, saturating at +-65504)
+int launch_bf16_to_f16(const __nv_bfloat16* src, __half* dst, size_t n, cudaStream_t st);
 // rotate q, k of every row (fp32 in), write q as fp16 [M, Hq*D] and append k, v as fp16 to the pages
 int launch_rope_kv_write(const float* qkv, __half* q16, __half* kv_layer, const float2* rope_table,
                          const BatchMeta& bm, const ModelDims& d, cudaStream_t st);

@@ -45,12 +45,11 @@ int launch_copy_f32(const float* src, float* dst, size_t n, cudaStream_t st) {
 }
 
 // h[r, :] = x[row, :] * rsqrt(mean(x[row, :]^2) + eps) * g, one CTA per output row.
-// row = row_index ? row_index[r] : r.  fp32 statistics, bf16 output.  With h_lo the rounding residue
-// bf16(y - bf16(y)) is stored too, so that a projection fed with both parts sees ~16 mantissa bits.
-template <int THREADS>
-__global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ g,
-                               __nv_bfloat16* __restrict__ h, __nv_bfloat16* __restrict__ h_lo, int H, float eps,
-                               const int32_t* __restrict__ row_index) {
+// row = row_index ? row_index[r] : r.  fp32 statistics; output bf16, or fp16 for the q/k/v projection
+// (whose inputs need fp16's 11 mantissa bits to keep the softmax weights inside the logit tolerance).
+template <int THREADS, bool F16>
+__global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ g, void* __restrict__ h,
+                               int H, float eps, const int32_t* __restrict__ row_index) {
   __shared__ float red[THREADS / 32];
   pdl_trigger();
   pdl_wait();
@@ -71,29 +70,38 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16*
   for (int w = 0; w < THREADS / 32; ++w) tot += red[w];
   const float rstd = rsqrtf(tot / (float)H + eps);
   const uint2* gr = reinterpret_cast<const uint2*>(g);
-  uint2* hr = reinterpret_cast<uint2*>(h + (size_t)r * H);
-  uint2* lr = h_lo ? reinterpret_cast<uint2*>(h_lo + (size_t)r * H) : nullptr;
+  uint2* hr = reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(h) + (size_t)r * H);
   for (int i = threadIdx.x; i < n4; i += THREADS) {
     const float4 v = xr[i];
     const uint2 gg = gr[i];
     const float y0 = v.x * rstd * bf16_lo(gg.x), y1 = v.y * rstd * bf16_hi(gg.x);
     const float y2 = v.z * rstd * bf16_lo(gg.y), y3 = v.w * rstd * bf16_hi(gg.y);
     uint2 o;
-    o.x = pack_bf16(y0, y1);
-    o.y = pack_bf16(y2, y3);
+    o.x = F16 ? pack_f16_sat(y0, y1) : pack_bf16(y0, y1);
+    o.y = F16 ? pack_f16_sat(y2, y3) : pack_bf16(y2, y3);
     hr[i] = o;
-    if (lr) {
-      uint2 l;
-      l.x = pack_bf16(y0 - bf16_lo(o.x), y1 - bf16_hi(o.x));
-      l.y = pack_bf16(y2 - bf16_lo(o.y), y3 - bf16_hi(o.y));
-      lr[i] = l;
-    }
   }
 }
 
-int launch_rmsnorm(const float* x, const __nv_bfloat16* g, __nv_bfloat16* h, __nv_bfloat16* h_lo, int M, int H,
-                   float eps, const int32_t* row_index, cudaStream_t st) {
-  HYP_CUDA_TRY(launch_pdl(rmsnorm_kernel<256>, dim3(M), dim3(256), 0, st, x, g, h, h_lo, H, eps, row_index));
+int launch_rmsnorm(const float* x, const __nv_bfloat16* g, void* h, bool out_f16, int M, int H, float eps,
+                   const int32_t* row_index, cudaStream_t st) {
+  if (out_f16)
+    HYP_CUDA_TRY(launch_pdl(rmsnorm_kernel<256, true>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
+  else
+    HYP_CUDA_TRY(launch_pdl(rmsnorm_kernel<256, false>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
+  return 1;
+}
+
+__global__ void bf16_to_f16_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n8) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x) {
+    const uint4 v = src[i];
+    dst[i] = make_uint4(pack_f16_sat(bf16_lo(v.x), bf16_hi(v.x)), pack_f16_sat(bf16_lo(v.y), bf16_hi(v.y)),
+                        pack_f16_sat(bf16_lo(v.z), bf16_hi(v.z)), pack_f16_sat(bf16_lo(v.w), bf16_hi(v.w)));
+  }
+}
+
+int launch_bf16_to_f16(const __nv_bfloat16* src, __half* dst, size_t n, cudaStream_t st) {
+  bf16_to_f16_kernel<<<148 * 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(dst), n / 8);
   return 1;
 }
 

@@ -35,7 +35,7 @@ __device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t& r0, uint32_t& r1,
 
 // TILES = 1: 16 output columns per CTA.  TILES = 2: 32 adjacent columns, or (SwiGLU) 16 gate rows and
 // the 16 matching up rows.  S = ring slots per warp.
-template <int NB, int EPI, int TILES>
+template <int NB, int EPI, int TILES, bool F16>
 __global__ void __launch_bounds__(GS_THREADS)
 gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_a, int N, int K,
                    int M, void* __restrict__ out, int ldo, int S, int* __restrict__ err) {
@@ -114,7 +114,12 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
           uint32_t a0, a1, a2, a3;
           ldsm4(sw + i * W_TILE_BYTES + sw_off((lane & 7) + (((lane >> 3) & 1) << 3), 2 * ks + (lane >> 4)), a0, a1, a2, a3);
 #pragma unroll
-          for (int j = 0; j < NB; ++j) mma_bf16_16816(acc[i][j], a0, a1, a2, a3, bf[j][2 * h], bf[j][2 * h + 1]);
+          for (int j = 0; j < NB; ++j) {
+            if (F16)
+              mma_f16_16816(acc[i][j], a0, a1, a2, a3, bf[j][2 * h], bf[j][2 * h + 1]);
+            else
+              mma_bf16_16816(acc[i][j], a0, a1, a2, a3, bf[j][2 * h], bf[j][2 * h + 1]);
+          }
         }
       }
     }
@@ -159,9 +164,7 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
     for (int ww = 0; ww < GS_WARPS; ++ww) {
       v += red[ww][r][m];
       if (SWIGLU) v2 += red[ww][16 + r][m];
-      if (EPI == EPI_PAIR_F32) v2 += red[ww][r][m + 4 * NB];  // the low parts sit 8*NB/2 token rows further on
     }
-    if (EPI == EPI_PAIR_F32) v += v2;
     const size_t o = (size_t)m * ldo + n;
     if (EPI == EPI_STORE_BF16) {
       reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(v);
@@ -175,7 +178,7 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   }
 }
 
-template <int NB, int EPI, int TILES>
+template <int NB, int EPI, int TILES, bool F16 = false>
 int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, int K, void* out, int ldo, cudaStream_t st) {
   static bool configured = false;
   static int num_sms = 0;
@@ -183,9 +186,9 @@ int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
   constexpr int MAX_DYN = GS_WARPS * GS_MAX_SLOTS * STAGE_BYTES + 1024 > 200 * 1024 ? 200 * 1024
                                                                                        : GS_WARPS * GS_MAX_SLOTS * STAGE_BYTES + 1024;
   if (!configured) {
-    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_stream_kernel<NB, EPI, TILES>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN));
+    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_stream_kernel<NB, EPI, TILES, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN));
     // several CTAs per SM share the ring space: ask for the largest shared-memory carve-out
-    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_stream_kernel<NB, EPI, TILES>, cudaFuncAttributePreferredSharedMemoryCarveout,
+    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_stream_kernel<NB, EPI, TILES, F16>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                       cudaSharedmemCarveoutMaxShared));
     int dev = 0;
     HYP_CUDA_TRY(cudaGetDevice(&dev));
@@ -208,7 +211,7 @@ int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
   if (slots < 2) slots = 2;
   while (slots > 1 && GS_WARPS * slots * STAGE_BYTES + 1024 > MAX_DYN) --slots;
   const int smem = GS_WARPS * slots * STAGE_BYTES + 1024;
-  HYP_CUDA_TRY(launch_pdl(gemm_stream_kernel<NB, EPI, TILES>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
+  HYP_CUDA_TRY(launch_pdl(gemm_stream_kernel<NB, EPI, TILES, F16>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
                           (TILES == 2 && !SWIGLU) ? w.map_small[1] : w.map_small[0], act.map_small[NB - 1], N, K, M, out,
                           ldo, slots, tc_err_flag_ptr()));
   return 1;
@@ -225,28 +228,22 @@ int launch_nb(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi,
       return wide ? launch_cfg<NB, EPI_RESID_F32, 2>(act, w, M, N, K, out, ldo, st)
                   : launch_cfg<NB, EPI_RESID_F32, 1>(act, w, M, N, K, out, ldo, st);
     case EPI_STORE_F32:
+      if (act.f16)
+        return wide ? launch_cfg<NB, EPI_STORE_F32, 2, true>(act, w, M, N, K, out, ldo, st)
+                    : launch_cfg<NB, EPI_STORE_F32, 1, true>(act, w, M, N, K, out, ldo, st);
       return wide ? launch_cfg<NB, EPI_STORE_F32, 2>(act, w, M, N, K, out, ldo, st)
                   : launch_cfg<NB, EPI_STORE_F32, 1>(act, w, M, N, K, out, ldo, st);
     case EPI_SWIGLU_BF16: return launch_cfg<NB, EPI_SWIGLU_BF16, 2>(act, w, M, N, K, out, ldo, st);
-    case EPI_PAIR_F32:
-      if (NB % 2) return HYP_EINVAL;
-      return wide ? launch_cfg<NB, EPI_PAIR_F32, 2>(act, w, M, N, K, out, ldo, st)
-                  : launch_cfg<NB, EPI_PAIR_F32, 1>(act, w, M, N, K, out, ldo, st);
     default: return HYP_EINVAL;
   }
 }
 
 }  // namespace
 
-// EPI_PAIR_F32: the activation matrix holds the high parts in rows [0, M) and the low parts in rows
-// [8 nb, 8 nb + M) with nb = ceil(M / 8); M <= 16.
 int launch_gemm_stream(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
                        cudaStream_t st) {
   if (M < 1 || M > 32 || N < 1 || K < 8 || act.K != K || w.K != K || !tc_err_flag_ptr()) return HYP_EINVAL;
-  if (epi == EPI_PAIR_F32) {
-    if (M > 16) return HYP_EINVAL;
-    return M <= 8 ? launch_nb<2>(act, w, M, N, K, epi, out, ldo, st) : launch_nb<4>(act, w, M, N, K, epi, out, ldo, st);
-  }
+  if (act.f16 != w.f16 || (act.f16 && epi != EPI_STORE_F32)) return HYP_EINVAL;  // fp16 operands: q/k/v only
   switch ((M + 7) / 8) {
     case 1: return launch_nb<1>(act, w, M, N, K, epi, out, ldo, st);
     case 2: return launch_nb<2>(act, w, M, N, K, epi, out, ldo, st);

@@ -62,8 +62,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   d |= (uint64_t)2 << 61;            // 128-byte swizzle
   return d;
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 256.
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// Instruction descriptor: (bf16 x bf16 | fp16 x fp16) -> fp32, both operands K-major, M = 128, N = 256.
+constexpr uint32_t IDESC_BF16 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+constexpr uint32_t IDESC_F16 = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
 // Walks the work of one CTA as a sequence of (tile, k-block range) segments.  All three roles of a CTA
 // run the same walk, so they agree on the order without communicating.
@@ -177,7 +178,7 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[16], const ui
 template <int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int M, int N, int K,
-               void* __restrict__ out, int ldo, int team, int* __restrict__ err) {
+               void* __restrict__ out, int ldo, int team, uint32_t idesc, int* __restrict__ err) {
   constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
   const bool STREAMK = EPI == EPI_RESID_F32 && team > 0;
   constexpr int BN_OUT = SWIGLU ? BN / 2 : BN;  // output columns per tile
@@ -267,7 +268,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
           const uint64_t da = smem_desc(sa), db = smem_desc(sb);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k)
-            tc_mma(d_tmem, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), IDESC,
+            tc_mma(d_tmem, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
                    (kb > kb0 || k > 0) ? 1u : 0u);
           tc_commit(empty_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -343,7 +344,7 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-int encode_map(CUtensorMap* map, const __nv_bfloat16* ptr, int rows, int K, int box_rows) {
+int encode_map(CUtensorMap* map, const void* ptr, int rows, int K, int box_rows, bool f16) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return HYP_ECUDA;
   if ((K % 8) != 0 || ((uintptr_t)ptr & 15) != 0) return HYP_EINVAL;
@@ -351,7 +352,7 @@ int encode_map(CUtensorMap* map, const __nv_bfloat16* ptr, int rows, int K, int 
   const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
   const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1u, 1u};
-  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)ptr, dims, strides, box, estr,
+  CUresult r = enc(map, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)ptr, dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
@@ -396,26 +397,26 @@ int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
     grid = (int)(tiles < num_sms ? tiles : num_sms);
   }
   HYP_CUDA_TRY(launch_pdl(gemm_tc_kernel<EPI>, dim3(grid), dim3(TC_THREADS), (size_t)SMEM_BYTES, st, act.map, w.map, M, N,
-                          K, out, ldo, team, g_err_flag));
+                          K, out, ldo, team, act.f16 ? IDESC_F16 : IDESC_BF16, g_err_flag));
   return 1;
 }
 
 }  // namespace
 
 // Weights: 128-row boxes for the tile kernel, 16- and 32-row boxes for the weight-streaming kernel.
-int tc_make_weight(TcWeight* w, const __nv_bfloat16* ptr, int rows, int K) {
-  w->ptr = ptr; w->rows = rows; w->K = K;
-  int rc = encode_map(&w->map, ptr, rows, K, 128);
+int tc_make_weight(TcWeight* w, const void* ptr, int rows, int K, bool f16) {
+  w->ptr = (const __nv_bfloat16*)ptr; w->rows = rows; w->K = K; w->f16 = f16;
+  int rc = encode_map(&w->map, ptr, rows, K, 128, f16);
   if (rc) return rc;
-  rc = encode_map(&w->map_small[0], ptr, rows, K, 16);
+  rc = encode_map(&w->map_small[0], ptr, rows, K, 16, f16);
   if (rc) return rc;
-  return encode_map(&w->map_small[1], ptr, rows, K, 32);
+  return encode_map(&w->map_small[1], ptr, rows, K, 32, f16);
 }
 // Activations: 128-row boxes for the tile kernel, 8/16/24/32-row boxes for the weight-streaming kernel.
-int tc_make_act(TcAct* a, const __nv_bfloat16* ptr, int rows, int K) {
-  a->ptr = ptr; a->rows = rows; a->K = K;
-  int rc = encode_map(&a->map, ptr, rows, K, 128);
-  for (int nb = 1; nb <= 4 && !rc; ++nb) rc = encode_map(&a->map_small[nb - 1], ptr, rows, K, 8 * nb);
+int tc_make_act(TcAct* a, const void* ptr, int rows, int K, bool f16) {
+  a->ptr = (const __nv_bfloat16*)ptr; a->rows = rows; a->K = K; a->f16 = f16;
+  int rc = encode_map(&a->map, ptr, rows, K, 128, f16);
+  for (int nb = 1; nb <= 4 && !rc; ++nb) rc = encode_map(&a->map_small[nb - 1], ptr, rows, K, 8 * nb, f16);
   return rc;
 }
 
@@ -439,6 +440,7 @@ int tc_error_flag(int* value_out) {
 int launch_gemm_tc(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
                    cudaStream_t st) {
   if (M < 1 || N < 1 || K < 8 || act.K != K || w.K != K || M > act.rows || !g_err_flag) return HYP_EINVAL;
+  if (act.f16 != w.f16) return HYP_EINVAL;  // one instruction takes both operands in the same 16-bit type
   switch (epi) {
     case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16>(act, w, M, N, K, out, ldo, st);
     case EPI_RESID_F32: return launch_epi<EPI_RESID_F32>(act, w, M, N, K, out, ldo, st);

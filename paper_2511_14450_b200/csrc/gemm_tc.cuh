@@ -6,18 +6,20 @@
 
 namespace hyp {
 
-// A bf16 matrix [rows, K] row-major together with the TMA descriptor that tiles it.
+// A 16-bit matrix [rows, K] row-major (bf16, or fp16 when f16) together with the TMA descriptors that tile
+// it.  Both operands of a projection must have the same type.
 struct TcOperand {
   CUtensorMap map;
   const __nv_bfloat16* ptr = nullptr;
   int rows = 0, K = 0;
+  bool f16 = false;
   CUtensorMap map_small[4];  // weight-streaming kernel: weights [0], [1] = 16-, 32-row boxes; activations [nb-1] = 8*nb rows
 };
 typedef TcOperand TcWeight;
 typedef TcOperand TcAct;
 
-int tc_make_weight(TcWeight* w, const __nv_bfloat16* ptr, int rows, int K);
-int tc_make_act(TcAct* a, const __nv_bfloat16* ptr, int rows, int K);
+int tc_make_weight(TcWeight* w, const void* ptr, int rows, int K, bool f16 = false);
+int tc_make_act(TcAct* a, const void* ptr, int rows, int K, bool f16 = false);
 
 // One-time set-up of the device-side error word (allocates; call from stage creation, not from the hot path).
 int tc_prepare();

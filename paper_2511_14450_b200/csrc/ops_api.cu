@@ -35,7 +35,7 @@ int finish(int rc) {
 
 extern "C" int hyp_op_rmsnorm(const float* x, const void* g, void* out, int32_t M, int32_t H, float eps, void* stream) {
   if (!x || !g || !out || M < 1 || H < 8 || H % 8 || !(eps > 0.f)) return HYP_EINVAL;
-  return finish(launch_rmsnorm(x, (const __nv_bfloat16*)g, (__nv_bfloat16*)out, nullptr, M, H, eps, nullptr,
+  return finish(launch_rmsnorm(x, (const __nv_bfloat16*)g, out, false, M, H, eps, nullptr,
                                (cudaStream_t)stream));
 }
 

@@ -52,8 +52,9 @@ struct hyp_stage {
   float* x = nullptr;
   float* qkv32 = nullptr;             // q | k | v straight from the projection's accumulators
   __half* q16 = nullptr;              // rotated queries
-  bf16 *h = nullptr, *h_lo = nullptr, *h_pair = nullptr, *attn = nullptr, *u = nullptr;
-  TcAct tc_h, tc_h_lo, tc_h_pair, tc_attn, tc_u;
+  bf16 *h = nullptr, *attn = nullptr, *u = nullptr;
+  __half* h16 = nullptr;              // normalised activations for the q/k/v projection
+  TcAct tc_h, tc_h16, tc_attn, tc_u;
   float* attn_scratch = nullptr;
   int max_splits = 32;
   float2* rope_table = nullptr;
@@ -260,22 +261,11 @@ int run_blocks(hyp_stage* s, const BatchMeta& bm, bool decode, int n_splits, cud
   for (int li = 0; li < s->L; ++li) {
     LayerW& lw = s->layers[li];
     __half* kv_layer = s->kv_pool + (size_t)li * s->kv_layer_elems;
-    // q, k, v are projected from the normalised activations split into a bf16 high and low part (the
-    // softmax is the one place where bf16's 8 mantissa bits on the inputs would not fit the tolerance)
-    if (M <= 16) {
-      // weight-streaming kernel: both parts ride along as extra token rows, the weights are read once
-      const int lo_row = 8 * ((M + 7) / 8);
-      HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g1, s->h_pair, s->h_pair + (size_t)lo_row * d.H, M, d.H, d.eps,
-                                              nullptr, st));
-      HYP_LAUNCH_T(HYP_K_GEMM_QKV, launch_gemm_stream(s->tc_h_pair, lw.tc_qkv, M, d.qkv_rows, d.H, EPI_PAIR_F32,
-                                                      s->qkv32, d.qkv_rows, st));
-    } else {
-      HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g1, s->h, s->h_lo, M, d.H, d.eps, nullptr, st));
-      HYP_LAUNCH_T(HYP_K_GEMM_QKV, project(s, s->tc_h, s->h, d.H, lw.tc_qkv, lw.wqkv, d.qkv_rows, d.H, M,
-                                           EPI_STORE_F32, s->qkv32, d.qkv_rows, st));
-      HYP_LAUNCH_T(HYP_K_GEMM_QKV, project(s, s->tc_h_lo, s->h_lo, d.H, lw.tc_qkv, lw.wqkv, d.qkv_rows, d.H, M,
-                                           EPI_RESID_F32, s->qkv32, d.qkv_rows, st));
-    }
+    // q, k, v: fp16 activations x fp16 weights -> fp32 (the softmax is the one place where bf16's 8
+    // mantissa bits on the inputs would not fit the logit tolerance)
+    HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g1, s->h16, true, M, d.H, d.eps, nullptr, st));
+    HYP_LAUNCH_T(HYP_K_GEMM_QKV, project(s, s->tc_h16, nullptr, d.H, lw.tc_qkv, nullptr, d.qkv_rows, d.H, M,
+                                         EPI_STORE_F32, s->qkv32, d.qkv_rows, st));
     HYP_LAUNCH_T(HYP_K_ROPE, launch_rope_kv_write(s->qkv32, s->q16, kv_layer, s->rope_table, bm, d, st));
     if (decode)
       HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_decode(s->q16, d.Hq * d.D, kv_layer, s->attn, s->attn_scratch, n_splits, bm,
@@ -284,7 +274,7 @@ int run_blocks(hyp_stage* s, const BatchMeta& bm, bool decode, int n_splits, cud
       HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_prefill(s->q16, d.Hq * d.D, kv_layer, s->attn, bm, d, st));
     HYP_LAUNCH_T(HYP_K_GEMM_O, project(s, s->tc_attn, s->attn, d.Hq * d.D, lw.tc_o, lw.wo, d.H, d.Hq * d.D, M,
                                        EPI_RESID_F32, s->x, d.H, st));
-    HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g2, s->h, nullptr, M, d.H, d.eps, nullptr, st));
+    HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g2, s->h, false, M, d.H, d.eps, nullptr, st));
     HYP_LAUNCH_T(HYP_K_GEMM_GATE_UP, project(s, s->tc_h, s->h, d.H, lw.tc_gu, lw.wgu, d.F, d.H, M, EPI_SWIGLU_BF16,
                                              s->u, d.F, st));
     HYP_LAUNCH_T(HYP_K_GEMM_DOWN, project(s, s->tc_u, s->u, d.F, lw.tc_d, lw.wd, d.H, d.F, M, EPI_RESID_F32, s->x,
@@ -307,7 +297,7 @@ int enqueue_stage(hyp_stage* s, const BatchMeta& bm, int n_seqs, bool decode, bo
   if (rc) return rc;
   if (s->last) {
     const int rows = all_rows ? M : n_seqs;
-    HYP_LAUNCH(launch_rmsnorm(s->x, s->gf, s->h, nullptr, rows, d.H, d.eps, all_rows ? nullptr : bm.last_row, st));
+    HYP_LAUNCH(launch_rmsnorm(s->x, s->gf, s->h, false, rows, d.H, d.eps, all_rows ? nullptr : bm.last_row, st));
     HYP_LAUNCH_T(HYP_K_LM_HEAD,
                  project(s, s->tc_h, s->h, d.H, s->tc_lm, s->wlm, d.V, d.H, rows, EPI_STORE_F32, out, d.V, st));
   } else {
@@ -476,7 +466,7 @@ extern "C" void hyp_stage_destroy(hyp_stage* s) {
     cudaFree(lw.wqkv); cudaFree(lw.wo); cudaFree(lw.wgu); cudaFree(lw.wd); cudaFree(lw.g1); cudaFree(lw.g2);
   }
   cudaFree(s->embed); cudaFree(s->gf); cudaFree(s->wlm); cudaFree(s->kv_pool);
-  cudaFree(s->x); cudaFree(s->h); cudaFree(s->h_lo); cudaFree(s->h_pair); cudaFree(s->qkv32); cudaFree(s->q16);
+  cudaFree(s->x); cudaFree(s->h); cudaFree(s->h16); cudaFree(s->qkv32); cudaFree(s->q16);
   cudaFree(s->attn); cudaFree(s->u);
   cudaFree(s->attn_scratch); cudaFree(s->rope_table); cudaFree(s->meta_dev);
   cudaFree(s->io_in); cudaFree(s->io_out);
@@ -551,22 +541,20 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
   const size_t rows_pad = ((size_t)s->max_rows + 127) / 128 * 128;
   TRY(dev_alloc(&s->x, rows_pad * d.H));
   TRY(dev_alloc(&s->h, rows_pad * d.H));
-  TRY(dev_alloc(&s->h_lo, rows_pad * d.H));
-  TRY(dev_alloc(&s->h_pair, (size_t)64 * d.H));
+  TRY(dev_alloc(&s->h16, rows_pad * d.H));
   TRY(dev_alloc(&s->qkv32, rows_pad * d.qkv_rows));
   TRY(dev_alloc(&s->q16, rows_pad * d.Hq * d.D));
   TRY(dev_alloc(&s->attn, rows_pad * d.Hq * d.D));
   TRY(dev_alloc(&s->u, rows_pad * d.F));
   TRY_CUDA(cudaMemset(s->h, 0, rows_pad * d.H * sizeof(bf16)));
-  TRY_CUDA(cudaMemset(s->h_lo, 0, rows_pad * d.H * sizeof(bf16)));
-  TRY_CUDA(cudaMemset(s->h_pair, 0, (size_t)64 * d.H * sizeof(bf16)));
+  TRY_CUDA(cudaMemset(s->h16, 0, rows_pad * d.H * sizeof(__half)));
   TRY_CUDA(cudaMemset(s->attn, 0, rows_pad * d.Hq * d.D * sizeof(bf16)));
   TRY_CUDA(cudaMemset(s->u, 0, rows_pad * d.F * sizeof(bf16)));
   const size_t scratch_bytes =
       attn_decode_scratch_bytes(std::min(c.max_seqs, HYP_MAX_DECODE_BATCH), d.Hq, d.D, s->max_splits);
   TRY(dev_alloc(&s->attn_scratch, scratch_bytes / sizeof(float)));
   s->workspace_bytes = rows_pad * ((size_t)d.H * 8 + (size_t)d.qkv_rows * 4 + ((size_t)2 * d.Hq * d.D + d.F) * 2) +
-                       (size_t)64 * d.H * 2 + scratch_bytes;
+                       scratch_bytes;
   // rotary table: cos/sin of pos * theta^(-2i/D), angles evaluated in double on the host
   {
     const int half = d.D / 2;
@@ -598,12 +586,11 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
   // tensor-core operand descriptors over the fixed workspace buffers
   TRY(tc_prepare());
   TRY(tc_make_act(&s->tc_h, s->h, (int)rows_pad, d.H));
-  TRY(tc_make_act(&s->tc_h_lo, s->h_lo, (int)rows_pad, d.H));
-  TRY(tc_make_act(&s->tc_h_pair, s->h_pair, 64, d.H));
+  TRY(tc_make_act(&s->tc_h16, s->h16, (int)rows_pad, d.H, true));
   TRY(tc_make_act(&s->tc_attn, s->attn, (int)rows_pad, d.Hq * d.D));
   TRY(tc_make_act(&s->tc_u, s->u, (int)rows_pad, d.F));
   for (LayerW& lw : s->layers) {
-    TRY(tc_make_weight(&lw.tc_qkv, lw.wqkv, d.qkv_rows, d.H));
+    TRY(tc_make_weight(&lw.tc_qkv, lw.wqkv, d.qkv_rows, d.H, true));  // held as fp16, see hyp_stage_load
     TRY(tc_make_weight(&lw.tc_o, lw.wo, d.H, d.Hq * d.D));
     TRY(tc_make_weight(&lw.tc_gu, lw.wgu, 2 * d.F, d.H));
     TRY(tc_make_weight(&lw.tc_d, lw.wd, d.H, d.F));
@@ -638,7 +625,19 @@ extern "C" int hyp_stage_load(hyp_stage* s, int32_t layer, int32_t tensor_id, co
     return HYP_EINVAL;
   }
   if (bytes != tensor_elems(s, tensor_id) * sizeof(bf16)) return HYP_EINVAL;
-  HYP_CUDA_TRY(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  if (tensor_id == HYP_W_QKV) {
+    // kept as fp16 so that the q/k/v projection can take fp16 activations (bf16 -> fp16 is exact for
+    // |w| >= 2^-17 and off by < 3e-8 below that)
+    if (((uintptr_t)src & 15) != 0) return HYP_EINVAL;
+    launch_bf16_to_f16((const bf16*)src, (__half*)dst, bytes / sizeof(bf16), (cudaStream_t)stream);
+    cudaError_t e = cudaPeekAtLastError();
+    if (e != cudaSuccess) {
+      set_last_cuda_error((int)e);
+      return HYP_ECUDA;
+    }
+  } else {
+    HYP_CUDA_TRY(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  }
   *mask |= 1u << tensor_id;
   return HYP_OK;
 }
