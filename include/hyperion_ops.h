@@ -40,7 +40,8 @@ typedef struct {
 HYP_API int hyp_op_rmsnorm(const float* x, const void* g, void* out, int32_t M, int32_t H, float eps, void* stream);
 
 /* Projection (the QKV, O, gate/up, down and LM-head contractions of the block):
- * acc[m, n] = sum_k a[m, k] * w[n, k], bf16 inputs, fp32 accumulation, then `epilogue`.
+ * acc[m, n] = sum_k a[m, k] * w[n, k], bf16 inputs, fp32 accumulation, then `epilogue`.  (The same kernels
+ * run inside hyp_stage_* with fp16 operands; this entry point exposes the bf16 instantiation.)
  * a bf16 [M, K] row-major, w bf16 [N (2N for SwiGLU), K] row-major, K multiple of 8, N multiple of 16
  * unless M <= 32.  M <= 32 runs the weight-streaming kernel, larger M the tcgen05 tile kernel.
  * The first call with M > 32 on a process allocates one device word for error reporting. */
@@ -59,7 +60,7 @@ HYP_API size_t hyp_op_attn_decode_scratch_bytes(int32_t n_seqs, int32_t n_q_head
  *   kv_pages   one block's page pool (layout above)
  *   block_table int32 [n_seqs, max_pages_per_seq];  ctx_lens int32 [n_seqs]
  *   scratch    fp32, at least hyp_op_attn_decode_scratch_bytes(...) bytes: per-split partial results
- *   out        bf16 [n_seqs, n_q_heads * D]
+ *   out        fp16 [n_seqs, n_q_heads * D]
  * n_splits in [1, 32]. */
 HYP_API int hyp_op_attn_decode(const hyp_attn_shape* shape, int32_t n_seqs, const void* q, int32_t q_stride,
                                const void* kv_pages, const int32_t* block_table, int32_t max_pages_per_seq,
@@ -99,7 +100,7 @@ HYP_API int hyp_op_attn_decode_static(const hyp_attn_shape* shape, int32_t n_seq
  * sees cached positions 0 .. its own (all of the sequence's k, v, new rows included, must already be in
  * the cache).
  *   q fp16 [M, q_stride]; cu_q int32 [n_seqs + 1] (cu_q[n_seqs] = M); ctx_lens int32 [n_seqs];
- *   block_table int32 [n_seqs, max_pages_per_seq]; out bf16 [M, n_q_heads * D]. */
+ *   block_table int32 [n_seqs, max_pages_per_seq]; out fp16 [M, n_q_heads * D]. */
 HYP_API int hyp_op_attn_prefill(const hyp_attn_shape* shape, int32_t n_seqs, int32_t M, const void* q,
                                 int32_t q_stride, const void* kv_pages, const int32_t* block_table,
                                 int32_t max_pages_per_seq, const int32_t* cu_q, const int32_t* ctx_lens, void* out,

@@ -9,7 +9,7 @@
 //   no cross-warp traffic inside the loop; the four warps are combined once at the end.  Tensor cores
 //   are used because the scalar version needs ~130 instructions per KB of cache and is issue-bound at
 //   HBM speed; the roofline of this kernel is HBM.
-//   merge kernel: grid (n_seqs * Hq).  Combines the split partials and writes bf16.
+//   merge kernel: grid (n_seqs * Hq).  Combines the split partials and writes fp16.
 //
 // Scratch layout (fp32): acc [n_seqs][Hq][n_splits][D], then ml [n_seqs][Hq][n_splits][2].
 #include "attn_common.cuh"
@@ -199,7 +199,7 @@ attn_decode_partial_kernel(const __half* __restrict__ qkv, const __half* __restr
 
 template <int D>
 __global__ void attn_decode_merge_kernel(const float* __restrict__ part_acc, const float* __restrict__ part_ml,
-                                         __nv_bfloat16* __restrict__ out, int n_splits, int Hq) {
+                                         __half* __restrict__ out, int n_splits, int Hq) {
   const int bh = blockIdx.x;  // b * Hq + hq
   const int dd = threadIdx.x;
   pdl_trigger();
@@ -213,11 +213,11 @@ __global__ void attn_decode_merge_kernel(const float* __restrict__ part_acc, con
     l += wgt * part_ml[slot * 2 + 1];
     a += wgt * part_acc[slot * D + dd];
   }
-  out[(size_t)bh * D + dd] = __float2bfloat16_rn(a / l);
+  out[(size_t)bh * D + dd] = __float2half_rn(fminf(fmaxf(a / l, -65504.f), 65504.f));
 }
 
 template <int D, int G>
-static int launch_dg(const __half* qkv, const __half* kv_layer, __nv_bfloat16* attn_out,
+static int launch_dg(const __half* qkv, const __half* kv_layer, __half* attn_out,
                      float* scratch, int n_splits, const BatchMeta& bm, const ModelDims& d, cudaStream_t st) {
   static bool configured = false;
   constexpr int smem = 4 * AD_TILE * D * 2;  // K[2] + V[2]; also covers the end-of-kernel combine buffers
@@ -235,7 +235,7 @@ static int launch_dg(const __half* qkv, const __half* kv_layer, __nv_bfloat16* a
   return 2;
 }
 
-int launch_attn_decode(const __half* qkv, int q_stride, const __half* kv_layer, __nv_bfloat16* attn_out,
+int launch_attn_decode(const __half* qkv, int q_stride, const __half* kv_layer, __half* attn_out,
                        float* scratch, int n_splits, const BatchMeta& bm, const ModelDims& d_in, cudaStream_t st) {
   ModelDims d = d_in;
   d.qkv_rows = q_stride;

@@ -67,7 +67,7 @@ extern "C" int hyp_op_attn_decode_static(const hyp_attn_shape* shape, int32_t n_
   d.page_tokens = 16;
   // Nothing in the array has to be cleared first: the partial kernel writes every (sequence, head,
   // split) slot - weighted sum, running maximum and denominator - before the merge kernel reads it.
-  rc = launch_attn_decode((const __half*)q, q_stride, (const __half*)kv_pages, (__nv_bfloat16*)out, scratch, n_splits,
+  rc = launch_attn_decode((const __half*)q, q_stride, (const __half*)kv_pages, (__half*)out, scratch, n_splits,
                           bm, d, (cudaStream_t)stream);
   if (rc < 0) return rc;
   cudaError_t e = cudaPeekAtLastError();

@@ -19,7 +19,7 @@ constexpr int FA_BQ = 64, FA_BKV = 64, FA_THREADS = 128, PT = 16;
 template <int D>
 __global__ void __launch_bounds__(FA_THREADS)
 attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict__ kv_layer,
-                       __nv_bfloat16* __restrict__ out, BatchMeta bm, ModelDims d) {
+                       __half* __restrict__ out, BatchMeta bm, ModelDims d) {
   constexpr int KS = D / 16;       // k-steps of the QK^T contraction
   constexpr int DN = D / 8;        // 8-wide output column tiles of O
   constexpr int CPR = D / 8;       // 16-byte chunks per K/V row
@@ -190,19 +190,19 @@ attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict_
   l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
   const float inv_lo = 1.f / l_lo, inv_hi = 1.f / l_hi;
   const int r_lo = 16 * warp + g, r_hi = r_lo + 8;
-  __nv_bfloat16* o_lo = out + (size_t)(row_base + r_lo) * d.Hq * D + (size_t)hq * D;
-  __nv_bfloat16* o_hi = out + (size_t)(row_base + r_hi) * d.Hq * D + (size_t)hq * D;
+  __half* o_lo = out + (size_t)(row_base + r_lo) * d.Hq * D + (size_t)hq * D;
+  __half* o_hi = out + (size_t)(row_base + r_hi) * d.Hq * D + (size_t)hq * D;
 #pragma unroll
   for (int dn = 0; dn < DN; ++dn) {
     if (r_lo < rows_here)
-      *reinterpret_cast<uint32_t*>(o_lo + 8 * dn + 2 * tq) = pack_bf16(o[dn][0] * inv_lo, o[dn][1] * inv_lo);
+      *reinterpret_cast<uint32_t*>(o_lo + 8 * dn + 2 * tq) = pack_f16_sat(o[dn][0] * inv_lo, o[dn][1] * inv_lo);
     if (r_hi < rows_here)
-      *reinterpret_cast<uint32_t*>(o_hi + 8 * dn + 2 * tq) = pack_bf16(o[dn][2] * inv_hi, o[dn][3] * inv_hi);
+      *reinterpret_cast<uint32_t*>(o_hi + 8 * dn + 2 * tq) = pack_f16_sat(o[dn][2] * inv_hi, o[dn][3] * inv_hi);
   }
 }
 
 template <int D>
-int launch_fa(const __half* qkv, const __half* kv_layer, __nv_bfloat16* attn_out, const BatchMeta& bm,
+int launch_fa(const __half* qkv, const __half* kv_layer, __half* attn_out, const BatchMeta& bm,
               const ModelDims& d, cudaStream_t st) {
   static bool configured = false;
   constexpr int smem = 4 * FA_BKV * D * 2;
@@ -220,7 +220,7 @@ int launch_fa(const __half* qkv, const __half* kv_layer, __nv_bfloat16* attn_out
 }  // namespace
 
 // Needs bm.cu_q, bm.ctx_lens, bm.block_table, bm.n_seqs, bm.n_tokens.  Head h of row t: q + t*q_stride + h*D.
-int launch_attn_prefill(const __half* q, int q_stride, const __half* kv_layer, __nv_bfloat16* attn_out,
+int launch_attn_prefill(const __half* q, int q_stride, const __half* kv_layer, __half* attn_out,
                         const BatchMeta& bm, const ModelDims& d_in, cudaStream_t st) {
   ModelDims d = d_in;
   d.qkv_rows = q_stride;

@@ -137,9 +137,9 @@ __host__ __device__ __forceinline__ size_t kv_page_elems(int Hkv, int page_token
 
 // epilogues of the projection kernels
 enum Epilogue : int {
-  EPI_STORE_BF16 = 0,  // out_bf16[m, n] = acc
+  EPI_STORE_BF16 = 0,  // out_16[m, n] = acc            (16-bit results take the operands' type: bf16 or fp16)
   EPI_RESID_F32 = 1,   // out_f32[m, n] += acc         (residual stream)
-  EPI_SWIGLU_BF16 = 2, // out_bf16[m, n] = silu(acc_gate) * acc_up, gate row n, up row n + N
+  EPI_SWIGLU_BF16 = 2, // out_16[m, n] = silu(acc_gate) * acc_up, gate row n, up row n + N
   EPI_STORE_F32 = 3    // out_f32[m, n] = acc          (logits, q/k/v)
 };
 
@@ -157,12 +157,12 @@ int launch_bf16_to_f16(const __nv_bfloat16* src, __half* dst, size_t n, cudaStre
 int launch_rope_kv_write(const float* qkv, __half* q16, __half* kv_layer, const float2* rope_table,
                          const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
 // q: fp16 [M, q_stride]
-int launch_attn_prefill(const __half* q, int q_stride, const __half* kv_layer, __nv_bfloat16* attn_out,
+int launch_attn_prefill(const __half* q, int q_stride, const __half* kv_layer, __half* attn_out,
                         const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
 // decode attention: one query row per sequence; `scratch` holds split partials
 size_t attn_decode_scratch_bytes(int max_seqs, int Hq, int D, int max_splits);
 int attn_decode_splits(int n_seqs, int Hkv, int max_ctx);
-int launch_attn_decode(const __half* q, int q_stride, const __half* kv_layer, __nv_bfloat16* attn_out,
+int launch_attn_decode(const __half* q, int q_stride, const __half* kv_layer, __half* attn_out,
                        float* scratch, int n_splits, const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
 
 }  // namespace hyp

@@ -166,19 +166,22 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       if (SWIGLU) v2 += red[ww][16 + r][m];
     }
     const size_t o = (size_t)m * ldo + n;
-    if (EPI == EPI_STORE_BF16) {
-      reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(v);
+    if (EPI == EPI_STORE_BF16 || EPI == EPI_SWIGLU_BF16) {
+      // 16-bit results take the operands' type
+      const float y = EPI == EPI_SWIGLU_BF16 ? v / (1.f + __expf(-v)) * v2 : v;
+      if (F16)
+        reinterpret_cast<__half*>(out)[o] = __float2half_rn(fminf(fmaxf(y, -65504.f), 65504.f));
+      else
+        reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(y);
     } else if (EPI == EPI_RESID_F32) {
       reinterpret_cast<float*>(out)[o] += v;
-    } else if (EPI == EPI_SWIGLU_BF16) {
-      reinterpret_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(v / (1.f + __expf(-v)) * v2);
     } else {
       reinterpret_cast<float*>(out)[o] = v;
     }
   }
 }
 
-template <int NB, int EPI, int TILES, bool F16 = false>
+template <int NB, int EPI, int TILES, bool F16>
 int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, int K, void* out, int ldo, cudaStream_t st) {
   static bool configured = false;
   static int num_sms = 0;
@@ -217,24 +220,31 @@ int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
   return 1;
 }
 
-template <int NB>
+template <int NB, bool F16>
 int launch_nb(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo, cudaStream_t st) {
   const bool wide = N > 8192;  // many rows: 32 columns per CTA keep the CTA count within one resident wave
   switch (epi) {
     case EPI_STORE_BF16:
-      return wide ? launch_cfg<NB, EPI_STORE_BF16, 2>(act, w, M, N, K, out, ldo, st)
-                  : launch_cfg<NB, EPI_STORE_BF16, 1>(act, w, M, N, K, out, ldo, st);
+      return wide ? launch_cfg<NB, EPI_STORE_BF16, 2, F16>(act, w, M, N, K, out, ldo, st)
+                  : launch_cfg<NB, EPI_STORE_BF16, 1, F16>(act, w, M, N, K, out, ldo, st);
     case EPI_RESID_F32:
-      return wide ? launch_cfg<NB, EPI_RESID_F32, 2>(act, w, M, N, K, out, ldo, st)
-                  : launch_cfg<NB, EPI_RESID_F32, 1>(act, w, M, N, K, out, ldo, st);
+      return wide ? launch_cfg<NB, EPI_RESID_F32, 2, F16>(act, w, M, N, K, out, ldo, st)
+                  : launch_cfg<NB, EPI_RESID_F32, 1, F16>(act, w, M, N, K, out, ldo, st);
     case EPI_STORE_F32:
-      if (act.f16)
-        return wide ? launch_cfg<NB, EPI_STORE_F32, 2, true>(act, w, M, N, K, out, ldo, st)
-                    : launch_cfg<NB, EPI_STORE_F32, 1, true>(act, w, M, N, K, out, ldo, st);
-      return wide ? launch_cfg<NB, EPI_STORE_F32, 2>(act, w, M, N, K, out, ldo, st)
-                  : launch_cfg<NB, EPI_STORE_F32, 1>(act, w, M, N, K, out, ldo, st);
-    case EPI_SWIGLU_BF16: return launch_cfg<NB, EPI_SWIGLU_BF16, 2>(act, w, M, N, K, out, ldo, st);
+      return wide ? launch_cfg<NB, EPI_STORE_F32, 2, F16>(act, w, M, N, K, out, ldo, st)
+                  : launch_cfg<NB, EPI_STORE_F32, 1, F16>(act, w, M, N, K, out, ldo, st);
+    case EPI_SWIGLU_BF16: return launch_cfg<NB, EPI_SWIGLU_BF16, 2, F16>(act, w, M, N, K, out, ldo, st);
     default: return HYP_EINVAL;
+  }
+}
+
+template <bool F16>
+int launch_type(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo, cudaStream_t st) {
+  switch ((M + 7) / 8) {
+    case 1: return launch_nb<1, F16>(act, w, M, N, K, epi, out, ldo, st);
+    case 2: return launch_nb<2, F16>(act, w, M, N, K, epi, out, ldo, st);
+    case 3: return launch_nb<3, F16>(act, w, M, N, K, epi, out, ldo, st);
+    default: return launch_nb<4, F16>(act, w, M, N, K, epi, out, ldo, st);
   }
 }
 
@@ -243,13 +253,9 @@ int launch_nb(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi,
 int launch_gemm_stream(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
                        cudaStream_t st) {
   if (M < 1 || M > 32 || N < 1 || K < 8 || act.K != K || w.K != K || !tc_err_flag_ptr()) return HYP_EINVAL;
-  if (act.f16 != w.f16 || (act.f16 && epi != EPI_STORE_F32)) return HYP_EINVAL;  // fp16 operands: q/k/v only
-  switch ((M + 7) / 8) {
-    case 1: return launch_nb<1>(act, w, M, N, K, epi, out, ldo, st);
-    case 2: return launch_nb<2>(act, w, M, N, K, epi, out, ldo, st);
-    case 3: return launch_nb<3>(act, w, M, N, K, epi, out, ldo, st);
-    default: return launch_nb<4>(act, w, M, N, K, epi, out, ldo, st);
-  }
+  if (act.f16 != w.f16) return HYP_EINVAL;  // one instruction takes both operands in the same 16-bit type
+  return act.f16 ? launch_type<true>(act, w, M, N, K, epi, out, ldo, st)
+                 : launch_type<false>(act, w, M, N, K, epi, out, ldo, st);
 }
 
 }  // namespace hyp

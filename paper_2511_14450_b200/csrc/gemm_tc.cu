@@ -120,7 +120,7 @@ __device__ __forceinline__ void red_add_f32x4(float* p, float a, float b, float 
 
 template <int EPI>
 __device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[16], const uint32_t (&v2)[16], void* out, int ldo,
-                                               int row, int col, int N, bool partial) {
+                                               int row, int col, int N, bool partial, bool f16) {
   const size_t o = (size_t)row * ldo + col;
   const bool full = col + 16 <= N;
   if (EPI == EPI_STORE_BF16 || EPI == EPI_SWIGLU_BF16) {
@@ -130,17 +130,18 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[16], const ui
       const float a = __uint_as_float(v[i]);
       f[i] = (EPI == EPI_SWIGLU_BF16) ? a / (1.f + __expf(-a)) * __uint_as_float(v2[i]) : a;
     }
-    __nv_bfloat16* p = reinterpret_cast<__nv_bfloat16*>(out) + o;
+    // 16-bit results take the operands' type (bf16 or fp16, both 2 bytes)
+    uint16_t* p = reinterpret_cast<uint16_t*>(out) + o;
+    uint32_t pk[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) pk[i] = f16 ? pack_f16_sat(f[2 * i], f[2 * i + 1]) : pack_bf16(f[2 * i], f[2 * i + 1]);
     if (full) {
-      uint4 w0 = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
-      uint4 w1 = make_uint4(pack_bf16(f[8], f[9]), pack_bf16(f[10], f[11]), pack_bf16(f[12], f[13]),
-                            pack_bf16(f[14], f[15]));
-      reinterpret_cast<uint4*>(p)[0] = w0;
-      reinterpret_cast<uint4*>(p)[1] = w1;
+      reinterpret_cast<uint4*>(p)[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      reinterpret_cast<uint4*>(p)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
     } else {
 #pragma unroll
       for (int i = 0; i < 16; ++i)
-        if (col + i < N) p[i] = __float2bfloat16_rn(f[i]);
+        if (col + i < N) p[i] = (uint16_t)((i & 1) ? (pk[i >> 1] >> 16) : (pk[i >> 1] & 0xffffu));
     }
   } else {
     float* p = reinterpret_cast<float*>(out) + o;
@@ -307,7 +308,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         tmem_ld16(t0 + c, v);
         if (SWIGLU) tmem_ld16(t0 + BN / 2 + c, v2);
         tmem_ld_wait();
-        if (row < M) epilogue_chunk<EPI>(v, v2, out, ldo, row, n0 + c, N, partial);
+        if (row < M) epilogue_chunk<EPI>(v, v2, out, ldo, row, n0 + c, N, partial, idesc == IDESC_F16);
       }
       tc_fence_before();
       mbar_arrive(tempty_bar(acc));

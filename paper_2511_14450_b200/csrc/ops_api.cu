@@ -83,7 +83,7 @@ extern "C" int hyp_op_attn_decode(const hyp_attn_shape* shape, int32_t n_seqs, c
   bm.ctx_lens = ctx_lens;
   bm.block_table = block_table;
   const ModelDims d = attn_dims(shape, q_stride);
-  return finish(launch_attn_decode((const __half*)q, q_stride, (const __half*)kv_pages, (__nv_bfloat16*)out, scratch,
+  return finish(launch_attn_decode((const __half*)q, q_stride, (const __half*)kv_pages, (__half*)out, scratch,
                                    n_splits, bm, d, (cudaStream_t)stream));
 }
 
@@ -102,6 +102,6 @@ extern "C" int hyp_op_attn_prefill(const hyp_attn_shape* shape, int32_t n_seqs, 
   bm.ctx_lens = ctx_lens;
   bm.block_table = block_table;
   const ModelDims d = attn_dims(shape, q_stride);
-  return finish(launch_attn_prefill((const __half*)q, q_stride, (const __half*)kv_pages, (__nv_bfloat16*)out, bm, d,
+  return finish(launch_attn_prefill((const __half*)q, q_stride, (const __half*)kv_pages, (__half*)out, bm, d,
                                     (cudaStream_t)stream));
 }

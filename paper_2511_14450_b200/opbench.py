@@ -57,7 +57,7 @@ def attn_decode(batch, ctx, Hq=40, Hkv=10, D=128, iters=20):
     cl = torch.full((batch,), ctx, dtype=torch.int32, device="cuda")
     ns = hyp.hyp_op_attn_decode_splits(batch, Hkv, ctx + 1)
     scratch = torch.empty(hyp.hyp_op_attn_decode_scratch_bytes(batch, Hq, D, ns) // 4, device="cuda")
-    out = torch.empty(batch, Hq * D, device="cuda", dtype=torch.bfloat16)
+    out = torch.empty(batch, Hq * D, device="cuda", dtype=torch.float16)
     ms = _time(lambda i: hyp.hyp_op_attn_decode((Hq, Hkv, D), q, pools[i % 4], table, cl, ns, scratch, out), iters)
     return {"op": "attn_decode", "batch": batch, "ctx": ctx, "splits": ns, "us": ms * 1e3,
             "kv_gbs": batch * (ctx + 1) * 2 * Hkv * D * 2 / ms / 1e6}
@@ -72,7 +72,7 @@ def attn_prefill(batch, ctx, Hq=40, Hkv=10, D=128, iters=10):
     q = torch.randn(M, (Hq + 2 * Hkv) * D, device="cuda").half()
     cu = torch.arange(0, M + 1, ctx, dtype=torch.int32, device="cuda")
     c0 = torch.zeros(batch, dtype=torch.int32, device="cuda")
-    out = torch.empty(M, Hq * D, device="cuda", dtype=torch.bfloat16)
+    out = torch.empty(M, Hq * D, device="cuda", dtype=torch.float16)
     ms = _time(lambda i: hyp.hyp_op_attn_prefill((Hq, Hkv, D), q, pool, table, cu, c0, out), iters, warmup=2)
     return {"op": "attn_prefill", "batch": batch, "ctx": ctx, "us": ms * 1e3,
             "tflops_causal": 4.0 * batch * (ctx * (ctx + 1) / 2) * Hq * D / ms / 1e9}

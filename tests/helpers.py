@@ -14,8 +14,15 @@ def oracle_shape(sh):
     return od.Shape(sh.hidden, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.ffn, sh.vocab, sh.rms_eps, sh.rope_theta)
 
 
+def _gen_device():
+    """Where the seeded generator runs.  Its integer hash + table lookup is bit-identical on CPU and CUDA
+    (pinned by test_generator_is_identical_on_cpu_and_cuda), so large tensors are generated on the GPU
+    when there is one and copied to the host for the oracle."""
+    return "cuda" if torch.cuda.is_available() else "cpu"
+
+
 def oracle_layer(sh, layer, random_gains=False):
-    w = inputs.layer_weights(sh, layer, device="cpu", random_gains=random_gains)
+    w = inputs.layer_weights(sh, layer, device=_gen_device(), random_gains=random_gains)
     return {k: inputs.bf16_bits_to_f64(v) for k, v in w.items()}
 
 
@@ -34,13 +41,13 @@ def oracle_stage(sh, lo, hi, x_or_ids, random_gains=False, logits=True):
     """Full-sequence pass of blocks [lo, hi) on one sequence.  ids (int) if lo == 0 else activations."""
     osh = oracle_shape(sh)
     if lo == 0:
-        E = inputs.bf16_bits_to_f64(inputs.embed_weights(sh))
+        E = inputs.bf16_bits_to_f64(inputs.embed_weights(sh, device=_gen_device()))
         x = od.embed(np.asarray(x_or_ids), E)
     else:
         x = np.asarray(x_or_ids, np.float64)
     x = od.stage_forward(x, OracleLayers(sh, lo, hi, random_gains), osh)
     if hi == sh.n_layers_total and logits:
-        gf, wlm = inputs.head_weights(sh, random_gains=random_gains)
+        gf, wlm = inputs.head_weights(sh, device=_gen_device(), random_gains=random_gains)
         return od.lm_head(x, inputs.bf16_bits_to_f64(gf), inputs.bf16_bits_to_f64(wlm), sh.rms_eps)
     return x
 

@@ -1,6 +1,8 @@
 """Parity at the benchmark configurations' full sizes, in the launch configuration bench.py times
 (tcgen05 tiles for prefill, weight-streaming kernels + graph replay for decode).  The oracle computes
 sampled outputs: one sequence of the batch, all of its rows, from a full-sequence causal pass."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -82,3 +84,41 @@ def test_config2_stage14_batch8_ctx1024_decode_sampled_sequence():
     for s in range(steps):
         H.assert_hidden_close(got_steps[s][None], want[C + s:C + s + 1], f"config 2 decode step {s}")
     st.close()
+
+
+def _full_model_case(prompt_len, steps, B=4, probe=1):
+    """40 blocks + LM head as ONE stage, batch B, equal prompts of `prompt_len`, `steps` forced decode steps;
+    per-step logits of sequence `probe` against the oracle's full-sequence pass."""
+    sh = inputs.phi3_medium_shape()
+    L = sh.n_layers_total
+    st = H.gpu_stage(sh, 0, L, max_seqs=B, max_ctx=prompt_len + steps + 16, max_tokens=B * prompt_len)
+    prompts = [inputs.token_ids(inputs.SEED_PROMPTS, 400 + b, prompt_len, sh.vocab) for b in range(B)]
+    forced = [inputs.token_ids(inputs.SEED_FORCED, 400 + b, steps, sh.vocab) for b in range(B)]
+    logits = torch.empty(B, sh.vocab, dtype=torch.float32, device="cuda")
+    st.prefill(list(range(B)), [prompt_len] * B, [0] * B, torch.cat(prompts).cuda(), logits)   # one call, B * prompt rows
+    torch.cuda.synchronize()
+    got = [logits[probe].cpu().numpy().astype(np.float64)]
+    for s in range(steps):
+        tok = torch.stack([forced[b][s] for b in range(B)]).cuda()
+        st.decode(list(range(B)), [prompt_len + s] * B, tok, logits)
+        torch.cuda.synchronize()
+        got.append(logits[probe].cpu().numpy().astype(np.float64))
+    st.close()
+    torch.cuda.empty_cache()
+    want = H.oracle_stage(sh, 0, L, torch.cat([prompts[probe], forced[probe]]).numpy())      # logits of every row
+    errs = []
+    for i, g in enumerate(got):
+        errs.append(H.assert_logits_close(g[None], want[prompt_len - 1 + i][None], f"full model, step {i - 1}"))
+    return max(errs)
+
+
+def test_config4_shape_40_blocks_with_head_prompt_512():
+    """The long-generation configuration's model (40 blocks + 32064-way head, batch 4) at a prompt the oracle
+    finishes in about two minutes; checks real per-step logits (no probe head involved)."""
+    _full_model_case(prompt_len=512, steps=4)
+
+
+@pytest.mark.skipif(os.environ.get("HYP_RUN_SLOW") != "1", reason="oracle needs ~10 min; set HYP_RUN_SLOW=1")
+def test_config4_full_size_prompt_2048():
+    """configs[4] at full size: batch 4, 2048-token prompts (8192 rows in one prefill call), first decode steps."""
+    _full_model_case(prompt_len=2048, steps=2)

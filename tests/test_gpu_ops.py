@@ -96,7 +96,7 @@ def test_attn_decode(Hq, Hkv, D, n_splits):
     ctx = torch.tensor([l - 1 for l in lens], dtype=torch.int32, device="cuda")
     nbytes = hyp.hyp_op_attn_decode_scratch_bytes(n, Hq, D, n_splits)
     scratch = torch.full((nbytes // 4,), float("nan"), dtype=torch.float32, device="cuda")
-    out = torch.empty(n, Hq * D, dtype=torch.bfloat16, device="cuda")
+    out = torch.empty(n, Hq * D, dtype=torch.float16, device="cuda")
     hyp.hyp_op_attn_decode((Hq, Hkv, D), q, pool, table, ctx, n_splits, scratch, out)
     torch.cuda.synchronize()
     for i, L in enumerate(lens):
@@ -109,7 +109,7 @@ def test_attn_decode_rejects_small_scratch():
     pool, table, _, _ = build_cache([20], 2, 64, seed=1)
     q = bf16_normal(51, (1, 256)).half()
     ctx = torch.tensor([19], dtype=torch.int32, device="cuda")
-    out = torch.empty(1, 256, dtype=torch.bfloat16, device="cuda")
+    out = torch.empty(1, 256, dtype=torch.float16, device="cuda")
     with pytest.raises(hyp.HyperionError) as ei:
         hyp.hyp_op_attn_decode((4, 2, 64), q, pool, table, ctx, 4, torch.empty(8, device="cuda"), out)
     assert ei.value.code == hyp.HYP_ECAPACITY
@@ -125,7 +125,7 @@ def test_attn_prefill(Hq, Hkv, D, lens, new):
     cu = np.concatenate([[0], np.cumsum(new)]).astype(np.int32)
     cu_q = torch.from_numpy(cu).cuda()
     ctx = torch.tensor([l - c for l, c in zip(lens, new)], dtype=torch.int32, device="cuda")
-    out = torch.full((M, Hq * D), 5.0, dtype=torch.bfloat16, device="cuda")
+    out = torch.full((M, Hq * D), 5.0, dtype=torch.float16, device="cuda")
     hyp.hyp_op_attn_prefill((Hq, Hkv, D), q, pool, table, cu_q, ctx, out)
     torch.cuda.synchronize()
     row = 0

@@ -37,7 +37,7 @@ def _both(lens, Hq, Hkv, D, n_splits, seed):
     nbytes = hyp.hyp_op_attn_decode_scratch_bytes(n, Hq, D, n_splits)
     assert nbytes <= hyp.HYP_STATIC_SCRATCH_BYTES
     scratch = torch.zeros(nbytes // 4, dtype=torch.float32, device="cuda")
-    want = torch.empty(n, Hq * D, dtype=torch.bfloat16, device="cuda")
+    want = torch.empty(n, Hq * D, dtype=torch.float16, device="cuda")
     got = torch.full_like(want, 9.0)
     hyp.hyp_op_attn_decode((Hq, Hkv, D), q, pool, table, ctx, n_splits, scratch, want)
     hyp.hyp_op_attn_decode_static((Hq, Hkv, D), q, pool, table, ctx, n_splits, got)
@@ -55,7 +55,7 @@ def test_static_scratch_matches_caller_scratch_on_two_calls_in_a_row():
 def test_static_scratch_rejects_batches_beyond_its_limit():
     q, pool, table, ctx = _case([20] * 32, 40, 10, 128, seed=3)
     assert hyp.hyp_op_attn_decode_scratch_bytes(32, 40, 128, 32) > hyp.HYP_STATIC_SCRATCH_BYTES
-    out = torch.zeros(32, 40 * 128, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(32, 40 * 128, dtype=torch.float16, device="cuda")
     with pytest.raises(hyp.HyperionError) as ei:
         hyp.hyp_op_attn_decode_static((40, 10, 128), q, pool, table, ctx, 32, out)
     assert ei.value.code == hyp.HYP_ECAPACITY
