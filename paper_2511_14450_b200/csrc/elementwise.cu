@@ -50,6 +50,7 @@ int launch_copy_f32(const float* src, float* dst, size_t n, cudaStream_t st) {
 template <int THREADS, bool F16>
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ g, void* __restrict__ h,
                                int H, float eps, const int32_t* __restrict__ row_index) {
+  constexpr int CACHE = 8;  // float4 per thread kept in registers: rows up to THREADS * 32 wide are read once
   __shared__ float red[THREADS / 32];
   pdl_trigger();
   pdl_wait();
@@ -57,8 +58,15 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16*
   const int row = row_index ? row_index[r] : r;
   const float4* xr = reinterpret_cast<const float4*>(x + (size_t)row * H);
   const int n4 = H / 4;
+  float4 keep[CACHE];
   float ss = 0.f;
-  for (int i = threadIdx.x; i < n4; i += THREADS) {
+#pragma unroll
+  for (int c = 0; c < CACHE; ++c) {
+    const int i = threadIdx.x + c * THREADS;
+    keep[c] = i < n4 ? xr[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+    ss += keep[c].x * keep[c].x + keep[c].y * keep[c].y + keep[c].z * keep[c].z + keep[c].w * keep[c].w;
+  }
+  for (int i = threadIdx.x + CACHE * THREADS; i < n4; i += THREADS) {
     const float4 v = xr[i];
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
@@ -71,8 +79,7 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16*
   const float rstd = rsqrtf(tot / (float)H + eps);
   const uint2* gr = reinterpret_cast<const uint2*>(g);
   uint2* hr = reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(h) + (size_t)r * H);
-  for (int i = threadIdx.x; i < n4; i += THREADS) {
-    const float4 v = xr[i];
+  auto emit = [&](int i, const float4& v) {
     const uint2 gg = gr[i];
     const float y0 = v.x * rstd * bf16_lo(gg.x), y1 = v.y * rstd * bf16_hi(gg.x);
     const float y2 = v.z * rstd * bf16_lo(gg.y), y3 = v.w * rstd * bf16_hi(gg.y);
@@ -80,7 +87,13 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16*
     o.x = F16 ? pack_f16_sat(y0, y1) : pack_bf16(y0, y1);
     o.y = F16 ? pack_f16_sat(y2, y3) : pack_bf16(y2, y3);
     hr[i] = o;
+  };
+#pragma unroll
+  for (int c = 0; c < CACHE; ++c) {
+    const int i = threadIdx.x + c * THREADS;
+    if (i < n4) emit(i, keep[c]);
   }
+  for (int i = threadIdx.x + CACHE * THREADS; i < n4; i += THREADS) emit(i, xr[i]);
 }
 
 int launch_rmsnorm(const float* x, const __nv_bfloat16* g, void* h, bool out_f16, int M, int H, float eps,

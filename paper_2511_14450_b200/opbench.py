@@ -48,14 +48,14 @@ def gemm(M, N, K, epi, iters=20):
             "tflops": 2.0 * M * rows * K / ms / 1e9, "weight_gbs": rows * K * 2 / ms / 1e6}
 
 
-def attn_decode(batch, ctx, Hq=40, Hkv=10, D=128, iters=20):
+def attn_decode(batch, ctx, Hq=40, Hkv=10, D=128, iters=20, splits=0):
     mpps = (ctx + 16) // 16
     n_pages = batch * mpps
     pools = [torch.randn(n_pages, 2, Hkv, 16, D, device="cuda").half() for _ in range(4)]
     table = torch.randperm(n_pages, device="cuda").to(torch.int32).view(batch, mpps)
     q = torch.randn(batch, (Hq + 2 * Hkv) * D, device="cuda").half()
     cl = torch.full((batch,), ctx, dtype=torch.int32, device="cuda")
-    ns = hyp.hyp_op_attn_decode_splits(batch, Hkv, ctx + 1)
+    ns = splits if splits > 0 else hyp.hyp_op_attn_decode_splits(batch, Hkv, ctx + 1)
     scratch = torch.empty(hyp.hyp_op_attn_decode_scratch_bytes(batch, Hq, D, ns) // 4, device="cuda")
     out = torch.empty(batch, Hq * D, device="cuda", dtype=torch.float16)
     ms = _time(lambda i: hyp.hyp_op_attn_decode((Hq, Hkv, D), q, pools[i % 4], table, cl, ns, scratch, out), iters)
@@ -97,11 +97,12 @@ def main():
     ap.add_argument("--batch", type=int, default=8)
     ap.add_argument("--ctx", type=int, default=1024)
     ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--splits", type=int, default=0, help="attn_decode: context splits (0 = the library's choice)")
     a = ap.parse_args()
     if a.op == "gemm":
         out = [gemm(a.M, a.N, a.K, a.epi, a.iters)]
     elif a.op == "attn_decode":
-        out = [attn_decode(a.batch, a.ctx, iters=a.iters)]
+        out = [attn_decode(a.batch, a.ctx, iters=a.iters, splits=a.splits)]
     elif a.op == "attn_prefill":
         out = [attn_prefill(a.batch, a.ctx, iters=a.iters)]
     else:
