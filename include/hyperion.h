@@ -141,7 +141,11 @@ HYP_API int hyp_stage_prefill(hyp_stage* s, const hyp_batch* batch, const void* 
 
 /* Decode: one new row per sequence (q_lens all 1, n_seqs <= HYP_MAX_DECODE_BATCH), attending to
  * the sequence's whole cache.  Same data flow as prefill with M = n_seqs; uses the
- * weight-streaming kernels.  in: ids [B] or activations [B, H]; out: [B, H] or logits [B, V]. */
+ * weight-streaming kernels.  in: ids [B] or activations [B, H]; out: [B, H] or logits [B, V].
+ * The kernel sequence of a step is captured into a CUDA graph the second time a (batch size,
+ * attention split count) pair is seen and replayed afterwards; `in` is copied into and `out` out of
+ * fixed library buffers around the replay, so the caller's pointers may change from call to call.
+ * While hyp_stage_kernel_timing is active the step is launched kernel by kernel instead. */
 HYP_API int hyp_stage_decode(hyp_stage* s, const hyp_batch* batch, const void* in, void* out, void* stream);
 
 /* Same two calls with HOST `in` / `out` buffers (pinned memory recommended): the library copies
