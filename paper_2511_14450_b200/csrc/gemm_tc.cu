@@ -329,6 +329,211 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Two-CTA variant (thread-block cluster of 2, tcgen05 cta_group::2): a CTA pair computes a 256 x 256 tile.
+// Each CTA loads its own 128 activation rows and HALF of the weight tile (128 of the 256 rows; for SwiGLU the
+// leader holds the gate rows, its peer the matching up rows), so a k-block costs 32 KB of shared-memory
+// fill per SM instead of 48 KB and the ring is 6 stages deep.  The leader's lane issues one MMA for both
+// CTAs; each CTA keeps its 128 x 256 half of the accumulator in its own tensor memory and runs its own
+// epilogue.  All copies of a stage (from both CTAs) complete on the leader's "full" barrier; the MMA commit
+// is multicast to both CTAs' "empty" / "accumulator ready" barriers; the peer's epilogue threads arrive
+// remotely on the leader's "accumulator free" barrier.  No multicast loads.  Used for the non-residual
+// epilogues (whole tiles per pair).
+// ---------------------------------------------------------------------------------------------------------
+constexpr int STAGES2 = 6;
+constexpr int STAGE2_BYTES = A_BYTES + B_BYTES / 2;  // per CTA: 16 KB of A + 16 KB of its half of B
+constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 + 256;
+constexpr uint32_t IDESC2_BF16 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+constexpr uint32_t IDESC2_F16 = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t mapa_rank(uint32_t addr, uint32_t rank) {  // same offset in CTA `rank`
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA tile load of a CTA pair: data lands in the executing CTA, completion bytes go to `bar` (a
+// shared::cluster address, here always the leader's barrier).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {  // arrive on `bar` (same offset) in both CTAs
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3)
+               : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+
+template <int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int M, int N, int K,
+                void* __restrict__ out, int ldo, uint32_t idesc, int* __restrict__ err) {
+  constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
+  constexpr int BN_OUT = SWIGLU ? BN / 2 : BN;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* aligned = smem_raw + (base - smem_u32(smem_raw));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(aligned + STAGES2 * STAGE2_BYTES);
+  // bars: full[STAGES2] | empty[STAGES2] | tmem_full[2] | tmem_empty[2] | tmem base (u32) | abort (int)
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES2 + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES2 + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES2 + 2 + a); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES2 + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();      // 0 = leader
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int pairs_m = (M + 2 * BM - 1) / (2 * BM), tiles_n = (N + BN_OUT - 1) / BN_OUT;
+  const int n_tiles = pairs_m * tiles_n;
+  const int KB = (K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES2; ++s) {
+      mbar_init(full_bar(s), 1);    // the leader's arrive.expect_tx; bytes come from both CTAs' copies
+      mbar_init(empty_bar(s), 1);   // the leader's MMA commit (multicast)
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);      // MMA commit (multicast)
+      mbar_init(tempty_bar(a), 256);   // 128 epilogue threads of each CTA (used in the leader only)
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::);
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();   // both CTAs' barriers exist before anybody signals across
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_trigger();
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---------------- TMA producer (both CTAs) ----------------
+      pdl_wait();
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+        const int m0 = (tile % pairs_m) * (2 * BM) + (int)rank * BM;
+        const int n0 = (tile / pairs_m) * BN_OUT;
+        const int rb = SWIGLU ? (int)rank * N + n0 : n0 + (int)rank * (BN / 2);  // this CTA's half of the weight tile
+        for (int kb = 0; kb < KB; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) { ok = false; break; }
+          const uint32_t sa = base + stage * STAGE2_BYTES, sb = sa + A_BYTES;
+          const uint32_t lead_full = mapa_rank(full_bar(stage), 0);
+          if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * STAGE2_BYTES);
+          tma_load_2d_pair(sa, &tm_a, kb * BK, m0, lead_full);
+          tma_load_2d_pair(sb, &tm_b, kb * BK, rb, lead_full);
+          if (++stage == STAGES2) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicCAS(err, 0, 6);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      // ---------------- MMA issuer (leader only) ----------------
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < KB; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = base + stage * STAGE2_BYTES, sb = sa + A_BYTES;
+          const uint64_t da = smem_desc(sa), db = smem_desc(sb);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            tc_mma_pair(d_tmem, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
+                        (kb > 0 || k > 0) ? 1u : 0u);
+          tc_commit_pair(empty_bar(stage));
+          if (++stage == STAGES2) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        tc_commit_pair(tfull_bar(acc));
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1;
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicCAS(err, 0, 7);
+      }
+    }
+  } else {
+    // ---------------- epilogue warps (both CTAs, each its own 128 rows) ----------------
+    const int q = warp & 3;
+    pdl_wait();
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+      const int m0 = (tile % pairs_m) * (2 * BM) + (int)rank * BM;
+      const int n0 = (tile / pairs_m) * BN_OUT;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int row = m0 + 32 * q + lane;
+      const uint32_t t0 = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * BN);
+#pragma unroll 2
+      for (int c = 0; c < BN_OUT; c += 16) {
+        if (n0 + c >= N) break;
+        uint32_t v[16], v2[16];
+        tmem_ld16(t0 + c, v);
+        if (SWIGLU) tmem_ld16(t0 + BN / 2 + c, v2);
+        tmem_ld_wait();
+        if (row < M) epilogue_chunk<EPI>(v, v2, out, ldo, row, n0 + c, N, false, idesc == IDESC2_F16);
+      }
+      tc_fence_before();
+      mbar_arrive_cluster(mapa_rank(tempty_bar(acc), 0));
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1;
+    }
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      atomicCAS(err, 0, 8);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();   // nobody leaves (or frees tensor memory) while its peer may still signal it
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+  }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -366,6 +571,23 @@ int encode_map(CUtensorMap* map, const void* ptr, int rows, int K, int box_rows,
 int* g_err_flag = nullptr;  // one device word per process: first non-zero code wins
 
 template <int EPI>
+int launch_pair(const TcAct& act, const TcWeight& w, int M, int N, int K, void* out, int ldo, cudaStream_t st,
+                int num_sms) {
+  static bool configured = false;
+  if (!configured) {
+    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_tc2_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
+    configured = true;
+  }
+  constexpr int BN_OUT = EPI == EPI_SWIGLU_BF16 ? BN / 2 : BN;
+  const long tiles = (long)((M + 2 * BM - 1) / (2 * BM)) * ((N + BN_OUT - 1) / BN_OUT);
+  long pairs = num_sms / 2;
+  if (tiles < pairs) pairs = tiles;
+  HYP_CUDA_TRY(launch_pdl(gemm_tc2_kernel<EPI>, dim3((unsigned)(2 * pairs)), dim3(TC_THREADS), (size_t)SMEM2_BYTES, st, act.map,
+                          w.map, M, N, K, out, ldo, act.f16 ? IDESC2_F16 : IDESC2_BF16, g_err_flag));
+  return 1;
+}
+
+template <int EPI>
 int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* out, int ldo, cudaStream_t st) {
   static bool configured = false;
   static int num_sms = 0;
@@ -378,6 +600,7 @@ int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
   }
   constexpr int BN_OUT = EPI == EPI_SWIGLU_BF16 ? BN / 2 : BN;
   const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN_OUT - 1) / BN_OUT;
+  if (EPI != EPI_RESID_F32 && tiles_m >= 2) return launch_pair<EPI>(act, w, M, N, K, out, ldo, st, num_sms);
   int grid, team = 0;  // team 0 = whole tiles per CTA
   if (EPI == EPI_RESID_F32 && tiles_m <= 16) {
     // stream-K (up to 2048 rows; beyond that whole tiles already balance and reuse A better): pick the team size (a divisor of tiles_m) that keeps most SMs busy, larger teams preferred
