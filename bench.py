@@ -296,7 +296,7 @@ def run_ours(args):
         line = {
             "metric": METRIC, "value": tokens / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic", "config": workload_config(K, W),
+            "dtype": "f16", "data": "synthetic", "config": workload_config(K, W),
             "e2e": {"value": e2e_tokens / (e2e_ms / 1e3), "unit": UNIT,
                     "h2d_bytes_per_step": BATCH * 4, "d2h_bytes_per_step": BATCH * sh.hidden * 4},
             "gpu_launches": int(launches),

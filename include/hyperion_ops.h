@@ -39,14 +39,37 @@ typedef struct {
  * x fp32 [M, H], g bf16 [H], out bf16 [M, H]; H multiple of 8. */
 HYP_API int hyp_op_rmsnorm(const float* x, const void* g, void* out, int32_t M, int32_t H, float eps, void* stream);
 
+/* Packed weight layout.  The projection kernels read a weight matrix w[n, k] (row n = output feature, [out, in]
+ * as in y = x W^T) from a tiled copy that the library makes once: tiles of 16 rows x 64 k (2 KB each), all
+ * k-blocks of a 16-row strip contiguous, each 128-byte tile row stored with its 16-byte chunks XOR-permuted by
+ * (row & 7) (the shared-memory swizzle of the tensor-core operands, applied at load time), zero padding to whole
+ * tiles.  Decode then streams every strip as one sequential run; prefill fetches 128-row operand tiles as eight
+ * 2 KB pieces.  hyp_op_weight_packed_bytes gives the size of that copy (0 on bad arguments); hyp_op_pack_weight
+ * writes it.
+ *   w       bf16 [N, K] row-major (swiglu != 0: [2N, K], N gate rows then N up rows), 16-byte aligned
+ *   packed  at least hyp_op_weight_packed_bytes(N, K, swiglu) bytes, 128-byte aligned; values stay bf16
+ * K multiple of 8.  Errors: HYP_EINVAL, HYP_ECAPACITY (packed_bytes too small). */
+HYP_API size_t hyp_op_weight_packed_bytes(int32_t N, int32_t K, int32_t swiglu);
+HYP_API int hyp_op_pack_weight(const void* w, int32_t N, int32_t K, int32_t swiglu, void* packed, size_t packed_bytes,
+                               void* stream);
+
 /* Projection (the QKV, O, gate/up, down and LM-head contractions of the block):
  * acc[m, n] = sum_k a[m, k] * w[n, k], bf16 inputs, fp32 accumulation, then `epilogue`.  (The same kernels
  * run inside hyp_stage_* with fp16 operands; this entry point exposes the bf16 instantiation.)
- * a bf16 [M, K] row-major, w bf16 [N (2N for SwiGLU), K] row-major, K multiple of 8, N multiple of 16
- * unless M <= 32.  M <= 32 runs the weight-streaming kernel, larger M the tcgen05 tile kernel.
- * The first call with M > 32 on a process allocates one device word for error reporting. */
-HYP_API int hyp_op_gemm(const void* a, const void* w, int32_t M, int32_t N, int32_t K, int32_t epilogue, void* out,
-                        int32_t ldo, void* stream);
+ * a bf16 [M, K] row-major; w_packed = the output of hyp_op_pack_weight for the same N, K and
+ * swiglu = (epilogue == HYP_EPI_SWIGLU_BF16); K multiple of 8, N multiple of 16 unless M <= 32.
+ * M <= 32 runs the weight-streaming kernel, larger M the tcgen05 tile kernel.
+ * The first call on a process allocates one device word for error reporting. */
+HYP_API int hyp_op_gemm(const void* a, const void* w_packed, int32_t M, int32_t N, int32_t K, int32_t epilogue,
+                        void* out, int32_t ldo, void* stream);
+
+/* Process-wide tuning switches (measurement aids; the defaults are the measured best).
+ *   HYP_TUNE_PDL           value != 0: launch the block's kernels with programmatic dependent launch, so a
+ *                          kernel's prologue and weight prefetch may overlap its predecessor's tail
+ *   HYP_TUNE_STREAM_SLOTS  ring slots per warp of the weight-streaming kernel, 1..8 (0 = built-in choice)
+ * Affects launches made after the call; decode graphs already captured keep their setting. */
+enum { HYP_TUNE_PDL = 0, HYP_TUNE_STREAM_SLOTS = 1 };
+HYP_API int hyp_tune(int32_t key, int32_t value);
 
 /* Number of context splits hyp_op_attn_decode would pick for this batch, and the scratch bytes
  * that n_splits needs.  Pure host helpers. */

@@ -49,6 +49,7 @@ attn_decode_partial_kernel(const __half* __restrict__ qkv, const __half* __restr
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, tq = lane & 3;
+  pdl_trigger();
   pdl_wait();  // the cache pages, the query row and the metadata all come from earlier kernels / copies
 
   const int ctx_total = bm.ctx_lens[b] + 1;  // the new token's k, v are already in the cache
@@ -155,7 +156,6 @@ attn_decode_partial_kernel(const __half* __restrict__ qkv, const __half* __restr
     __syncthreads();
   }
   cp_async_wait<0>();
-  pdl_trigger();
   __syncthreads();  // the staging buffers are reused below
 
   // combine the four warps: (m, l) per head, then rescaled O

@@ -74,24 +74,24 @@ __device__ __forceinline__ uint32_t pack_f16_sat(float a, float b) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// programmatic dependent launch: every kernel of the block sequence can be launched so that it may start
-// while its predecessor drains.  A kernel calls pdl_trigger() when its successor may be scheduled and
-// pdl_wait() before the first access to memory its predecessor writes or reads; everything before
-// pdl_wait() - barrier set-up, weight prefetch - then overlaps the predecessor's tail.  Without the
-// launch attribute both are no-ops.  Measured on B200 the overlap made the decode step slower (2.55 ms
-// against 2.14 ms for the 14-block stage: successors that become resident early add copies in flight
-// beyond the point where HBM throughput peaks), so the attribute is off by default.
+// programmatic dependent launch.  A kernel launched with the attribute may start while its predecessor still
+// runs; it calls pdl_wait() before the first access to memory the predecessor writes or reads, and everything
+// before that - barrier set-up, weight prefetch - overlaps the predecessor.  A kernel calls pdl_trigger() when its
+// successor may be scheduled.  Without the attribute both are no-ops.  Only the weight-streaming projections are
+// launched with it (launch_pdl<true>): their prefetch is worth overlapping, and a chain of early launches stays
+// one kernel deep.  Measured on B200 (14-block decode stage, batch 8): with the attribute on every kernel of the
+// block the step got slower (waiting CTAs of several future kernels pile up on the SMs).
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// Process-wide switch for the launch attribute (see above for why it defaults to off).
+// Process-wide switch for the launch attribute.
 inline bool& pdl_enabled() {
-  static bool on = false;
+  static bool on = true;
   return on;
 }
 
-template <typename... KArgs, typename... Args>
+template <bool OVERLAP = false, typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
                               Args&&... args) {
   cudaLaunchConfig_t cfg = {};
@@ -103,7 +103,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  cfg.numAttrs = (OVERLAP && pdl_enabled()) ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 

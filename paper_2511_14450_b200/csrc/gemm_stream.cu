@@ -1,92 +1,130 @@
 // Weight-streaming projection for M <= 32 rows (decode): out[m, n] (+)= sum_k a[m, k] * w[n, k].
 //
-// HBM-bound: every weight byte is read exactly once.  A CTA owns 16 (or 2 x 16) weight rows; its four
-// warps take the 64-wide k-blocks round-robin.  Each warp runs its own TMA ring: lane 0 keeps a run of
-// k-blocks (weight tile + the matching slice of the <= 32 activation rows, 128-byte swizzle) in flight
-// into the warp's shared-memory slots, the warp reads a landed slot back with ldmatrix, runs
-// mma.sync.m16n8k16 (weights are the 16-row operand, tokens the 8-wide operand) and lane 0 refills the
-// slot at once.  The bytes in flight are set by the ring depth, not by registers or occupancy, a slot
-// only ever has one waiter, and four lanes per CTA issue copies in parallel.  Batch 8-32 costs no more
-// issue slots than batch 1.  Each warp keeps a partial sum over its k-blocks; the warps meet in shared
-// memory and the epilogue (bf16 store, residual add, SiLU(gate) * up, fp32 store) is applied once.
-// Every mbarrier wait is bounded.
+// HBM-bound: every weight byte is read exactly once.  Weights are held packed (see gemm_tc.cuh): all k-blocks of
+// a 16-row strip are contiguous, so a CTA, which owns one strip (or two), reads it as a sequential run of 4 KB
+// bulk copies.  Its four warps take the copies round-robin.  Each warp runs its own ring: lane 0 keeps a run of
+// copies in flight into the warp's shared-memory slots, the warp reads a landed slot back, runs
+// mma.sync.m16n8k16 (weights are the 16-row operand, tokens the 8-wide operand) and lane 0 refills the slot at
+// once.  The ring holds weights only and is sized to fill the SM's shared memory when every CTA of the grid is
+// resident, so a CTA launched early (programmatic dependent launch) pulls a large part of its strip on chip while
+// its predecessor drains.  A slot only ever has one waiter, and four lanes per CTA issue copies in parallel.
+// Activations never touch shared memory: each lane reads the 16 bytes (8 consecutive k of one token) it needs
+// for a pair of MMAs straight from global memory (L2-resident, written by the predecessor), one copy ahead.  The
+// MMA's sixteen k slots are assigned to those k so that a lane's 16 bytes are exactly its fragment entries:
+// slots {2t, 2t+1, 2t+8, 2t+9} of the first MMA of a pair hold k = 8t .. 8t+3, the same slots of the second hold
+// 8t+4 .. 8t+7 (t = lane % 4); the weight fragments are read from shared memory with the same assignment (two
+// 128-bit loads per pair), which a dot product does not notice.  Batch 8-32 costs no more copy traffic than batch 1.
+// Each warp keeps a partial sum over its k-blocks; the warps meet in shared memory and the epilogue (16-bit store,
+// residual add, SiLU(gate) * up, fp32 store) is applied once.  Every mbarrier wait is bounded.
 #include "gemm_tc.cuh"
 #include "hyperion.h"
 #include "sm100_common.cuh"
 
 namespace hyp {
 
+int& gemm_stream_slots_override() {
+  static int v = 0;
+  return v;
+}
+
 namespace {
 
-constexpr int GS_BK = 64;
+constexpr int GS_CH = 2;  // k-blocks per weight copy: 4 KB contiguous per 16-row strip
 constexpr int GS_WARPS = 4;
 constexpr int GS_THREADS = 32 * GS_WARPS;
-constexpr int GS_MAX_SLOTS = 16;  // ring slots per warp
-constexpr int W_TILE_BYTES = 16 * GS_BK * 2;  // 16 rows x 64 k
-constexpr int A_TILE_BYTES = 8 * GS_BK * 2;   // 8 tokens x 64 k
+constexpr int GS_MAX_SLOTS = 8;  // ring slots per warp
+constexpr int W_TILE_BYTES = PK_TILE_BYTES;          // 16 rows x 64 k
+constexpr int W_CHUNK_BYTES = GS_CH * W_TILE_BYTES;  // one copy
+constexpr int GS_CHUNK_K = GS_CH * 64;               // k per copy
+constexpr int GS_GROUPS = GS_CHUNK_K / 32;           // 32-k groups (one MMA pair each) per copy
 
-__device__ __forceinline__ uint32_t sw_off(int r, int c) {  // 128-byte rows, 16-byte chunks XOR-swizzled by the row
-  return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
 }
-__device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+// activations are written by the predecessor grid and only read here: the non-coherent path may cache them in L1
+__device__ __forceinline__ uint4 ldg_act(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+  return r;
 }
 
-// TILES = 1: 16 output columns per CTA.  TILES = 2: 32 adjacent columns, or (SwiGLU) 16 gate rows and
-// the 16 matching up rows.  S = ring slots per warp.
+// TILES = 1: 16 output columns per CTA (one strip).  TILES = 2: 32 adjacent columns (strips 2b, 2b + 1), or (SwiGLU)
+// gate strip b and the matching up strip tile1_off + b.  S = ring slots per warp; a slot holds TILES copies.
 template <int NB, int EPI, int TILES, bool F16>
 __global__ void __launch_bounds__(GS_THREADS)
-gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_a, int N, int K,
-                   int M, void* __restrict__ out, int ldo, int S, int* __restrict__ err) {
+gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ act, int lda, int K, int N, int KBp,
+                   int tile1_off, int M, void* __restrict__ out, int ldo, int S, int* __restrict__ err) {
   constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
-  static_assert(!SWIGLU || TILES == 2, "SwiGLU pairs a gate tile with an up tile");
+  static_assert(!SWIGLU || TILES == 2, "SwiGLU pairs a gate strip with an up strip");
   constexpr int OUT_COLS = (TILES == 2 && !SWIGLU) ? 32 : 16;
-  constexpr int STAGE_BYTES = TILES * W_TILE_BYTES + NB * A_TILE_BYTES;
+  constexpr int STAGE_BYTES = TILES * W_CHUNK_BYTES;
+  constexpr int RED_LD = NB * 8 + 1;
+  static_assert(16 * TILES * RED_LD * 4 <= 2 * STAGE_BYTES, "a warp's partial sums reuse its own ring space");
   extern __shared__ uint8_t gs_smem_raw[];
-  __shared__ float red[GS_WARPS][16 * TILES][NB * 8 + 1];
   __shared__ uint64_t bars[GS_WARPS * GS_MAX_SLOTS];
-  const uint32_t base = (smem_u32(gs_smem_raw) + 1023u) & ~1023u;
+  const uint32_t base = (smem_u32(gs_smem_raw) + 127u) & ~127u;
+  uint8_t* base_ptr = gs_smem_raw + (base - smem_u32(gs_smem_raw));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
   const int n0 = blockIdx.x * OUT_COLS;
-  const int KB = (K + GS_BK - 1) / GS_BK;
+  const int NCH = KBp / GS_CH;  // copies per strip
   const uint32_t my_bars = smem_u32(bars) + 8u * (warp * GS_MAX_SLOTS);
   const uint32_t my_ring = base + (uint32_t)(warp * S) * STAGE_BYTES;
-  const int row1 = N + n0;  // SwiGLU: the up rows that pair with this CTA's gate rows
+  const int strip0 = SWIGLU ? (int)blockIdx.x : (int)blockIdx.x * TILES;
+  const int strip1 = SWIGLU ? tile1_off + (int)blockIdx.x : strip0 + 1;
+  const uint8_t* w0 = wp + (size_t)strip0 * KBp * W_TILE_BYTES;
+  const uint8_t* w1 = wp + (size_t)strip1 * KBp * W_TILE_BYTES;
 
-  // one k-block into one of this warp's slots (lane 0 only).  CTAs walk K from staggered starting points
-  // (a fixed rotation per CTA, so the summation order stays reproducible): otherwise every resident CTA
-  // would ask for the same activation slice and the same column offsets of its rows at the same moment.
-  const int rot = (int)((blockIdx.x * 13u) % (unsigned)KB);
+  // CTAs walk K from staggered starting points (a fixed rotation per CTA, so the summation order stays
+  // reproducible): otherwise every resident CTA would ask for the same activation lines at the same moment.
+  const int rot = (int)((blockIdx.x * 13u) % (unsigned)NCH);
+  auto actual = [&](int ch_logical) {
+    const int ch = ch_logical + rot;
+    return ch >= NCH ? ch - NCH : ch;
+  };
   // weights: never written by any kernel, may be fetched before the predecessor has finished
-  auto issue_w = [&](int kb_logical, int slot) {
-    int kb = kb_logical + rot;
-    if (kb >= KB) kb -= KB;
+  auto issue_w = [&](int ch_logical, int slot) {
+    const int ch = actual(ch_logical);
     const uint32_t dst = my_ring + slot * STAGE_BYTES, bar = my_bars + 8u * slot;
     mbar_expect_tx(bar, STAGE_BYTES);
-    tma_load_2d(dst, &tm_w, kb * GS_BK, n0, bar);  // 16 rows, or one 32-row box
-    if (SWIGLU) tma_load_2d(dst + W_TILE_BYTES, &tm_w, kb * GS_BK, row1, bar);
-  };
-  // activations: produced by the predecessor
-  auto issue_a = [&](int kb_logical, int slot) {
-    int kb = kb_logical + rot;
-    if (kb >= KB) kb -= KB;
-    tma_load_2d(my_ring + slot * STAGE_BYTES + TILES * W_TILE_BYTES, &tm_a, kb * GS_BK, 0, my_bars + 8u * slot);
+    bulk_load(dst, w0 + (size_t)ch * W_CHUNK_BYTES, W_CHUNK_BYTES, bar);
+    if (TILES == 2) bulk_load(dst + W_CHUNK_BYTES, w1 + (size_t)ch * W_CHUNK_BYTES, W_CHUNK_BYTES, bar);
   };
 
+  // Every CTA of this grid is resident by the time the last one gets here, so the successor may be scheduled
+  // into whatever room is left: it only sets up and prefetches until this grid has completed.
+  pdl_trigger();
   if (lane == 0) {
     for (int sl = 0; sl < S; ++sl) mbar_init(my_bars + 8u * sl, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     for (int sl = 0; sl < S; ++sl)
-      if (warp + GS_WARPS * sl < KB) issue_w(warp + GS_WARPS * sl, sl);
-  }
-  pdl_wait();
-  if (lane == 0) {
-    for (int sl = 0; sl < S; ++sl)
-      if (warp + GS_WARPS * sl < KB) issue_a(warp + GS_WARPS * sl, sl);
+      if (warp + GS_WARPS * sl < NCH) issue_w(warp + GS_WARPS * sl, sl);
   }
   __syncwarp();
+
+  // this lane's activation rows: token 8j + g of group j; rows >= M and k >= K read as zero
+  const uint16_t* arow[NB];
+  bool avalid[NB];
+#pragma unroll
+  for (int j = 0; j < NB; ++j) {
+    avalid[j] = 8 * j + g < M;
+    arow[j] = act + (size_t)(avalid[j] ? 8 * j + g : 0) * lda + 8 * t;
+  }
+  uint4 bq[GS_GROUPS][NB];  // fragment entries of the copy being worked on, refilled group by group for the next one
+  auto load_act = [&](int ch_logical, int q, uint4 (&dst)[NB]) {
+    const int k = actual(ch_logical) * GS_CHUNK_K + q * 32;
+#pragma unroll
+    for (int j = 0; j < NB; ++j)
+      dst[j] = (avalid[j] && k + 8 * t < K) ? ldg_act(arow[j] + k) : make_uint4(0u, 0u, 0u, 0u);
+  };
+  pdl_wait();  // activations (and, for the residual epilogue, the output) belong to the predecessor until here
+  if (warp < NCH) {
+#pragma unroll
+    for (int q = 0; q < GS_GROUPS; ++q) load_act(warp, q, bq[q]);
+  }
 
   float acc[TILES][NB][4];
 #pragma unroll
@@ -97,60 +135,59 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   bool ok = true;
   int slot = 0;
   uint32_t phase = 0;
-  for (int kb = warp; kb < KB; kb += GS_WARPS) {
+  // shared-memory offset of this lane's 16 bytes in tile row g, first 32-k group (the tile is stored swizzled:
+  // 16-byte chunk c of row r sits at chunk position c ^ (r & 7); rows g and g + 8 share g & 7)
+  for (int ch = warp; ch < NCH; ch += GS_WARPS) {
     if (!mbar_wait(my_bars + 8u * slot, phase, nullptr)) { ok = false; break; }
-    const uint32_t sw = my_ring + slot * STAGE_BYTES, sa = sw + TILES * W_TILE_BYTES;
+    const uint32_t sbase = my_ring + slot * STAGE_BYTES;
+    const bool more = ch + GS_WARPS < NCH;
 #pragma unroll
-    for (int kp = 0; kp < 2; ++kp) {  // pairs of 16-wide k steps
-      uint32_t bf[NB][4];              // [n tile]: b0, b1 of step 2kp, then of step 2kp + 1
-#pragma unroll
-      for (int j = 0; j < NB; ++j)
-        ldsm4(sa + sw_off(8 * j + (lane & 7), 4 * kp + (lane >> 3)), bf[j][0], bf[j][1], bf[j][2], bf[j][3]);
+    for (int q = 0; q < GS_GROUPS; ++q) {
+      const uint32_t off = (uint32_t)((q >> 1) * W_TILE_BYTES + g * 128 + (((4 * (q & 1) + t) ^ g) << 4));
 #pragma unroll
       for (int i = 0; i < TILES; ++i) {
+        const uint4 lo = lds128(sbase + i * W_CHUNK_BYTES + off);          // row g:     k 8t .. 8t+7 of the group
+        const uint4 hi = lds128(sbase + i * W_CHUNK_BYTES + off + 1024u);  // row g + 8
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const int ks = 2 * kp + h;
-          uint32_t a0, a1, a2, a3;
-          ldsm4(sw + i * W_TILE_BYTES + sw_off((lane & 7) + (((lane >> 3) & 1) << 3), 2 * ks + (lane >> 4)), a0, a1, a2, a3);
-#pragma unroll
-          for (int j = 0; j < NB; ++j) {
-            if (F16)
-              mma_f16_16816(acc[i][j], a0, a1, a2, a3, bf[j][2 * h], bf[j][2 * h + 1]);
-            else
-              mma_bf16_16816(acc[i][j], a0, a1, a2, a3, bf[j][2 * h], bf[j][2 * h + 1]);
+        for (int j = 0; j < NB; ++j) {
+          if (F16) {
+            mma_f16_16816(acc[i][j], lo.x, hi.x, lo.y, hi.y, bq[q][j].x, bq[q][j].y);
+            mma_f16_16816(acc[i][j], lo.z, hi.z, lo.w, hi.w, bq[q][j].z, bq[q][j].w);
+          } else {
+            mma_bf16_16816(acc[i][j], lo.x, hi.x, lo.y, hi.y, bq[q][j].x, bq[q][j].y);
+            mma_bf16_16816(acc[i][j], lo.z, hi.z, lo.w, hi.w, bq[q][j].z, bq[q][j].w);
           }
         }
       }
+      if (more) load_act(ch + GS_WARPS, q, bq[q]);  // the same group of this warp's next copy
     }
-    // Every ldmatrix result above has been consumed by an MMA that is already issued, so after this
+    // Every shared-memory read above has been consumed by an MMA that is already issued, so after this
     // warp barrier no lane still reads the slot and lane 0 may hand it back to the copy engine.
     __syncwarp();
     if (lane == 0) {
-      const int next = kb + GS_WARPS * S;
-      if (next < KB) {
-        issue_w(next, slot);
-        issue_a(next, slot);
-      }
+      const int next = ch + GS_WARPS * S;
+      if (next < NCH) issue_w(next, slot);
     }
     if (++slot == S) { slot = 0; phase ^= 1u; }
   }
-  pdl_trigger();  // this warp has no more copies to issue: the successor may begin its own prefetch
   if (!ok) {
     // a copy never landed: record it and let whatever is still in flight arrive (bounded) before leaving
     if (lane == 0) atomicCAS(err, 0, 4);
     for (int sl = 0; sl < S; ++sl) mbar_wait(my_bars + 8u * sl, 0, nullptr), mbar_wait(my_bars + 8u * sl, 1, nullptr);
   }
+  // partial sums of this warp go to the start of its own ring space (nothing is in flight into it any more)
+  float* red = reinterpret_cast<float*>(base_ptr);
+  const int red_warp = S * STAGE_BYTES / 4;  // floats between two warps' areas
   {
-    const int g = lane >> 2, t = lane & 3;
+    float* mine = red + warp * red_warp;
 #pragma unroll
     for (int i = 0; i < TILES; ++i)
 #pragma unroll
       for (int j = 0; j < NB; ++j) {
-        red[warp][16 * i + g][8 * j + 2 * t] = acc[i][j][0];
-        red[warp][16 * i + g][8 * j + 2 * t + 1] = acc[i][j][1];
-        red[warp][16 * i + g + 8][8 * j + 2 * t] = acc[i][j][2];
-        red[warp][16 * i + g + 8][8 * j + 2 * t + 1] = acc[i][j][3];
+        mine[(16 * i + g) * RED_LD + 8 * j + 2 * t] = acc[i][j][0];
+        mine[(16 * i + g) * RED_LD + 8 * j + 2 * t + 1] = acc[i][j][1];
+        mine[(16 * i + g + 8) * RED_LD + 8 * j + 2 * t] = acc[i][j][2];
+        mine[(16 * i + g + 8) * RED_LD + 8 * j + 2 * t + 1] = acc[i][j][3];
       }
   }
   __syncthreads();
@@ -162,8 +199,8 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
     float v = 0.f, v2 = 0.f;
 #pragma unroll
     for (int ww = 0; ww < GS_WARPS; ++ww) {
-      v += red[ww][r][m];
-      if (SWIGLU) v2 += red[ww][16 + r][m];
+      v += red[ww * red_warp + r * RED_LD + m];
+      if (SWIGLU) v2 += red[ww * red_warp + (16 + r) * RED_LD + m];
     }
     const size_t o = (size_t)m * ldo + n;
     if (EPI == EPI_STORE_BF16 || EPI == EPI_SWIGLU_BF16) {
@@ -182,12 +219,12 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
 }
 
 template <int NB, int EPI, int TILES, bool F16>
-int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, int K, void* out, int ldo, cudaStream_t st) {
+int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, void* out, int ldo, cudaStream_t st) {
   static bool configured = false;
-  static int num_sms = 0;
-  constexpr int STAGE_BYTES = TILES * W_TILE_BYTES + NB * A_TILE_BYTES;
-  constexpr int MAX_DYN = GS_WARPS * GS_MAX_SLOTS * STAGE_BYTES + 1024 > 200 * 1024 ? 200 * 1024
-                                                                                       : GS_WARPS * GS_MAX_SLOTS * STAGE_BYTES + 1024;
+  static int num_sms = 0, smem_per_sm = 0;
+  constexpr int STAGE_BYTES = TILES * W_CHUNK_BYTES;
+  constexpr int MAX_DYN = GS_WARPS * GS_MAX_SLOTS * STAGE_BYTES + 128 > 200 * 1024 ? 200 * 1024
+                                                                                     : GS_WARPS * GS_MAX_SLOTS * STAGE_BYTES + 128;
   if (!configured) {
     HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_stream_kernel<NB, EPI, TILES, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN));
     // several CTAs per SM share the ring space: ask for the largest shared-memory carve-out
@@ -196,55 +233,59 @@ int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
     int dev = 0;
     HYP_CUDA_TRY(cudaGetDevice(&dev));
     HYP_CUDA_TRY(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
+    HYP_CUDA_TRY(cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev));
     configured = true;
   }
   constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
   constexpr int OUT_COLS = (TILES == 2 && !SWIGLU) ? 32 : 16;
   const int n_ctas = (N + OUT_COLS - 1) / OUT_COLS;
-  // Ring depth (slots per warp).  Measured on B200: throughput peaks when roughly 28 k-block copies (and
-  // no more than ~110 KB) are in flight per SM and falls off sharply beyond that (3 slots at 3.2 CTAs/SM run at half the speed of 2),
-  // so the depth follows from how many CTAs share an SM; two slots are the floor (one slot exposes the
-  // full memory latency), four the ceiling.
-  double ctas_per_sm = (double)n_ctas / num_sms;
-  if (ctas_per_sm > 5.0) ctas_per_sm = 5.0;
-  int slots = (int)(28.0 / (GS_WARPS * ctas_per_sm));
-  const int by_bytes = (int)(110.0 * 1024 / (GS_WARPS * ctas_per_sm * STAGE_BYTES));  // and ~110 KB in flight per SM
-  if (by_bytes < slots) slots = by_bytes;
-  if (slots > 4) slots = 4;
+  // Ring depth (slots per warp).  A grid whose CTAs are not all resident at once ends with a partial wave that
+  // cannot keep HBM busy (measured on B200: 320 CTAs at 2 per SM take 1.4x the time of the same CTAs at 3 per
+  // SM), and one that could fit more CTAs per SM than it needs may be placed unevenly when it starts while its
+  // predecessor still holds part of the SMs.  So when the grid fits in one wave the ring takes whatever shared
+  // memory that residency leaves: this caps the CTAs per SM at ceil(CTAs / SMs), and the more of a strip a CTA
+  // holds, the more it fetches while its predecessor drains.  Grids of several waves take two slots (more
+  // CTAs per SM hide each other's start and end).  1 KB per CTA is reserved by the driver; 512 B cover barriers
+  // and alignment.
+  const int per_sm = (n_ctas + num_sms - 1) / num_sms;
+  int slots = (smem_per_sm / per_sm - 1024 - 512) / (GS_WARPS * STAGE_BYTES);
+  if (slots > GS_MAX_SLOTS) slots = GS_MAX_SLOTS;
   if (slots < 2) slots = 2;
-  while (slots > 1 && GS_WARPS * slots * STAGE_BYTES + 1024 > MAX_DYN) --slots;
-  const int smem = GS_WARPS * slots * STAGE_BYTES + 1024;
-  HYP_CUDA_TRY(launch_pdl(gemm_stream_kernel<NB, EPI, TILES, F16>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
-                          (TILES == 2 && !SWIGLU) ? w.map_small[1] : w.map_small[0], act.map_small[NB - 1], N, K, M, out,
-                          ldo, slots, tc_err_flag_ptr()));
+  if (gemm_stream_slots_override() > 0) slots = gemm_stream_slots_override();
+  if (slots > GS_MAX_SLOTS) slots = GS_MAX_SLOTS;
+  while (slots > 2 && GS_WARPS * slots * STAGE_BYTES + 128 > MAX_DYN) --slots;
+  const int smem = GS_WARPS * slots * STAGE_BYTES + 128;
+  HYP_CUDA_TRY(launch_pdl<true>(gemm_stream_kernel<NB, EPI, TILES, F16>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
+                          (const uint8_t*)w.packed, (const uint16_t*)act.ptr, act.K, act.K, N, w.KBp, w.N16p, M, out, ldo,
+                          slots, tc_err_flag_ptr()));
   return 1;
 }
 
 template <int NB, bool F16>
-int launch_nb(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo, cudaStream_t st) {
-  const bool wide = N > 8192;  // many rows: 32 columns per CTA keep the CTA count within one resident wave
+int launch_nb(const TcAct& act, const TcWeight& w, int M, int N, int epi, void* out, int ldo, cudaStream_t st) {
+  const bool wide = N > 8192;  // many rows: 32 columns per CTA keep the CTA count down
   switch (epi) {
     case EPI_STORE_BF16:
-      return wide ? launch_cfg<NB, EPI_STORE_BF16, 2, F16>(act, w, M, N, K, out, ldo, st)
-                  : launch_cfg<NB, EPI_STORE_BF16, 1, F16>(act, w, M, N, K, out, ldo, st);
+      return wide ? launch_cfg<NB, EPI_STORE_BF16, 2, F16>(act, w, M, N, out, ldo, st)
+                  : launch_cfg<NB, EPI_STORE_BF16, 1, F16>(act, w, M, N, out, ldo, st);
     case EPI_RESID_F32:
-      return wide ? launch_cfg<NB, EPI_RESID_F32, 2, F16>(act, w, M, N, K, out, ldo, st)
-                  : launch_cfg<NB, EPI_RESID_F32, 1, F16>(act, w, M, N, K, out, ldo, st);
+      return wide ? launch_cfg<NB, EPI_RESID_F32, 2, F16>(act, w, M, N, out, ldo, st)
+                  : launch_cfg<NB, EPI_RESID_F32, 1, F16>(act, w, M, N, out, ldo, st);
     case EPI_STORE_F32:
-      return wide ? launch_cfg<NB, EPI_STORE_F32, 2, F16>(act, w, M, N, K, out, ldo, st)
-                  : launch_cfg<NB, EPI_STORE_F32, 1, F16>(act, w, M, N, K, out, ldo, st);
-    case EPI_SWIGLU_BF16: return launch_cfg<NB, EPI_SWIGLU_BF16, 2, F16>(act, w, M, N, K, out, ldo, st);
+      return wide ? launch_cfg<NB, EPI_STORE_F32, 2, F16>(act, w, M, N, out, ldo, st)
+                  : launch_cfg<NB, EPI_STORE_F32, 1, F16>(act, w, M, N, out, ldo, st);
+    case EPI_SWIGLU_BF16: return launch_cfg<NB, EPI_SWIGLU_BF16, 2, F16>(act, w, M, N, out, ldo, st);
     default: return HYP_EINVAL;
   }
 }
 
 template <bool F16>
-int launch_type(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo, cudaStream_t st) {
+int launch_type(const TcAct& act, const TcWeight& w, int M, int N, int epi, void* out, int ldo, cudaStream_t st) {
   switch ((M + 7) / 8) {
-    case 1: return launch_nb<1, F16>(act, w, M, N, K, epi, out, ldo, st);
-    case 2: return launch_nb<2, F16>(act, w, M, N, K, epi, out, ldo, st);
-    case 3: return launch_nb<3, F16>(act, w, M, N, K, epi, out, ldo, st);
-    default: return launch_nb<4, F16>(act, w, M, N, K, epi, out, ldo, st);
+    case 1: return launch_nb<1, F16>(act, w, M, N, epi, out, ldo, st);
+    case 2: return launch_nb<2, F16>(act, w, M, N, epi, out, ldo, st);
+    case 3: return launch_nb<3, F16>(act, w, M, N, epi, out, ldo, st);
+    default: return launch_nb<4, F16>(act, w, M, N, epi, out, ldo, st);
   }
 }
 
@@ -253,9 +294,10 @@ int launch_type(const TcAct& act, const TcWeight& w, int M, int N, int K, int ep
 int launch_gemm_stream(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
                        cudaStream_t st) {
   if (M < 1 || M > 32 || N < 1 || K < 8 || act.K != K || w.K != K || !tc_err_flag_ptr()) return HYP_EINVAL;
+  if (w.rows != N || w.halves != (epi == EPI_SWIGLU_BF16 ? 2 : 1)) return HYP_EINVAL;
   if (act.f16 != w.f16) return HYP_EINVAL;  // one instruction takes both operands in the same 16-bit type
-  return act.f16 ? launch_type<true>(act, w, M, N, K, epi, out, ldo, st)
-                 : launch_type<false>(act, w, M, N, K, epi, out, ldo, st);
+  if (((uintptr_t)act.ptr & 15) != 0 || (K % 8) != 0) return HYP_EINVAL;  // 128-bit activation loads
+  return act.f16 ? launch_type<true>(act, w, M, N, epi, out, ldo, st) : launch_type<false>(act, w, M, N, epi, out, ldo, st);
 }
 
 }  // namespace hyp

@@ -17,6 +17,8 @@
 // Every mbarrier wait is bounded: on expiry the kernel records an error code and unwinds.
 #include <cuda.h>
 
+#include <algorithm>
+
 #include "gemm_tc.cuh"
 #include "sm100_common.cuh"
 #include "hyperion.h"
@@ -179,7 +181,7 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[16], const ui
 template <int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int M, int N, int K,
-               void* __restrict__ out, int ldo, int team, uint32_t idesc, int* __restrict__ err) {
+               int up_tile0, void* __restrict__ out, int ldo, int team, uint32_t idesc, int* __restrict__ err) {
   constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
   const bool STREAMK = EPI == EPI_RESID_F32 && team > 0;
   constexpr int BN_OUT = SWIGLU ? BN / 2 : BN;  // output columns per tile
@@ -234,14 +236,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       while (ok && seg.next(tile, kb0, kb1)) {
         const int m0 = (tile % tiles_m) * BM;
         const int n0 = (tile / tiles_m) * BN_OUT;
-        const int rb0 = n0, rb1 = SWIGLU ? N + n0 : n0 + 128;
+        // weight tiles (16 rows each) of the two 128-row boxes: SwiGLU pairs gate rows with the matching up rows
+        const int tb0 = n0 >> 4, tb1 = SWIGLU ? up_tile0 + (n0 >> 4) : (n0 >> 4) + 8;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) { ok = false; break; }
           const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
           mbar_expect_tx(full_bar(stage), STAGE_BYTES);
           tma_load_2d(sa, &tm_a, kb * BK, m0, full_bar(stage));
-          tma_load_2d(sb, &tm_b, kb * BK, rb0, full_bar(stage));
-          tma_load_2d(sb + B_BYTES / 2, &tm_b, kb * BK, rb1, full_bar(stage));
+          tma_load_4d(sb, &tm_b, 0, 0, kb, tb0, full_bar(stage));
+          tma_load_4d(sb + B_BYTES / 2, &tm_b, 0, 0, kb, tb1, full_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
       }
@@ -370,6 +373,13 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
       : "memory");
 }
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                                 uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {  // arrive on `bar` (same offset) in both CTAs
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                ::"r"(bar), "h"((uint16_t)3)
@@ -387,7 +397,7 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uin
 template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int M, int N, int K,
-                void* __restrict__ out, int ldo, uint32_t idesc, int* __restrict__ err) {
+                int up_tile0, void* __restrict__ out, int ldo, uint32_t idesc, int* __restrict__ err) {
   constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
   constexpr int BN_OUT = SWIGLU ? BN / 2 : BN;
   extern __shared__ uint8_t smem_raw[];
@@ -443,14 +453,15 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
         const int m0 = (tile % pairs_m) * (2 * BM) + (int)rank * BM;
         const int n0 = (tile / pairs_m) * BN_OUT;
-        const int rb = SWIGLU ? (int)rank * N + n0 : n0 + (int)rank * (BN / 2);  // this CTA's half of the weight tile
+        // this CTA's half of the weight tile, as an index of 16-row packed tiles
+        const int tb = SWIGLU ? (int)rank * up_tile0 + (n0 >> 4) : (n0 >> 4) + (int)rank * 8;
         for (int kb = 0; kb < KB; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) { ok = false; break; }
           const uint32_t sa = base + stage * STAGE2_BYTES, sb = sa + A_BYTES;
           const uint32_t lead_full = mapa_rank(full_bar(stage), 0);
           if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * STAGE2_BYTES);
           tma_load_2d_pair(sa, &tm_a, kb * BK, m0, lead_full);
-          tma_load_2d_pair(sb, &tm_b, kb * BK, rb, lead_full);
+          tma_load_4d_pair(sb, &tm_b, 0, 0, kb, tb, lead_full);
           if (++stage == STAGES2) { stage = 0; phase ^= 1; }
         }
       }
@@ -583,7 +594,7 @@ int launch_pair(const TcAct& act, const TcWeight& w, int M, int N, int K, void* 
   long pairs = num_sms / 2;
   if (tiles < pairs) pairs = tiles;
   HYP_CUDA_TRY(launch_pdl(gemm_tc2_kernel<EPI>, dim3((unsigned)(2 * pairs)), dim3(TC_THREADS), (size_t)SMEM2_BYTES, st, act.map,
-                          w.map, M, N, K, out, ldo, act.f16 ? IDESC2_F16 : IDESC2_BF16, g_err_flag));
+                          w.map, M, N, K, w.N16p, out, ldo, act.f16 ? IDESC2_F16 : IDESC2_BF16, g_err_flag));
   return 1;
 }
 
@@ -621,24 +632,73 @@ int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
     grid = (int)(tiles < num_sms ? tiles : num_sms);
   }
   HYP_CUDA_TRY(launch_pdl(gemm_tc_kernel<EPI>, dim3(grid), dim3(TC_THREADS), (size_t)SMEM_BYTES, st, act.map, w.map, M, N,
-                          K, out, ldo, team, act.f16 ? IDESC_F16 : IDESC_BF16, g_err_flag));
+                          K, w.N16p, out, ldo, team, act.f16 ? IDESC_F16 : IDESC_BF16, g_err_flag));
   return 1;
 }
 
 }  // namespace
 
-// Weights: 128-row boxes for the tile kernel, 16- and 32-row boxes for the weight-streaming kernel.
-int tc_make_weight(TcWeight* w, const void* ptr, int rows, int K, bool f16) {
-  w->ptr = (const __nv_bfloat16*)ptr; w->rows = rows; w->K = K; w->f16 = f16;
-  int rc = encode_map(&w->map, ptr, rows, K, 128, f16);
-  if (rc) return rc;
-  rc = encode_map(&w->map_small[0], ptr, rows, K, 16, f16);
-  if (rc) return rc;
-  return encode_map(&w->map_small[1], ptr, rows, K, 32, f16);
+// Packed weights: one 4-D descriptor whose box is eight 16-row tiles of one k-block (a 128-row operand tile).  The
+// tiles already carry the 128-byte swizzle, so the copy itself applies none.
+int tc_make_weight(TcWeight* w, const void* packed, int rows, int halves, int K, bool f16) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return HYP_ECUDA;
+  if (rows < 1 || (halves != 1 && halves != 2) || K < 8 || (K % 8) != 0 || ((uintptr_t)packed & 127) != 0) return HYP_EINVAL;
+  w->packed = packed; w->rows = rows; w->halves = halves; w->K = K; w->f16 = f16;
+  w->KBp = pk_kbp(K);
+  w->N16p = pk_n16p(rows);
+  const cuuint64_t dims[4] = {64, 16, (cuuint64_t)w->KBp, (cuuint64_t)halves * w->N16p};
+  const cuuint64_t strides[3] = {128, (cuuint64_t)PK_TILE_BYTES, (cuuint64_t)w->KBp * PK_TILE_BYTES};
+  const cuuint32_t box[4] = {64, 16, 1, 8};
+  const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  CUresult r = enc(&w->map, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void*)packed, dims,
+                   strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error((int)r);
+    return HYP_ECUDA;
+  }
+  return HYP_OK;
 }
+
+namespace {
+// One thread per 16-byte chunk of the packed buffer: finds the source row and k of its chunk, converts, stores.
+__global__ void pack_weight_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int rows, int halves, int K,
+                                   int N16p, int KBp, bool to_f16) {
+  const size_t total = (size_t)halves * N16p * KBp * (PK_TILE_BYTES / 16);
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+    const int c_sw = (int)(idx & 7), r = (int)((idx >> 3) & 15);
+    const size_t tile = idx >> 7;
+    const int kb = (int)(tile % KBp);
+    const int t = (int)(tile / KBp);
+    const int half = t / N16p, n = (t % N16p) * 16 + r;
+    const int k = kb * 64 + ((c_sw ^ (r & 7)) << 3);
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (n < rows && k < K) {
+      v = src[((size_t)(half * rows + n) * K + k) >> 3];
+      if (to_f16) {
+        uint32_t* p = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) p[i] = pack_f16_sat(bf16_lo(p[i]), bf16_hi(p[i]));
+      }
+    }
+    dst[idx] = v;
+  }
+}
+}  // namespace
+
+int tc_pack_weight(const void* src, void* dst, int rows, int halves, int K, bool to_f16, cudaStream_t st) {
+  if (!src || !dst || rows < 1 || (halves != 1 && halves != 2) || K < 8 || (K % 8) != 0) return HYP_EINVAL;
+  if (((uintptr_t)src & 15) != 0 || ((uintptr_t)dst & 15) != 0) return HYP_EINVAL;
+  const size_t chunks = tc_packed_bytes(rows, halves, K) / 16;
+  const int blocks = (int)std::min<size_t>((chunks + 255) / 256, (size_t)148 * 16);
+  pack_weight_kernel<<<blocks, 256, 0, st>>>((const uint4*)src, (uint4*)dst, rows, halves, K, pk_n16p(rows), pk_kbp(K), to_f16);
+  return 1;
+}
+
 // Activations: 128-row boxes for the tile kernel, 8/16/24/32-row boxes for the weight-streaming kernel.
 int tc_make_act(TcAct* a, const void* ptr, int rows, int K, bool f16) {
-  a->ptr = (const __nv_bfloat16*)ptr; a->rows = rows; a->K = K; a->f16 = f16;
+  a->ptr = ptr; a->rows = rows; a->K = K; a->f16 = f16;
   int rc = encode_map(&a->map, ptr, rows, K, 128, f16);
   for (int nb = 1; nb <= 4 && !rc; ++nb) rc = encode_map(&a->map_small[nb - 1], ptr, rows, K, 8 * nb, f16);
   return rc;
@@ -664,6 +724,7 @@ int tc_error_flag(int* value_out) {
 int launch_gemm_tc(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
                    cudaStream_t st) {
   if (M < 1 || N < 1 || K < 8 || act.K != K || w.K != K || M > act.rows || !g_err_flag) return HYP_EINVAL;
+  if (w.rows != N || w.halves != (epi == EPI_SWIGLU_BF16 ? 2 : 1)) return HYP_EINVAL;
   if (act.f16 != w.f16) return HYP_EINVAL;  // one instruction takes both operands in the same 16-bit type
   switch (epi) {
     case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16>(act, w, M, N, K, out, ldo, st);

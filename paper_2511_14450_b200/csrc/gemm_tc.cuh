@@ -1,4 +1,4 @@
-// Tensor-core projection for any row count (prefill): operand descriptors and launcher.
+// Projection operands (packed weights, activation descriptors) and the launchers of the two projection kernels.
 #pragma once
 #include <cuda.h>
 
@@ -6,19 +6,41 @@
 
 namespace hyp {
 
-// A 16-bit matrix [rows, K] row-major (bf16, or fp16 when f16) together with the TMA descriptors that tile
-// it.  Both operands of a projection must have the same type.
-struct TcOperand {
-  CUtensorMap map;
-  const __nv_bfloat16* ptr = nullptr;
+// Packed weight layout.  A projection matrix w[n, k] (n < rows, k < K; SwiGLU: two such halves, gate then up) is
+// held as tiles of 16 rows x 64 k (2 KB), tile (t, kb) at byte offset (t * KBp + kb) * 2048 with t = half * N16p +
+// n / 16: all k-blocks of one 16-row strip are contiguous, so the weight-streaming kernel reads every strip as one
+// sequential run of bulk copies and the tile kernel fetches a 128-row operand tile as eight 2 KB pieces.  Inside a
+// tile, row r (128 bytes) keeps its 16-byte chunk c at chunk position c ^ (r & 7): the 128-byte swizzle that
+// ldmatrix (conflict-free) and the tcgen05 shared-memory descriptors expect, applied once at load time.  Rows
+// beyond `rows` and k beyond K are zero.  N16p = tiles per half (even), KBp = k-blocks per strip (even).
+constexpr int PK_TILE_BYTES = 2048;
+struct TcWeight {
+  const void* packed = nullptr;
+  int rows = 0;    // logical rows per half
+  int halves = 1;  // 2: SwiGLU gate | up
+  int K = 0, KBp = 0, N16p = 0;
+  bool f16 = false;
+  CUtensorMap map;  // 4-D view {64 k, 16 rows, KBp, halves * N16p}, box = 8 tiles x 1 k-block (128 rows), no swizzle
+};
+inline int pk_kbp(int K) { return ((K + 63) / 64 + 1) & ~1; }
+inline int pk_n16p(int rows) { return ((rows + 15) / 16 + 1) & ~1; }
+inline size_t tc_packed_bytes(int rows, int halves, int K) {
+  return (size_t)halves * pk_n16p(rows) * pk_kbp(K) * PK_TILE_BYTES;
+}
+// src: bf16 [halves * rows, K] row-major (DEVICE, 16-byte aligned, K multiple of 8); dst: tc_packed_bytes(...) bytes.
+// to_f16 converts the values to fp16 (exact for |w| >= 2^-17, saturating at +-65504); otherwise they stay bf16.
+int tc_pack_weight(const void* src, void* dst, int rows, int halves, int K, bool to_f16, cudaStream_t st);
+int tc_make_weight(TcWeight* w, const void* packed, int rows, int halves, int K, bool f16);
+
+// A 16-bit activation matrix [rows, K] row-major (bf16, or fp16 when f16) with the TMA descriptors that tile it.
+// Both operands of a projection must have the same type.
+struct TcAct {
+  CUtensorMap map;  // 128-row boxes (tile kernel)
+  const void* ptr = nullptr;
   int rows = 0, K = 0;
   bool f16 = false;
-  CUtensorMap map_small[4];  // weight-streaming kernel: weights [0], [1] = 16-, 32-row boxes; activations [nb-1] = 8*nb rows
+  CUtensorMap map_small[4];  // weight-streaming kernel: [nb - 1] = boxes of 8 * nb rows
 };
-typedef TcOperand TcWeight;
-typedef TcOperand TcAct;
-
-int tc_make_weight(TcWeight* w, const void* ptr, int rows, int K, bool f16 = false);
 int tc_make_act(TcAct* a, const void* ptr, int rows, int K, bool f16 = false);
 
 // One-time set-up of the device-side error word (allocates; call from stage creation, not from the hot path).
@@ -29,11 +51,14 @@ int tc_error_flag(int* value_out);
 // Device word that kernels set when a bounded wait expires (null before tc_prepare).
 int* tc_err_flag_ptr();
 
-// Weight-streaming projection for M <= 32 rows (decode), fed by TMA; same contract as launch_gemm_tc.
+// Ring depth override of the weight-streaming kernel (0 = the built-in choice).
+int& gemm_stream_slots_override();
+
+// Weight-streaming projection for M <= 32 rows (decode); same contract as launch_gemm_tc.
 int launch_gemm_stream(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
                        cudaStream_t st);
 
-// out[m, n] (+)= sum_k act[m, k] * w[n, k] for m < M, n < N (SwiGLU: w holds 2N rows).
+// out[m, n] (+)= sum_k act[m, k] * w[n, k] for m < M, n < N (SwiGLU: w holds two halves of N rows).
 int launch_gemm_tc(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
                    cudaStream_t st);
 

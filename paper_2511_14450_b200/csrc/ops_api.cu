@@ -39,9 +39,33 @@ extern "C" int hyp_op_rmsnorm(const float* x, const void* g, void* out, int32_t 
                                (cudaStream_t)stream));
 }
 
+extern "C" size_t hyp_op_weight_packed_bytes(int32_t N, int32_t K, int32_t swiglu) {
+  if (N < 1 || K < 8 || K % 8) return 0;
+  return tc_packed_bytes(N, swiglu ? 2 : 1, K);
+}
+
+extern "C" int hyp_op_pack_weight(const void* w, int32_t N, int32_t K, int32_t swiglu, void* packed, size_t packed_bytes,
+                                  void* stream) {
+  if (!w || !packed || N < 1 || K < 8 || K % 8) return HYP_EINVAL;
+  if (((uintptr_t)w & 15) != 0 || ((uintptr_t)packed & 127) != 0) return HYP_EINVAL;
+  if (packed_bytes < tc_packed_bytes(N, swiglu ? 2 : 1, K)) return HYP_ECAPACITY;
+  return finish(tc_pack_weight(w, packed, N, swiglu ? 2 : 1, K, false, (cudaStream_t)stream));
+}
+
+extern "C" int hyp_tune(int32_t key, int32_t value) {
+  switch (key) {
+    case HYP_TUNE_PDL: pdl_enabled() = value != 0; return HYP_OK;
+    case HYP_TUNE_STREAM_SLOTS:
+      if (value < 0 || value > 8) return HYP_EINVAL;
+      gemm_stream_slots_override() = value;
+      return HYP_OK;
+    default: return HYP_EINVAL;
+  }
+}
+
 extern "C" int hyp_op_gemm(const void* a, const void* w, int32_t M, int32_t N, int32_t K, int32_t epilogue, void* out,
                            int32_t ldo, void* stream) {
-  if (!a || !w || !out || M < 1 || N < 1 || K < 8 || K % 8 || ldo < N) return HYP_EINVAL;
+  if (!a || !w || !out || M < 1 || N < 1 || K < 8 || K % 8 || ldo < N || ((uintptr_t)w & 127) != 0) return HYP_EINVAL;
   if (epilogue < HYP_EPI_STORE_BF16 || epilogue > HYP_EPI_STORE_F32) return HYP_EINVAL;
   cudaStream_t st = (cudaStream_t)stream;
   if (M > 32 && (N % 16 || ldo % 8)) return HYP_EINVAL;
@@ -51,7 +75,7 @@ extern "C" int hyp_op_gemm(const void* a, const void* w, int32_t M, int32_t N, i
   TcWeight tw;
   rc = tc_make_act(&ta, (const __nv_bfloat16*)a, M, K);
   if (rc) return rc;
-  rc = tc_make_weight(&tw, (const __nv_bfloat16*)w, epilogue == HYP_EPI_SWIGLU_BF16 ? 2 * N : N, K);
+  rc = tc_make_weight(&tw, w, N, epilogue == HYP_EPI_SWIGLU_BF16 ? 2 : 1, K, false);
   if (rc) return rc;
   if (M <= 32) return finish(launch_gemm_stream(ta, tw, M, N, K, epilogue, out, ldo, st));
   return finish(launch_gemm_tc(ta, tw, M, N, K, epilogue, out, ldo, st));

@@ -24,7 +24,9 @@ namespace {
 constexpr int META_RING = 4;
 
 struct LayerW {
-  bf16 *wqkv = nullptr, *wo = nullptr, *wgu = nullptr, *wd = nullptr, *g1 = nullptr, *g2 = nullptr;
+  // projection matrices in the packed fp16 layout of gemm_tc.cuh; gains as loaded (bf16)
+  void *wqkv = nullptr, *wo = nullptr, *wgu = nullptr, *wd = nullptr;
+  bf16 *g1 = nullptr, *g2 = nullptr;
   uint32_t loaded = 0;
   TcWeight tc_qkv, tc_o, tc_gu, tc_d;
 };
@@ -37,7 +39,8 @@ struct hyp_stage {
   bool first = false, last = false;
   ModelDims dims;
   std::vector<LayerW> layers;
-  bf16 *embed = nullptr, *gf = nullptr, *wlm = nullptr;
+  bf16 *embed = nullptr, *gf = nullptr;
+  void* wlm = nullptr;  // packed fp16
   TcWeight tc_lm;
   uint32_t loaded_extra = 0;
   // KV cache (fp16)
@@ -113,6 +116,31 @@ size_t tensor_elems(const hyp_stage* s, int tensor_id) {
     case HYP_W_LM_HEAD: return (size_t)d.V * d.H;
     default: return 0;
   }
+}
+
+// Rows per half, halves and K of a projection matrix (its packed form is sized from these).
+bool proj_geometry(const hyp_stage* s, int tensor_id, int* rows, int* halves, int* K) {
+  const ModelDims& d = s->dims;
+  *halves = 1;
+  switch (tensor_id) {
+    case HYP_W_QKV: *rows = d.qkv_rows; *K = d.H; return true;
+    case HYP_W_O: *rows = d.H; *K = d.Hq * d.D; return true;
+    case HYP_W_GATE_UP: *rows = d.F; *halves = 2; *K = d.H; return true;
+    case HYP_W_DOWN: *rows = d.H; *K = d.F; return true;
+    case HYP_W_LM_HEAD: *rows = d.V; *K = d.H; return true;
+    default: return false;
+  }
+}
+size_t proj_packed_bytes(const hyp_stage* s, int tensor_id) {
+  int rows, halves, K;
+  if (!proj_geometry(s, tensor_id, &rows, &halves, &K)) return 0;
+  return tc_packed_bytes(rows, halves, K);
+}
+int dev_alloc_bytes(void** p, size_t bytes) {
+  uint8_t* q = nullptr;
+  const int rc = dev_alloc(&q, bytes);
+  *p = q;
+  return rc;
 }
 
 struct HostBatch {
@@ -512,17 +540,17 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
   TRY_CUDA(cudaGetDevice(&s->device));
   s->layers.resize(s->L);
   for (LayerW& lw : s->layers) {
-    TRY(dev_alloc(&lw.wqkv, tensor_elems(s, HYP_W_QKV)));
-    TRY(dev_alloc(&lw.wo, tensor_elems(s, HYP_W_O)));
-    TRY(dev_alloc(&lw.wgu, tensor_elems(s, HYP_W_GATE_UP)));
-    TRY(dev_alloc(&lw.wd, tensor_elems(s, HYP_W_DOWN)));
+    TRY(dev_alloc_bytes(&lw.wqkv, proj_packed_bytes(s, HYP_W_QKV)));
+    TRY(dev_alloc_bytes(&lw.wo, proj_packed_bytes(s, HYP_W_O)));
+    TRY(dev_alloc_bytes(&lw.wgu, proj_packed_bytes(s, HYP_W_GATE_UP)));
+    TRY(dev_alloc_bytes(&lw.wd, proj_packed_bytes(s, HYP_W_DOWN)));
     TRY(dev_alloc(&lw.g1, (size_t)d.H));
     TRY(dev_alloc(&lw.g2, (size_t)d.H));
   }
   if (s->first) TRY(dev_alloc(&s->embed, tensor_elems(s, HYP_W_EMBED)));
   if (s->last) {
     TRY(dev_alloc(&s->gf, (size_t)d.H));
-    TRY(dev_alloc(&s->wlm, tensor_elems(s, HYP_W_LM_HEAD)));
+    TRY(dev_alloc_bytes(&s->wlm, proj_packed_bytes(s, HYP_W_LM_HEAD)));
   }
   // KV pool: [layer][page][K,V][Hkv][16][D]
   s->max_pages_per_seq = (c.max_ctx + c.kv_block_size - 1) / c.kv_block_size;
@@ -586,13 +614,13 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
   TRY(tc_make_act(&s->tc_attn, s->attn, (int)rows_pad, d.Hq * d.D, true));
   TRY(tc_make_act(&s->tc_u, s->u, (int)rows_pad, d.F, true));
   for (LayerW& lw : s->layers) {
-    // all projection matrices are held as fp16, see hyp_stage_load
-    TRY(tc_make_weight(&lw.tc_qkv, lw.wqkv, d.qkv_rows, d.H, true));
-    TRY(tc_make_weight(&lw.tc_o, lw.wo, d.H, d.Hq * d.D, true));
-    TRY(tc_make_weight(&lw.tc_gu, lw.wgu, 2 * d.F, d.H, true));
-    TRY(tc_make_weight(&lw.tc_d, lw.wd, d.H, d.F, true));
+    // all projection matrices are held packed as fp16, see hyp_stage_load
+    TRY(tc_make_weight(&lw.tc_qkv, lw.wqkv, d.qkv_rows, 1, d.H, true));
+    TRY(tc_make_weight(&lw.tc_o, lw.wo, d.H, 1, d.Hq * d.D, true));
+    TRY(tc_make_weight(&lw.tc_gu, lw.wgu, d.F, 2, d.H, true));
+    TRY(tc_make_weight(&lw.tc_d, lw.wd, d.H, 1, d.F, true));
   }
-  if (s->last) TRY(tc_make_weight(&s->tc_lm, s->wlm, d.V, d.H, true));
+  if (s->last) TRY(tc_make_weight(&s->tc_lm, s->wlm, d.V, 1, d.H, true));
 #undef TRY
 #undef TRY_CUDA
   *out = s;
@@ -607,7 +635,7 @@ extern "C" int hyp_stage_load(hyp_stage* s, int32_t layer, int32_t tensor_id, co
   if (tensor_id >= HYP_W_QKV && tensor_id <= HYP_W_NORM2) {
     if (layer < s->lo || layer >= s->hi) return HYP_EINVAL;
     LayerW& lw = s->layers[layer - s->lo];
-    bf16* ptrs[6] = {lw.wqkv, lw.wo, lw.wgu, lw.wd, lw.g1, lw.g2};
+    void* ptrs[6] = {lw.wqkv, lw.wo, lw.wgu, lw.wd, lw.g1, lw.g2};
     dst = ptrs[tensor_id];
     mask = &lw.loaded;
   } else if (tensor_id == HYP_W_EMBED) {
@@ -624,9 +652,12 @@ extern "C" int hyp_stage_load(hyp_stage* s, int32_t layer, int32_t tensor_id, co
   if (bytes != tensor_elems(s, tensor_id) * sizeof(bf16)) return HYP_EINVAL;
   if (tensor_id <= HYP_W_DOWN || tensor_id == HYP_W_LM_HEAD) {
     // projection matrices are kept as fp16 so that the projections can take fp16 activations
-    // (bf16 -> fp16 is exact for |w| >= 2^-17 and off by < 3e-8 below that)
+    // (bf16 -> fp16 is exact for |w| >= 2^-17 and off by < 3e-8 below that), in the packed tile order
     if (((uintptr_t)src & 15) != 0) return HYP_EINVAL;
-    launch_bf16_to_f16((const bf16*)src, (__half*)dst, bytes / sizeof(bf16), (cudaStream_t)stream);
+    int rows, halves, K;
+    proj_geometry(s, tensor_id, &rows, &halves, &K);
+    const int prc = tc_pack_weight(src, dst, rows, halves, K, true, (cudaStream_t)stream);
+    if (prc < 0) return prc;
     cudaError_t e = cudaPeekAtLastError();
     if (e != cudaSuccess) {
       set_last_cuda_error((int)e);

@@ -75,6 +75,9 @@ SIGNATURES = {
                                C.POINTER(C.c_double)]),
     "hyp_sched_rt": (C.c_int, [C.c_double, C.c_double, C.POINTER(hyp_node_state), C.c_int32, C.POINTER(C.c_int32)]),
     "hyp_op_rmsnorm": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_void_p]),
+    "hyp_op_weight_packed_bytes": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int32]),
+    "hyp_op_pack_weight": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "hyp_tune": (C.c_int, [C.c_int32, C.c_int32]),
     "hyp_op_gemm": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
                               C.c_int32, C.c_void_p]),
     "hyp_op_attn_decode_splits": (C.c_int, [C.c_int32, C.c_int32, C.c_int32]),
@@ -265,10 +268,30 @@ def hyp_op_rmsnorm(x, g, out, eps: float, stream=None):
     _check(lib().hyp_op_rmsnorm(_ptr(x), _ptr(g), _ptr(out), M, H, eps, _stream_handle(stream)), "hyp_op_rmsnorm")
 
 
-def hyp_op_gemm(a, w, N: int, epilogue: int, out, stream=None):
+HYP_TUNE_PDL, HYP_TUNE_STREAM_SLOTS = range(2)
+
+
+def hyp_tune(key: int, value: int):
+    _check(lib().hyp_tune(key, value), "hyp_tune")
+
+
+def hyp_op_pack_weight(w, N: int, swiglu: bool, stream=None):
+    """Packed copy of a bf16 [N (2N for SwiGLU), K] weight matrix, as hyp_op_gemm reads it (a uint8 tensor)."""
+    import torch
+    K = w.shape[1]
+    nbytes = lib().hyp_op_weight_packed_bytes(N, K, int(swiglu))
+    if nbytes == 0:
+        raise HyperionError(HYP_EINVAL, "hyp_op_weight_packed_bytes")
+    packed = torch.empty(nbytes, dtype=torch.uint8, device=w.device)
+    _check(lib().hyp_op_pack_weight(_ptr(w), N, K, int(swiglu), _ptr(packed), nbytes, _stream_handle(stream)),
+           "hyp_op_pack_weight")
+    return packed
+
+
+def hyp_op_gemm(a, w_packed, N: int, epilogue: int, out, stream=None):
     M, K = a.shape
-    _check(lib().hyp_op_gemm(_ptr(a), _ptr(w), M, N, K, epilogue, _ptr(out), out.stride(0), _stream_handle(stream)),
-           "hyp_op_gemm")
+    _check(lib().hyp_op_gemm(_ptr(a), _ptr(w_packed), M, N, K, epilogue, _ptr(out), out.stride(0),
+                             _stream_handle(stream)), "hyp_op_gemm")
 
 
 def hyp_op_attn_decode_splits(n_seqs: int, n_kv_heads: int, max_ctx: int) -> int:

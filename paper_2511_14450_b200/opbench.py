@@ -41,7 +41,8 @@ def gemm(M, N, K, epi, iters=20):
     rows = 2 * N if epi == "swiglu" else N
     n_w = max(2, min(8, int(600e6 // (rows * K * 2)) + 1))     # rotate > L2 worth of weights
     a = torch.randn(M, K, device="cuda").bfloat16()
-    ws = [(torch.randn(rows, K, device="cuda") * 0.02).bfloat16() for _ in range(n_w)]
+    ws = [hyp.hyp_op_pack_weight((torch.randn(rows, K, device="cuda") * 0.02).bfloat16(), N, epi == "swiglu")
+          for _ in range(n_w)]
     out = torch.zeros(M, N, device="cuda", dtype=torch.bfloat16 if epi in ("bf16", "swiglu") else torch.float32)
     ms = _time(lambda i: hyp.hyp_op_gemm(a, ws[i % n_w], N, EPI[epi], out), iters)
     return {"op": "gemm", "M": M, "N": N, "K": K, "epi": epi, "us": ms * 1e3,

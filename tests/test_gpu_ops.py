@@ -57,7 +57,7 @@ def test_gemm_all_epilogues(M, N, K, epi):
         out = res.clone()
         want = acc + (f64(res) if epi == hyp.HYP_EPI_RESID_F32 else 0.0)
         tol = 2e-5 * np.sqrt(K)
-    hyp.hyp_op_gemm(a, w, N, epi, out)
+    hyp.hyp_op_gemm(a, hyp.hyp_op_pack_weight(w, N, swiglu), N, epi, out)
     torch.cuda.synchronize()
     err = np.abs(f64(out) - want) / (np.abs(want) + 1.0)
     assert np.max(err) < tol, (np.max(err), np.unravel_index(np.argmax(err), err.shape))
