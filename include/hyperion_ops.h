@@ -64,8 +64,9 @@ HYP_API int hyp_op_gemm(const void* a, const void* w_packed, int32_t M, int32_t 
                         void* out, int32_t ldo, void* stream);
 
 /* Process-wide tuning switches (measurement aids; the defaults are the measured best).
- *   HYP_TUNE_PDL           value != 0: launch the block's kernels with programmatic dependent launch, so a
- *                          kernel's prologue and weight prefetch may overlap its predecessor's tail
+ *   HYP_TUNE_PDL           which kernels are launched with programmatic dependent launch, so that their
+ *                          prologue and weight prefetch may overlap the predecessor's tail: 0 none, 1 the
+ *                          weight-streaming projections, 2 also the norms between them, 3 every kernel
  *   HYP_TUNE_STREAM_SLOTS  ring slots per warp of the weight-streaming kernel, 1..8 (0 = built-in choice)
  * Affects launches made after the call; decode graphs already captured keep their setting. */
 enum { HYP_TUNE_PDL = 0, HYP_TUNE_STREAM_SLOTS = 1 };

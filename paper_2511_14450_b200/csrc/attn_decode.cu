@@ -71,8 +71,10 @@ attn_decode_partial_kernel(const __half* __restrict__ qkv, const __half* __restr
       const int kk = ok ? key : t_begin;
       const __half* src =
           kv_layer + (size_t)bt[kk / PT] * page_elems + ((size_t)kvh * PT + (kk % PT)) * D + c * 8;
-      cp_async16(k_tile(buf) + tile_off<D>(r, c), src, ok);
-      cp_async16(v_tile(buf) + tile_off<D>(r, c), src + v_off, ok);
+      // the cache row is stored with the tile's own chunk permutation (tiles start on page boundaries, so
+      // r & 7 is the token's slot & 7): chunk positions copy one to one
+      cp_async16(k_tile(buf) + r * (D * 2) + c * 16, src, ok);
+      cp_async16(v_tile(buf) + r * (D * 2) + c * 16, src + v_off, ok);
     }
   };
   if (n_tiles > 0) load_tile(0, 0);

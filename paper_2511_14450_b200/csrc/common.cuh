@@ -85,13 +85,14 @@ __device__ __forceinline__ uint32_t pack_f16_sat(float a, float b) {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// Process-wide switch for the launch attribute.
-inline bool& pdl_enabled() {
-  static bool on = true;
-  return on;
+// Process-wide level: a launch site of level L gets the attribute when L <= pdl_level().
+// 0 = nobody, 1 = the weight-streaming projections, 2 = also the norms between them, 3 = every kernel.
+inline int& pdl_level() {
+  static int level = 1;
+  return level;
 }
 
-template <bool OVERLAP = false, typename... KArgs, typename... Args>
+template <int OVERLAP = 3, typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
                               Args&&... args) {
   cudaLaunchConfig_t cfg = {};
@@ -103,7 +104,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = (OVERLAP && pdl_enabled()) ? 1 : 0;
+  cfg.numAttrs = (OVERLAP <= pdl_level()) ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
@@ -130,7 +131,11 @@ struct ModelDims {
   float eps, theta;
 };
 
-// KV pool of ONE layer: [n_pages][2 (K,V)][Hkv][page_tokens][D] fp16
+// KV pool of ONE layer: [n_pages][2 (K,V)][Hkv][page_tokens][D] fp16.  Within a token's row the 16-byte chunk c
+// (elements 8c .. 8c+7) is stored at chunk position c ^ (slot & 7), slot = the token's index in its page: a page's
+// 16 rows of one head (contiguous) then land in shared memory, by one bulk copy, already in the layout ldmatrix
+// reads without bank conflicts.
+__host__ __device__ __forceinline__ int kv_chunk_pos(int c, int slot) { return c ^ (slot & 7); }
 __host__ __device__ __forceinline__ size_t kv_page_elems(int Hkv, int page_tokens, int D) {
   return (size_t)2 * Hkv * page_tokens * D;
 }
@@ -164,5 +169,12 @@ size_t attn_decode_scratch_bytes(int max_seqs, int Hq, int D, int max_splits);
 int attn_decode_splits(int n_seqs, int Hkv, int max_ctx);
 int launch_attn_decode(const __half* q, int q_stride, const __half* kv_layer, __half* attn_out,
                        float* scratch, int n_splits, const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
+
+// decode attention of the stage path, fused with what surrounds it: rotates the new token's q and k (fp32
+// projection output, one row per sequence), appends k, v to the pages, attends over n_splits context slices
+// (a thread-block cluster, n_splits <= 8) and merges them.  `err`: device word set if a bounded wait expires.
+int attn_decode_fused_splits(int n_seqs, int Hkv, int max_ctx);
+int launch_attn_decode_fused(const float* qkv32, int stride, __half* kv_layer, const float2* rope_table, __half* attn_out,
+                             int n_splits, int slots, int* err, const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
 
 }  // namespace hyp

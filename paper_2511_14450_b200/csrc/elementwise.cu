@@ -99,9 +99,9 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16*
 int launch_rmsnorm(const float* x, const __nv_bfloat16* g, void* h, bool out_f16, int M, int H, float eps,
                    const int32_t* row_index, cudaStream_t st) {
   if (out_f16)
-    HYP_CUDA_TRY(launch_pdl(rmsnorm_kernel<256, true>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
+    HYP_CUDA_TRY(launch_pdl<2>(rmsnorm_kernel<256, true>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
   else
-    HYP_CUDA_TRY(launch_pdl(rmsnorm_kernel<256, false>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
+    HYP_CUDA_TRY(launch_pdl<2>(rmsnorm_kernel<256, false>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
   return 1;
 }
 
@@ -161,9 +161,11 @@ __global__ void rope_kv_write_kernel(const float* __restrict__ qkv, __half* __re
       dst = kv_layer + page_base + (size_t)d.Hkv * d.page_tokens * d.D +
             ((size_t)(head - d.Hq - d.Hkv) * d.page_tokens + slot) * d.D;
     }
-    *reinterpret_cast<uint4*>(dst + i0) =
+    // cache rows keep their 16-byte chunks XOR-permuted by the token's slot (see kv_chunk_pos); q rows are plain
+    const int sw = head < d.Hq ? 0 : (slot & 7);
+    *reinterpret_cast<uint4*>(dst + (((i0 >> 3) ^ sw) << 3)) =
         make_uint4(pack_f16_sat(a[0], a[1]), pack_f16_sat(a[2], a[3]), pack_f16_sat(a[4], a[5]), pack_f16_sat(a[6], a[7]));
-    *reinterpret_cast<uint4*>(dst + d.D / 2 + i0) =
+    *reinterpret_cast<uint4*>(dst + ((((d.D / 2 + i0) >> 3) ^ sw) << 3)) =
         make_uint4(pack_f16_sat(b[0], b[1]), pack_f16_sat(b[2], b[3]), pack_f16_sat(b[4], b[5]), pack_f16_sat(b[6], b[7]));
   }
 }

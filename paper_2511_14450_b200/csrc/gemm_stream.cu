@@ -255,7 +255,7 @@ int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, void* out, int
   if (slots > GS_MAX_SLOTS) slots = GS_MAX_SLOTS;
   while (slots > 2 && GS_WARPS * slots * STAGE_BYTES + 128 > MAX_DYN) --slots;
   const int smem = GS_WARPS * slots * STAGE_BYTES + 128;
-  HYP_CUDA_TRY(launch_pdl<true>(gemm_stream_kernel<NB, EPI, TILES, F16>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
+  HYP_CUDA_TRY(launch_pdl<1>(gemm_stream_kernel<NB, EPI, TILES, F16>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
                           (const uint8_t*)w.packed, (const uint16_t*)act.ptr, act.K, act.K, N, w.KBp, w.N16p, M, out, ldo,
                           slots, tc_err_flag_ptr()));
   return 1;

@@ -54,7 +54,10 @@ extern "C" int hyp_op_pack_weight(const void* w, int32_t N, int32_t K, int32_t s
 
 extern "C" int hyp_tune(int32_t key, int32_t value) {
   switch (key) {
-    case HYP_TUNE_PDL: pdl_enabled() = value != 0; return HYP_OK;
+    case HYP_TUNE_PDL:
+      if (value < 0 || value > 3) return HYP_EINVAL;
+      pdl_level() = value;
+      return HYP_OK;
     case HYP_TUNE_STREAM_SLOTS:
       if (value < 0 || value > 8) return HYP_EINVAL;
       gemm_stream_slots_override() = value;

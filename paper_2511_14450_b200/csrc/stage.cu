@@ -57,8 +57,7 @@ struct hyp_stage {
   __half* q16 = nullptr;              // rotated queries
   __half *h = nullptr, *attn = nullptr, *u = nullptr;  // projection inputs (fp16)
   TcAct tc_h, tc_attn, tc_u;
-  float* attn_scratch = nullptr;
-  int max_splits = 32;
+  int max_splits = 8;
   float2* rope_table = nullptr;
   size_t workspace_bytes = 0;
   // metadata staging
@@ -293,12 +292,14 @@ int run_blocks(hyp_stage* s, const BatchMeta& bm, bool decode, int n_splits, cud
     HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g1, s->h, true, M, d.H, d.eps, nullptr, st));
     HYP_LAUNCH_T(HYP_K_GEMM_QKV, project(s, s->tc_h, nullptr, d.H, lw.tc_qkv, nullptr, d.qkv_rows, d.H, M,
                                          EPI_STORE_F32, s->qkv32, d.qkv_rows, st));
-    HYP_LAUNCH_T(HYP_K_ROPE, launch_rope_kv_write(s->qkv32, s->q16, kv_layer, s->rope_table, bm, d, st));
-    if (decode)
-      HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_decode(s->q16, d.Hq * d.D, kv_layer, s->attn, s->attn_scratch, n_splits, bm,
-                                                  d, st));
-    else
+    if (decode) {
+      // rotation, cache append, attention and the merge of its splits in one launch
+      HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_decode_fused(s->qkv32, d.qkv_rows, kv_layer, s->rope_table, s->attn, n_splits,
+                                                        2, tc_err_flag_ptr(), bm, d, st));
+    } else {
+      HYP_LAUNCH_T(HYP_K_ROPE, launch_rope_kv_write(s->qkv32, s->q16, kv_layer, s->rope_table, bm, d, st));
       HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_prefill(s->q16, d.Hq * d.D, kv_layer, s->attn, bm, d, st));
+    }
     HYP_LAUNCH_T(HYP_K_GEMM_O, project(s, s->tc_attn, nullptr, d.Hq * d.D, lw.tc_o, nullptr, d.H, d.Hq * d.D, M,
                                        EPI_RESID_F32, s->x, d.H, st));
     HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g2, s->h, true, M, d.H, d.eps, nullptr, st));
@@ -366,8 +367,8 @@ int decode_with_graph(hyp_stage* s, const BatchMeta& bm, int n, int n_splits, co
     if (e2 != cudaSuccess) {
       cudaGetLastError();
       g->exec = nullptr;
-      if (pdl_enabled())
-        pdl_enabled() = false;  // retry on the next step without programmatic launches
+      if (pdl_level() > 0)
+        pdl_level() = 0;  // retry on the next step without programmatic launches
       else
         s->graphs_ok = false;   // this driver cannot capture the sequence: stay on the eager path
       return 1;
@@ -399,7 +400,7 @@ int run_stage(hyp_stage* s, const hyp_batch* b, const void* in, void* out, cudaS
   if (decode) {
     int max_ctx = 1;
     for (int i = 0; i < hb.n; ++i) max_ctx = std::max(max_ctx, b->ctx_lens[i] + 1);
-    n_splits = std::min(s->max_splits, attn_decode_splits(hb.n, d.Hkv, max_ctx));
+    n_splits = std::min(s->max_splits, attn_decode_fused_splits(hb.n, d.Hkv, max_ctx));
   }
   const bool all = (b->flags & HYP_BATCH_ALL_LOGITS) != 0 || decode;
   rc = 1;
@@ -495,7 +496,7 @@ extern "C" void hyp_stage_destroy(hyp_stage* s) {
   cudaFree(s->embed); cudaFree(s->gf); cudaFree(s->wlm); cudaFree(s->kv_pool);
   cudaFree(s->x); cudaFree(s->h); cudaFree(s->qkv32); cudaFree(s->q16);
   cudaFree(s->attn); cudaFree(s->u);
-  cudaFree(s->attn_scratch); cudaFree(s->rope_table); cudaFree(s->meta_dev);
+  cudaFree(s->rope_table); cudaFree(s->meta_dev);
   cudaFree(s->io_in); cudaFree(s->io_out);
   for (int i = 0; i < META_RING; ++i) {
     if (s->meta_host[i]) cudaFreeHost(s->meta_host[i]);
@@ -575,11 +576,7 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
   TRY_CUDA(cudaMemset(s->h, 0, rows_pad * d.H * sizeof(__half)));
   TRY_CUDA(cudaMemset(s->attn, 0, rows_pad * d.Hq * d.D * sizeof(__half)));
   TRY_CUDA(cudaMemset(s->u, 0, rows_pad * d.F * sizeof(__half)));
-  const size_t scratch_bytes =
-      attn_decode_scratch_bytes(std::min(c.max_seqs, HYP_MAX_DECODE_BATCH), d.Hq, d.D, s->max_splits);
-  TRY(dev_alloc(&s->attn_scratch, scratch_bytes / sizeof(float)));
-  s->workspace_bytes = rows_pad * ((size_t)d.H * 8 + (size_t)d.qkv_rows * 4 + ((size_t)2 * d.Hq * d.D + d.F) * 2) +
-                       scratch_bytes;
+  s->workspace_bytes = rows_pad * ((size_t)d.H * 8 + (size_t)d.qkv_rows * 4 + ((size_t)2 * d.Hq * d.D + d.F) * 2);
   // rotary table: cos/sin of pos * theta^(-2i/D), angles evaluated in double on the host
   {
     const int half = d.D / 2;
@@ -770,7 +767,7 @@ extern "C" int hyp_stage_profile(hyp_stage* s, int32_t mode, int32_t batch, int3
   rc = upload_meta(s, hb, st);
   if (rc) return rc;
   const BatchMeta bm = device_meta(s, hb);
-  const int n_splits = decode ? std::min(s->max_splits, attn_decode_splits(batch, s->dims.Hkv, total)) : 1;
+  const int n_splits = decode ? std::min(s->max_splits, attn_decode_fused_splits(batch, s->dims.Hkv, total)) : 1;
 
   std::vector<cudaEvent_t> ev((size_t)(s->L + 1) * iters, nullptr);
   for (auto& e : ev) HYP_CUDA_TRY(cudaEventCreate(&e));

@@ -63,6 +63,17 @@ def test_gemm_all_epilogues(M, N, K, epi):
     assert np.max(err) < tol, (np.max(err), np.unravel_index(np.argmax(err), err.shape))
 
 
+def kv_rows(x):
+    """Token rows [slots, Hkv, D] -> the cache's row layout [Hkv, slots, D]: 16-byte chunk c of the token in
+    page slot s sits at chunk position c ^ (s & 7)."""
+    slots, Hkv, D = x.shape
+    c = torch.arange(D // 8, device=x.device)
+    src = (c[None, :] ^ (torch.arange(slots, device=x.device)[:, None] & 7))          # [slots, chunks]
+    xc = x.reshape(slots, Hkv, D // 8, 8)
+    out = torch.gather(xc, 2, src[:, None, :, None].expand(slots, Hkv, D // 8, 8))
+    return out.reshape(slots, Hkv, D).permute(1, 0, 2)
+
+
 def build_cache(seq_lens, Hkv, D, seed):
     """Random rotated keys / values (fp16) for each sequence, scattered into a shuffled page pool."""
     n = len(seq_lens)
@@ -80,8 +91,8 @@ def build_cache(seq_lens, Hkv, D, seed):
             page = int(perm[i * mpps + p])
             table[i, p] = page
             t0, t1 = 16 * p, min(L, 16 * p + 16)
-            pool[page, 0, :, :t1 - t0] = k[t0:t1].permute(1, 0, 2)
-            pool[page, 1, :, :t1 - t0] = v[t0:t1].permute(1, 0, 2)
+            pool[page, 0, :, :t1 - t0] = kv_rows(k[t0:t1])
+            pool[page, 1, :, :t1 - t0] = kv_rows(v[t0:t1])
     return pool, table.cuda(), ks, vs
 
 
