@@ -68,8 +68,13 @@ HYP_API int hyp_op_gemm(const void* a, const void* w_packed, int32_t M, int32_t 
  *                          prologue and weight prefetch may overlap the predecessor's tail: 0 none, 1 the
  *                          weight-streaming projections, 2 also the norms between them, 3 every kernel
  *   HYP_TUNE_STREAM_SLOTS  ring slots per warp of the weight-streaming kernel, 1..8 (0 = built-in choice)
+ *   HYP_TUNE_ATTN_SPLITS   context splits (cluster size) of the stage's decode attention, 1..8 (0 = built-in)
+ *   HYP_TUNE_ATTN_SLOTS    ring slots per warp of that kernel, 2..4 (0 = built-in)
+ *   HYP_TUNE_STREAM_ROTATION  CTA b of the weight-streaming kernel starts its K walk at copy (b * value) mod copies
+ *                          (0 = all CTAs walk K in the same order)
  * Affects launches made after the call; decode graphs already captured keep their setting. */
-enum { HYP_TUNE_PDL = 0, HYP_TUNE_STREAM_SLOTS = 1 };
+enum { HYP_TUNE_PDL = 0, HYP_TUNE_STREAM_SLOTS = 1, HYP_TUNE_ATTN_SPLITS = 2, HYP_TUNE_ATTN_SLOTS = 3,
+       HYP_TUNE_STREAM_ROTATION = 4 };
 HYP_API int hyp_tune(int32_t key, int32_t value);
 
 /* Number of context splits hyp_op_attn_decode would pick for this batch, and the scratch bytes

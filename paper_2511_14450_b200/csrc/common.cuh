@@ -86,9 +86,10 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Process-wide level: a launch site of level L gets the attribute when L <= pdl_level().
-// 0 = nobody, 1 = the weight-streaming projections, 2 = also the norms between them, 3 = every kernel.
+// 0 = nobody, 1 = the weight-streaming projections, 2 = also the norms between them (the default: measured best on the
+// 14-block decode stage), 3 = every kernel.
 inline int& pdl_level() {
-  static int level = 1;
+  static int level = 2;
   return level;
 }
 
@@ -155,7 +156,8 @@ int launch_embed(const int32_t* ids, const __nv_bfloat16* E, float* x, int M, in
 int launch_copy_f32(const float* src, float* dst, size_t n, cudaStream_t st);
 // h = norm(x) as bf16, or as fp16 when out_f16 (h then points to __half storage)
 int launch_rmsnorm(const float* x, const __nv_bfloat16* g, void* h, bool out_f16, int M, int H, float eps,
-                   const int32_t* row_index /* optional gather of rows, may be null */, cudaStream_t st);
+                   const int32_t* row_index /* optional gather of rows, may be null */, cudaStream_t st,
+                   bool gains_are_constant = false /* true: g is a loaded weight, never a predecessor's output */);
 // dst[i] = fp16(src[i]) (exact for |x| >= 2^-17, saturating at +-65504)
 int launch_bf16_to_f16(const __nv_bfloat16* src, __half* dst, size_t n, cudaStream_t st);
 // rotate q, k of every row (fp32 in), write q as fp16 [M, Hq*D] and append k, v as fp16 to the pages
@@ -174,6 +176,8 @@ int launch_attn_decode(const __half* q, int q_stride, const __half* kv_layer, __
 // projection output, one row per sequence), appends k, v to the pages, attends over n_splits context slices
 // (a thread-block cluster, n_splits <= 8) and merges them.  `err`: device word set if a bounded wait expires.
 int attn_decode_fused_splits(int n_seqs, int Hkv, int max_ctx);
+int& attn_fused_splits_override();  // 0 = built-in choice
+int& attn_fused_slots_override();   // 0 = built-in choice
 int launch_attn_decode_fused(const float* qkv32, int stride, __half* kv_layer, const float2* rope_table, __half* attn_out,
                              int n_splits, int slots, int* err, const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
 

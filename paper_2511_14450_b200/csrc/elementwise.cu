@@ -52,12 +52,20 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16*
                                int H, float eps, const int32_t* __restrict__ row_index) {
   constexpr int CACHE = 8;  // float4 per thread kept in registers: rows up to THREADS * 32 wide are read once
   __shared__ float red[THREADS / 32];
+  const int r = blockIdx.x;
+  const int n4 = H / 4;
+  // the gains are weights: fetch them (a DRAM miss, they are read once per step) while the predecessor still runs
+  const uint2* gr = reinterpret_cast<const uint2*>(g);
+  uint2 gk[CACHE];
+#pragma unroll
+  for (int c = 0; c < CACHE; ++c) {
+    const int i = threadIdx.x + c * THREADS;
+    gk[c] = i < n4 ? gr[i] : make_uint2(0u, 0u);
+  }
   pdl_trigger();
   pdl_wait();
-  const int r = blockIdx.x;
   const int row = row_index ? row_index[r] : r;
   const float4* xr = reinterpret_cast<const float4*>(x + (size_t)row * H);
-  const int n4 = H / 4;
   float4 keep[CACHE];
   float ss = 0.f;
 #pragma unroll
@@ -77,10 +85,8 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16*
 #pragma unroll
   for (int w = 0; w < THREADS / 32; ++w) tot += red[w];
   const float rstd = rsqrtf(tot / (float)H + eps);
-  const uint2* gr = reinterpret_cast<const uint2*>(g);
   uint2* hr = reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(h) + (size_t)r * H);
-  auto emit = [&](int i, const float4& v) {
-    const uint2 gg = gr[i];
+  auto emit = [&](int i, const float4& v, const uint2 gg) {
     const float y0 = v.x * rstd * bf16_lo(gg.x), y1 = v.y * rstd * bf16_hi(gg.x);
     const float y2 = v.z * rstd * bf16_lo(gg.y), y3 = v.w * rstd * bf16_hi(gg.y);
     uint2 o;
@@ -91,17 +97,26 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16*
 #pragma unroll
   for (int c = 0; c < CACHE; ++c) {
     const int i = threadIdx.x + c * THREADS;
-    if (i < n4) emit(i, keep[c]);
+    if (i < n4) emit(i, keep[c], gk[c]);
   }
-  for (int i = threadIdx.x + CACHE * THREADS; i < n4; i += THREADS) emit(i, xr[i]);
+  for (int i = threadIdx.x + CACHE * THREADS; i < n4; i += THREADS) emit(i, xr[i], gr[i]);
 }
 
 int launch_rmsnorm(const float* x, const __nv_bfloat16* g, void* h, bool out_f16, int M, int H, float eps,
-                   const int32_t* row_index, cudaStream_t st) {
-  if (out_f16)
-    HYP_CUDA_TRY(launch_pdl<2>(rmsnorm_kernel<256, true>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
-  else
-    HYP_CUDA_TRY(launch_pdl<2>(rmsnorm_kernel<256, false>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
+                   const int32_t* row_index, cudaStream_t st, bool gains_are_constant) {
+  // the kernel reads g before it waits for its predecessor: only launched early when g cannot be that
+  // predecessor's output
+  if (gains_are_constant) {
+    if (out_f16)
+      HYP_CUDA_TRY(launch_pdl<2>(rmsnorm_kernel<256, true>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
+    else
+      HYP_CUDA_TRY(launch_pdl<2>(rmsnorm_kernel<256, false>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
+  } else {
+    if (out_f16)
+      HYP_CUDA_TRY(launch_pdl<4>(rmsnorm_kernel<256, true>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
+    else
+      HYP_CUDA_TRY(launch_pdl<4>(rmsnorm_kernel<256, false>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
+  }
   return 1;
 }
 

@@ -26,6 +26,10 @@ int& gemm_stream_slots_override() {
   static int v = 0;
   return v;
 }
+int& gemm_stream_rotation() {
+  static int v = 13;
+  return v;
+}
 
 namespace {
 
@@ -55,7 +59,7 @@ __device__ __forceinline__ uint4 ldg_act(const void* p) {
 template <int NB, int EPI, int TILES, bool F16>
 __global__ void __launch_bounds__(GS_THREADS)
 gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ act, int lda, int K, int N, int KBp,
-                   int tile1_off, int M, void* __restrict__ out, int ldo, int S, int* __restrict__ err) {
+                   int tile1_off, int M, void* __restrict__ out, int ldo, int S, int rot_mul, int* __restrict__ err) {
   constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
   static_assert(!SWIGLU || TILES == 2, "SwiGLU pairs a gate strip with an up strip");
   constexpr int OUT_COLS = (TILES == 2 && !SWIGLU) ? 32 : 16;
@@ -80,7 +84,7 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
 
   // CTAs walk K from staggered starting points (a fixed rotation per CTA, so the summation order stays
   // reproducible): otherwise every resident CTA would ask for the same activation lines at the same moment.
-  const int rot = (int)((blockIdx.x * 13u) % (unsigned)NCH);
+  const int rot = (int)((blockIdx.x * (unsigned)rot_mul) % (unsigned)NCH);
   auto actual = [&](int ch_logical) {
     const int ch = ch_logical + rot;
     return ch >= NCH ? ch - NCH : ch;
@@ -219,7 +223,7 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
 }
 
 template <int NB, int EPI, int TILES, bool F16>
-int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, void* out, int ldo, cudaStream_t st) {
+int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, void* out, int ldo, cudaStream_t st, bool early) {
   static bool configured = false;
   static int num_sms = 0, smem_per_sm = 0;
   constexpr int STAGE_BYTES = TILES * W_CHUNK_BYTES;
@@ -255,49 +259,56 @@ int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, void* out, int
   if (slots > GS_MAX_SLOTS) slots = GS_MAX_SLOTS;
   while (slots > 2 && GS_WARPS * slots * STAGE_BYTES + 128 > MAX_DYN) --slots;
   const int smem = GS_WARPS * slots * STAGE_BYTES + 128;
-  HYP_CUDA_TRY(launch_pdl<1>(gemm_stream_kernel<NB, EPI, TILES, F16>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
-                          (const uint8_t*)w.packed, (const uint16_t*)act.ptr, act.K, act.K, N, w.KBp, w.N16p, M, out, ldo,
-                          slots, tc_err_flag_ptr()));
+  // the kernel fetches weights before it waits for its predecessor: launched early only when the weights cannot
+  // be that predecessor's output
+  if (early)
+    HYP_CUDA_TRY(launch_pdl<1>(gemm_stream_kernel<NB, EPI, TILES, F16>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
+                               (const uint8_t*)w.packed, (const uint16_t*)act.ptr, act.K, act.K, N, w.KBp, w.N16p, M, out,
+                               ldo, slots, gemm_stream_rotation(), tc_err_flag_ptr()));
+  else
+    HYP_CUDA_TRY(launch_pdl<4>(gemm_stream_kernel<NB, EPI, TILES, F16>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
+                               (const uint8_t*)w.packed, (const uint16_t*)act.ptr, act.K, act.K, N, w.KBp, w.N16p, M, out,
+                               ldo, slots, gemm_stream_rotation(), tc_err_flag_ptr()));
   return 1;
 }
 
 template <int NB, bool F16>
-int launch_nb(const TcAct& act, const TcWeight& w, int M, int N, int epi, void* out, int ldo, cudaStream_t st) {
+int launch_nb(const TcAct& act, const TcWeight& w, int M, int N, int epi, void* out, int ldo, cudaStream_t st, bool early) {
   const bool wide = N > 8192;  // many rows: 32 columns per CTA keep the CTA count down
   switch (epi) {
     case EPI_STORE_BF16:
-      return wide ? launch_cfg<NB, EPI_STORE_BF16, 2, F16>(act, w, M, N, out, ldo, st)
-                  : launch_cfg<NB, EPI_STORE_BF16, 1, F16>(act, w, M, N, out, ldo, st);
+      return wide ? launch_cfg<NB, EPI_STORE_BF16, 2, F16>(act, w, M, N, out, ldo, st, early)
+                  : launch_cfg<NB, EPI_STORE_BF16, 1, F16>(act, w, M, N, out, ldo, st, early);
     case EPI_RESID_F32:
-      return wide ? launch_cfg<NB, EPI_RESID_F32, 2, F16>(act, w, M, N, out, ldo, st)
-                  : launch_cfg<NB, EPI_RESID_F32, 1, F16>(act, w, M, N, out, ldo, st);
+      return wide ? launch_cfg<NB, EPI_RESID_F32, 2, F16>(act, w, M, N, out, ldo, st, early)
+                  : launch_cfg<NB, EPI_RESID_F32, 1, F16>(act, w, M, N, out, ldo, st, early);
     case EPI_STORE_F32:
-      return wide ? launch_cfg<NB, EPI_STORE_F32, 2, F16>(act, w, M, N, out, ldo, st)
-                  : launch_cfg<NB, EPI_STORE_F32, 1, F16>(act, w, M, N, out, ldo, st);
-    case EPI_SWIGLU_BF16: return launch_cfg<NB, EPI_SWIGLU_BF16, 2, F16>(act, w, M, N, out, ldo, st);
+      return wide ? launch_cfg<NB, EPI_STORE_F32, 2, F16>(act, w, M, N, out, ldo, st, early)
+                  : launch_cfg<NB, EPI_STORE_F32, 1, F16>(act, w, M, N, out, ldo, st, early);
+    case EPI_SWIGLU_BF16: return launch_cfg<NB, EPI_SWIGLU_BF16, 2, F16>(act, w, M, N, out, ldo, st, early);
     default: return HYP_EINVAL;
   }
 }
 
 template <bool F16>
-int launch_type(const TcAct& act, const TcWeight& w, int M, int N, int epi, void* out, int ldo, cudaStream_t st) {
+int launch_type(const TcAct& act, const TcWeight& w, int M, int N, int epi, void* out, int ldo, cudaStream_t st, bool early) {
   switch ((M + 7) / 8) {
-    case 1: return launch_nb<1, F16>(act, w, M, N, epi, out, ldo, st);
-    case 2: return launch_nb<2, F16>(act, w, M, N, epi, out, ldo, st);
-    case 3: return launch_nb<3, F16>(act, w, M, N, epi, out, ldo, st);
-    default: return launch_nb<4, F16>(act, w, M, N, epi, out, ldo, st);
+    case 1: return launch_nb<1, F16>(act, w, M, N, epi, out, ldo, st, early);
+    case 2: return launch_nb<2, F16>(act, w, M, N, epi, out, ldo, st, early);
+    case 3: return launch_nb<3, F16>(act, w, M, N, epi, out, ldo, st, early);
+    default: return launch_nb<4, F16>(act, w, M, N, epi, out, ldo, st, early);
   }
 }
 
 }  // namespace
 
 int launch_gemm_stream(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
-                       cudaStream_t st) {
+                       cudaStream_t st, bool early) {
   if (M < 1 || M > 32 || N < 1 || K < 8 || act.K != K || w.K != K || !tc_err_flag_ptr()) return HYP_EINVAL;
   if (w.rows != N || w.halves != (epi == EPI_SWIGLU_BF16 ? 2 : 1)) return HYP_EINVAL;
   if (act.f16 != w.f16) return HYP_EINVAL;  // one instruction takes both operands in the same 16-bit type
   if (((uintptr_t)act.ptr & 15) != 0 || (K % 8) != 0) return HYP_EINVAL;  // 128-bit activation loads
-  return act.f16 ? launch_type<true>(act, w, M, N, epi, out, ldo, st) : launch_type<false>(act, w, M, N, epi, out, ldo, st);
+  return act.f16 ? launch_type<true>(act, w, M, N, epi, out, ldo, st, early) : launch_type<false>(act, w, M, N, epi, out, ldo, st, early);
 }
 
 }  // namespace hyp

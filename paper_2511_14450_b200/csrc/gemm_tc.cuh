@@ -53,10 +53,13 @@ int* tc_err_flag_ptr();
 
 // Ring depth override of the weight-streaming kernel (0 = the built-in choice).
 int& gemm_stream_slots_override();
+// Per-CTA stagger of the K walk of the weight-streaming kernel: CTA b starts at copy (b * rotation) mod copies.
+int& gemm_stream_rotation();
 
-// Weight-streaming projection for M <= 32 rows (decode); same contract as launch_gemm_tc.
+// Weight-streaming projection for M <= 32 rows (decode); same contract as launch_gemm_tc.  `early`: the packed
+// weights are long-lived (not written by the kernel launched just before), so the launch may overlap that kernel.
 int launch_gemm_stream(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
-                       cudaStream_t st);
+                       cudaStream_t st, bool early = false);
 
 // out[m, n] (+)= sum_k act[m, k] * w[n, k] for m < M, n < N (SwiGLU: w holds two halves of N rows).
 int launch_gemm_tc(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,

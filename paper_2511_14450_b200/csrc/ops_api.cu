@@ -62,6 +62,18 @@ extern "C" int hyp_tune(int32_t key, int32_t value) {
       if (value < 0 || value > 8) return HYP_EINVAL;
       gemm_stream_slots_override() = value;
       return HYP_OK;
+    case HYP_TUNE_STREAM_ROTATION:
+      if (value < 0 || value > 1024) return HYP_EINVAL;
+      gemm_stream_rotation() = value;
+      return HYP_OK;
+    case HYP_TUNE_ATTN_SPLITS:
+      if (value < 0 || value > 8) return HYP_EINVAL;
+      attn_fused_splits_override() = value;
+      return HYP_OK;
+    case HYP_TUNE_ATTN_SLOTS:
+      if (value < 0 || value > 4) return HYP_EINVAL;
+      attn_fused_slots_override() = value;
+      return HYP_OK;
     default: return HYP_EINVAL;
   }
 }

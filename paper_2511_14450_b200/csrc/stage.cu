@@ -274,7 +274,7 @@ int check_ready(const hyp_stage* s) {
 int project(hyp_stage* s, const TcAct& act, const bf16* a, int lda, const TcWeight& tw, const bf16* w, int N, int K,
             int M, int epi, void* out, int ldo, cudaStream_t st) {
   (void)a; (void)lda; (void)w;
-  if (M <= 32) return launch_gemm_stream(act, tw, M, N, K, epi, out, ldo, st);
+  if (M <= 32) return launch_gemm_stream(act, tw, M, N, K, epi, out, ldo, st, /*early=*/true);
   return launch_gemm_tc(act, tw, M, N, K, epi, out, ldo, st);
 }
 
@@ -289,7 +289,7 @@ int run_blocks(hyp_stage* s, const BatchMeta& bm, bool decode, int n_splits, cud
     __half* kv_layer = s->kv_pool + (size_t)li * s->kv_layer_elems;
     // every projection runs fp16 x fp16 -> fp32: with bf16 inputs the rounding of the activations alone
     // (8 mantissa bits, amplified from block to block) puts the 40-block logits outside the tolerance
-    HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g1, s->h, true, M, d.H, d.eps, nullptr, st));
+    HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g1, s->h, true, M, d.H, d.eps, nullptr, st, true));
     HYP_LAUNCH_T(HYP_K_GEMM_QKV, project(s, s->tc_h, nullptr, d.H, lw.tc_qkv, nullptr, d.qkv_rows, d.H, M,
                                          EPI_STORE_F32, s->qkv32, d.qkv_rows, st));
     if (decode) {
@@ -302,7 +302,7 @@ int run_blocks(hyp_stage* s, const BatchMeta& bm, bool decode, int n_splits, cud
     }
     HYP_LAUNCH_T(HYP_K_GEMM_O, project(s, s->tc_attn, nullptr, d.Hq * d.D, lw.tc_o, nullptr, d.H, d.Hq * d.D, M,
                                        EPI_RESID_F32, s->x, d.H, st));
-    HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g2, s->h, true, M, d.H, d.eps, nullptr, st));
+    HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g2, s->h, true, M, d.H, d.eps, nullptr, st, true));
     HYP_LAUNCH_T(HYP_K_GEMM_GATE_UP, project(s, s->tc_h, nullptr, d.H, lw.tc_gu, nullptr, d.F, d.H, M, EPI_SWIGLU_BF16,
                                              s->u, d.F, st));
     HYP_LAUNCH_T(HYP_K_GEMM_DOWN, project(s, s->tc_u, nullptr, d.F, lw.tc_d, nullptr, d.H, d.F, M, EPI_RESID_F32, s->x,
@@ -325,7 +325,7 @@ int enqueue_stage(hyp_stage* s, const BatchMeta& bm, int n_seqs, bool decode, bo
   if (rc) return rc;
   if (s->last) {
     const int rows = all_rows ? M : n_seqs;
-    HYP_LAUNCH(launch_rmsnorm(s->x, s->gf, s->h, true, rows, d.H, d.eps, all_rows ? nullptr : bm.last_row, st));
+    HYP_LAUNCH(launch_rmsnorm(s->x, s->gf, s->h, true, rows, d.H, d.eps, all_rows ? nullptr : bm.last_row, st, true));
     HYP_LAUNCH_T(HYP_K_LM_HEAD,
                  project(s, s->tc_h, nullptr, d.H, s->tc_lm, nullptr, d.V, d.H, rows, EPI_STORE_F32, out, d.V, st));
   } else {

@@ -268,7 +268,7 @@ def hyp_op_rmsnorm(x, g, out, eps: float, stream=None):
     _check(lib().hyp_op_rmsnorm(_ptr(x), _ptr(g), _ptr(out), M, H, eps, _stream_handle(stream)), "hyp_op_rmsnorm")
 
 
-HYP_TUNE_PDL, HYP_TUNE_STREAM_SLOTS = range(2)
+HYP_TUNE_PDL, HYP_TUNE_STREAM_SLOTS, HYP_TUNE_ATTN_SPLITS, HYP_TUNE_ATTN_SLOTS, HYP_TUNE_STREAM_ROTATION = range(5)
 
 
 def hyp_tune(key: int, value: int):
