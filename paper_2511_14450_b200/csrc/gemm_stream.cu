@@ -57,7 +57,7 @@ __device__ __forceinline__ uint4 ldg_act(const void* p) {
 // TILES = 1: 16 output columns per CTA (one strip).  TILES = 2: 32 adjacent columns (strips 2b, 2b + 1), or (SwiGLU)
 // gate strip b and the matching up strip tile1_off + b.  S = ring slots per warp; a slot holds TILES copies.
 template <int NB, int EPI, int TILES, bool F16>
-__global__ void __launch_bounds__(GS_THREADS)
+__global__ void __launch_bounds__(GS_THREADS, 3)
 gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ act, int lda, int K, int N, int KBp,
                    int tile1_off, int M, void* __restrict__ out, int ldo, int S, int rot_mul, int* __restrict__ err) {
   constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;

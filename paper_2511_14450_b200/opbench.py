@@ -4,6 +4,7 @@
     python -m paper_2511_14450_b200.opbench attn_decode --batch 8 --ctx 1024
     python -m paper_2511_14450_b200.opbench attn_prefill --batch 1 --ctx 512
     python -m paper_2511_14450_b200.opbench layer_gemms --M 512
+    python -m paper_2511_14450_b200.opbench decode_stage --layers 2 --batch 8 --ctx 1024
 
 Times with CUDA events after warm-up; weights / KV pools are rotated so that no launch finds its
 operands in L2.  Prints one JSON line per case.
@@ -88,9 +89,45 @@ def layer_gemms(M):
     return res + [{"op": "layer_gemms", "M": M, "us": us, "tflops": flops / us / 1e6}]
 
 
+def decode_stage(layers, batch, ctx, iters=20):
+    """Decode steps of a short stage of Phi-3-medium-shaped blocks (the library's own kernel sequence, graph
+    replay): a small stand-in for the benchmark's 14-block stage, e.g. for profiling one of its kernels."""
+    from paper_2511_14450_b200 import inputs
+    sh = inputs.phi3_medium_shape()
+    chunk = min(ctx, 2048)
+    st = hyp.Stage(sh, 0, layers, max_seqs=batch, max_ctx=ctx + iters + 16, max_tokens=chunk)
+    for layer in range(layers):
+        st.load_layer(layer, inputs.layer_weights(sh, layer, device="cuda"))
+        torch.cuda.synchronize()
+    st.load_embed(inputs.embed_weights(sh, device="cuda"))
+    hidden = torch.empty(chunk, sh.hidden, dtype=torch.float32, device="cuda")
+    for b in range(batch):
+        done = 0
+        while done < ctx:
+            n = min(chunk, ctx - done)
+            st.prefill([b], [n], [done], inputs.token_ids(inputs.SEED_PROMPTS, b, n, sh.vocab, device="cuda"), hidden)
+            done += n
+    out = torch.empty(batch, sh.hidden, dtype=torch.float32, device="cuda")
+    ids = inputs.token_ids(inputs.SEED_FORCED, 0, batch, sh.vocab, device="cuda")
+    slots = list(range(batch))
+    pos = [ctx]
+
+    def step(_):
+        st.decode(slots, [pos[0]] * batch, ids, out)
+        pos[0] += 1
+
+    ms = _time(step, iters, warmup=4)
+    st.close()
+    kv = layers * batch * (ctx + iters // 2) * 2 * sh.n_kv_heads * sh.head_dim * 2
+    return {"op": "decode_stage", "layers": layers, "batch": batch, "ctx": ctx, "us_per_step": ms * 1e3,
+            "us_per_layer": ms * 1e3 / layers,
+            "gbs": (layers * sh.layer_linear_params * 2 + kv) / ms / 1e6}
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["gemm", "attn_decode", "attn_prefill", "layer_gemms"])
+    ap.add_argument("op", choices=["gemm", "attn_decode", "attn_prefill", "layer_gemms", "decode_stage"])
+    ap.add_argument("--layers", type=int, default=2)
     ap.add_argument("--M", type=int, default=8)
     ap.add_argument("--N", type=int, default=17920)
     ap.add_argument("--K", type=int, default=5120)
@@ -106,6 +143,8 @@ def main():
         out = [attn_decode(a.batch, a.ctx, iters=a.iters, splits=a.splits)]
     elif a.op == "attn_prefill":
         out = [attn_prefill(a.batch, a.ctx, iters=a.iters)]
+    elif a.op == "decode_stage":
+        out = [decode_stage(a.layers, a.batch, a.ctx, iters=a.iters)]
     else:
         out = layer_gemms(a.M)
     for r in out:
