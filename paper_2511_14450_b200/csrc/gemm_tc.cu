@@ -79,18 +79,20 @@ struct Segments {
   long u, u_end;  // stream-K: position in the column list
   int tile, n_tiles, stride, KB, tiles_m, tiles_n, team, member;
   bool streamk;
-  __device__ Segments(bool sk, int tiles_m_, int tiles_n_, int KB_, int team_)
+  // `unit` of `n_units`: the CTA's index in the grid, or the CTA pair's index for the two-CTA kernel (whose
+  // M-tiles are 256 rows high)
+  __device__ Segments(bool sk, int tiles_m_, int tiles_n_, int KB_, int team_, int unit, int n_units)
       : n_tiles(tiles_m_ * tiles_n_), KB(KB_), tiles_m(tiles_m_), tiles_n(tiles_n_), team(team_), streamk(sk) {
     if (sk) {
-      const int n_teams = gridDim.x / team_;
-      const int my_team = blockIdx.x / team_;
-      member = blockIdx.x % team_;
+      const int n_teams = n_units / team_;
+      const int my_team = unit / team_;
+      member = unit % team_;
       const long total = (long)(tiles_m_ / team_) * tiles_n_ * KB_;
       u = total * my_team / n_teams;
       u_end = total * (my_team + 1) / n_teams;
     } else {
-      tile = blockIdx.x;
-      stride = gridDim.x;
+      tile = unit;
+      stride = n_units;
     }
   }
   __device__ bool next(int& t, int& kb0, int& kb1) {
@@ -231,7 +233,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       uint32_t phase = 0;
       bool ok = true;
       pdl_wait();  // the activation operand is the predecessor's output
-      Segments seg(STREAMK, tiles_m, tiles_n, KB, team);
+      Segments seg(STREAMK, tiles_m, tiles_n, KB, team, (int)blockIdx.x, (int)gridDim.x);
       int tile, kb0, kb1;
       while (ok && seg.next(tile, kb0, kb1)) {
         const int m0 = (tile % tiles_m) * BM;
@@ -259,7 +261,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      Segments seg(STREAMK, tiles_m, tiles_n, KB, team);
+      Segments seg(STREAMK, tiles_m, tiles_n, KB, team, (int)blockIdx.x, (int)gridDim.x);
       int tile, kb0, kb1;
       while (ok && seg.next(tile, kb0, kb1)) {
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag)) { ok = false; break; }
@@ -294,7 +296,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    Segments seg(STREAMK, tiles_m, tiles_n, KB, team);
+    Segments seg(STREAMK, tiles_m, tiles_n, KB, team, (int)blockIdx.x, (int)gridDim.x);
     int tile, kb0, kb1;
     while (ok && seg.next(tile, kb0, kb1)) {
       const int m0 = (tile % tiles_m) * BM;
@@ -397,8 +399,9 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uin
 template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int M, int N, int K,
-                int up_tile0, void* __restrict__ out, int ldo, uint32_t idesc, int* __restrict__ err) {
+                int up_tile0, void* __restrict__ out, int ldo, int team, uint32_t idesc, int* __restrict__ err) {
   constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
+  const bool STREAMK = EPI == EPI_RESID_F32 && team > 0;
   constexpr int BN_OUT = SWIGLU ? BN / 2 : BN;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -450,12 +453,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+      Segments seg(STREAMK, pairs_m, tiles_n, KB, team, pair, n_pairs);
+      int tile, kb0, kb1;
+      while (ok && seg.next(tile, kb0, kb1)) {
         const int m0 = (tile % pairs_m) * (2 * BM) + (int)rank * BM;
         const int n0 = (tile / pairs_m) * BN_OUT;
         // this CTA's half of the weight tile, as an index of 16-row packed tiles
         const int tb = SWIGLU ? (int)rank * up_tile0 + (n0 >> 4) : (n0 >> 4) + (int)rank * 8;
-        for (int kb = 0; kb < KB; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) { ok = false; break; }
           const uint32_t sa = base + stage * STAGE2_BYTES, sb = sa + A_BYTES;
           const uint32_t lead_full = mapa_rank(full_bar(stage), 0);
@@ -476,11 +481,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+      Segments seg(STREAMK, pairs_m, tiles_n, KB, team, pair, n_pairs);
+      int tile, kb0, kb1;
+      while (ok && seg.next(tile, kb0, kb1)) {
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = 0; kb < KB; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = base + stage * STAGE2_BYTES, sb = sa + A_BYTES;
@@ -488,7 +495,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k)
             tc_mma_pair(d_tmem, da + (uint64_t)(k * UMMA_K * 2 / 16), db + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
-                        (kb > 0 || k > 0) ? 1u : 0u);
+                        (kb > kb0 || k > 0) ? 1u : 0u);
           tc_commit_pair(empty_bar(stage));
           if (++stage == STAGES2) { stage = 0; phase ^= 1; }
         }
@@ -509,9 +516,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+    Segments seg(STREAMK, pairs_m, tiles_n, KB, team, pair, n_pairs);
+    int tile, kb0, kb1;
+    while (ok && seg.next(tile, kb0, kb1)) {
       const int m0 = (tile % pairs_m) * (2 * BM) + (int)rank * BM;
       const int n0 = (tile / pairs_m) * BN_OUT;
+      const bool partial = kb0 != 0 || kb1 != KB;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int row = m0 + 32 * q + lane;
@@ -523,7 +533,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         tmem_ld16(t0 + c, v);
         if (SWIGLU) tmem_ld16(t0 + BN / 2 + c, v2);
         tmem_ld_wait();
-        if (row < M) epilogue_chunk<EPI>(v, v2, out, ldo, row, n0 + c, N, false, idesc == IDESC2_F16);
+        if (row < M) epilogue_chunk<EPI>(v, v2, out, ldo, row, n0 + c, N, partial, idesc == IDESC2_F16);
       }
       tc_fence_before();
       mbar_arrive_cluster(mapa_rank(tempty_bar(acc), 0));
@@ -590,11 +600,30 @@ int launch_pair(const TcAct& act, const TcWeight& w, int M, int N, int K, void* 
     configured = true;
   }
   constexpr int BN_OUT = EPI == EPI_SWIGLU_BF16 ? BN / 2 : BN;
-  const long tiles = (long)((M + 2 * BM - 1) / (2 * BM)) * ((N + BN_OUT - 1) / BN_OUT);
+  const int pairs_m = (M + 2 * BM - 1) / (2 * BM), tiles_n = (N + BN_OUT - 1) / BN_OUT;
+  const long tiles = (long)pairs_m * tiles_n;
   long pairs = num_sms / 2;
-  if (tiles < pairs) pairs = tiles;
+  int team = 0;  // 0 = whole tiles per CTA pair
+  if (EPI == EPI_RESID_F32) {
+    // stream-K over CTA pairs: teams of `team` pairs (a divisor of the 256-row M-tiles) share the weight k-blocks
+    // they walk; every team gets the same number of k-blocks
+    double best = -1.0;
+    team = 1;
+    for (int ts = 1; ts <= pairs_m && ts <= pairs; ++ts) {
+      if (pairs_m % ts) continue;
+      const long teams = pairs / ts;
+      const double score = (double)(teams * ts) / (double)pairs + 0.003 * ts;
+      if (score > best) { best = score; team = ts; }
+    }
+    long teams = pairs / team;
+    const long cols = (long)(pairs_m / team) * tiles_n * ((K + BK - 1) / BK);
+    if (teams > cols) teams = cols;
+    pairs = teams * team;
+  } else if (tiles < pairs) {
+    pairs = tiles;
+  }
   HYP_CUDA_TRY(launch_pdl(gemm_tc2_kernel<EPI>, dim3((unsigned)(2 * pairs)), dim3(TC_THREADS), (size_t)SMEM2_BYTES, st, act.map,
-                          w.map, M, N, K, w.N16p, out, ldo, act.f16 ? IDESC2_F16 : IDESC2_BF16, g_err_flag));
+                          w.map, M, N, K, w.N16p, out, ldo, team, act.f16 ? IDESC2_F16 : IDESC2_BF16, g_err_flag));
   return 1;
 }
 
@@ -611,7 +640,9 @@ int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
   }
   constexpr int BN_OUT = EPI == EPI_SWIGLU_BF16 ? BN / 2 : BN;
   const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN_OUT - 1) / BN_OUT;
-  if (EPI != EPI_RESID_F32 && tiles_m >= 2) return launch_pair<EPI>(act, w, M, N, K, out, ldo, st, num_sms);
+  // two-CTA tiles (a third less shared-memory fill per flop) from 129 rows on; the residual epilogue up to 4096 rows
+  // (stream-K), beyond that whole one-CTA tiles balance by themselves
+  if (tiles_m >= 2 && (EPI != EPI_RESID_F32 || tiles_m <= 32)) return launch_pair<EPI>(act, w, M, N, K, out, ldo, st, num_sms);
   int grid, team = 0;  // team 0 = whole tiles per CTA
   if (EPI == EPI_RESID_F32 && tiles_m <= 16) {
     // stream-K (up to 2048 rows; beyond that whole tiles already balance and reuse A better): pick the team size (a divisor of tiles_m) that keeps most SMs busy, larger teams preferred
