@@ -24,12 +24,14 @@
  *    hyp_strerror are pure host functions, thread-safe, and never touch a GPU.
  *  - Activations crossing a stage boundary are fp32, row-major [M, hidden], rows packed in batch
  *    order (all rows of sequence 0, then sequence 1, ...).
- *  - Precision.  The residual stream, all accumulation, softmax and norms are fp32.  The O, gate/up,
- *    down and LM-head projections take bf16 inputs.  The q/k/v projection takes fp16 inputs and writes
- *    fp32; q, k are rotated in fp32 and q, k, v rounded once to fp16; the KV cache and the softmax
- *    weights are fp16 (values saturate at +-65504).  With bf16 there instead, the softmax weights alone
- *    carry ~0.5 % error and per-step logits of the 5120-wide model miss the 5e-2 tolerance.
- *  - Prefill rows: the residual projections split K across CTAs for row counts up to 2048 and add
+ *  - Precision.  The residual stream, all accumulation, softmax and norms are fp32.  Every projection
+ *    (q/k/v, O, gate/up, down, LM head) multiplies fp16 activations with weights held as fp16 (the bf16
+ *    values converted once at load: exact for |w| >= 2^-17, else off by < 3e-8) into fp32.  The q/k/v
+ *    projection writes fp32; q, k are rotated in fp32 and q, k, v rounded once to fp16; the KV cache and
+ *    the softmax weights are fp16 (values saturate at +-65504).  With bf16 activations instead, their
+ *    8 mantissa bits alone put the per-step logits of the 5120-wide 40-block model outside the 5e-2
+ *    tolerance.
+ *  - Prefill rows: the residual projections split K across CTAs for row counts up to 4096 and add
  *    partial sums with floating-point atomics, so the last bits of a prefill result may differ from
  *    run to run; decode is bit-reproducible.
  */
@@ -85,11 +87,12 @@ typedef struct {
   int32_t kv_pages;       /* pages in the pool; 0 = max_seqs * ceil(max_ctx / 16)                  */
 } hyp_cfg;
 
-/* Weight tensor ids for hyp_stage_load.  Every matrix is bf16, row-major [out, in] (y = x W^T). */
+/* Weight tensor ids for hyp_stage_load.  Every matrix is given as bf16, row-major [out, in] (y = x W^T).
+ * The library keeps its own copy of the projection matrices: fp16 values in a tiled order (16-row x 64-k
+ * tiles, all k-blocks of a 16-row strip contiguous; see hyperion_ops.h), which decode streams strip by
+ * strip and prefill reads tile by tile. */
 enum {
-  HYP_W_QKV = 0,     /* [(Hq + 2 Hkv) D, H]: rows = Q heads, then K heads, then V heads.  The library   */
-                     /* keeps this one as fp16 (exact for |w| >= 2^-17, else off by < 3e-8), because   */
-                     /* q/k/v are projected from fp16 activations: see "Precision" below              */
+  HYP_W_QKV = 0,     /* [(Hq + 2 Hkv) D, H]: rows = Q heads, then K heads, then V heads               */
   HYP_W_O = 1,       /* [H, Hq D]                                                                   */
   HYP_W_GATE_UP = 2, /* [2 F, H]: rows = gate (F) then up (F)                                       */
   HYP_W_DOWN = 3,    /* [H, F]                                                                      */
@@ -120,7 +123,8 @@ typedef struct {
  * Errors: HYP_EINVAL (shape / range), HYP_ENOMEM, HYP_ECUDA. */
 HYP_API int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cfg* cfg, hyp_stage** out);
 
-/* Copy one weight tensor into the stage (device-to-device, asynchronous on `stream`).
+/* Copy one weight tensor into the stage (device-to-device, asynchronous on `stream`; projection
+ * matrices are converted to fp16 and re-tiled on the way).
  * layer: block index in [layer_lo, layer_hi), or -1 / n_layers_total for embed / head tensors.
  * src: DEVICE, bf16, `bytes` must equal the tensor's exact size.  The caller may free src after
  * synchronising the stream.  Errors: HYP_EINVAL, HYP_ECUDA. */

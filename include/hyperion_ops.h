@@ -8,6 +8,9 @@
  * `stream` is a cudaStream_t as void*; calls enqueue and return; status codes as in hyperion.h.
  *
  * KV page pool layout of ONE block (fp16): [n_pages][2 (K then V)][n_kv_heads][16 tokens][head_dim].
+ * Inside a token's head_dim-wide row the 16-byte chunk c (elements 8c .. 8c+7) is stored at chunk position
+ * c ^ (slot & 7), slot = the token's index in its page: the 16 rows of a page and head are contiguous, and one
+ * bulk copy lands them in shared memory in the bank-conflict-free order the tensor-core loads read.
  * Attention operands (queries, cached keys and values) are IEEE fp16: the softmax weights need more
  * mantissa than bf16 offers to stay inside the library's logit tolerance; values are saturated at
  * +-65504 when the library writes them.
