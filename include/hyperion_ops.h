@@ -99,6 +99,26 @@ HYP_API int hyp_op_attn_decode(const hyp_attn_shape* shape, int32_t n_seqs, cons
                                const int32_t* ctx_lens, int32_t n_splits, float* scratch, size_t scratch_bytes,
                                void* out, void* stream);
 
+/* One decode step of the attention sub-layer as hyp_stage_decode runs it, in a single launch: rotary encoding
+ * (Section III-A: grouped-query attention "with rotary position encoding") of the new token's query and key,
+ * append of its key and value to the paged cache, attention of the new token over positions
+ * 0 .. ctx_lens[b] (itself included) and the merge of the context splits (a thread-block cluster per sequence
+ * and KV head, merged through distributed shared memory; no scratch buffer).
+ *   qkv        fp32 [n_seqs, stride]: the q/k/v projection of the new token, [Q heads | K heads | V heads], each
+ *              head head_dim wide, not rotated; stride >= (n_q_heads + 2 n_kv_heads) * head_dim
+ *   kv_pages   one block's page pool (layout above), READ AND WRITTEN: the new token's rotated key and its value
+ *              are stored (fp16) at position ctx_lens[b]; the page holding that position must already be
+ *              listed in the sequence's block-table row
+ *   rope_table fp32 [positions, head_dim / 2, 2]: (cos, sin) of pos * theta^(-2i / head_dim); must cover every
+ *              ctx_lens[b] (not checked: the lengths live on the device)
+ *   n_splits   1 .. 8 context splits, 0 = the library's choice
+ *   out        fp16 [n_seqs, n_q_heads * head_dim]
+ * The first call on a process allocates one device word for error reporting (bounded waits). */
+HYP_API int hyp_op_attn_decode_step(const hyp_attn_shape* shape, int32_t n_seqs, const float* qkv, int32_t stride,
+                                    void* kv_pages, const int32_t* block_table, int32_t max_pages_per_seq,
+                                    const int32_t* ctx_lens, const float* rope_table, int32_t n_splits, void* out,
+                                    void* stream);
+
 /* Decode attention for callers that must not allocate device memory.  (The paper has no counterpart
  * to this call; it is a packaging variant of hyp_op_attn_decode.)
  *

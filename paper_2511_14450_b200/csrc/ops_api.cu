@@ -126,6 +126,28 @@ extern "C" int hyp_op_attn_decode(const hyp_attn_shape* shape, int32_t n_seqs, c
                                    n_splits, bm, d, (cudaStream_t)stream));
 }
 
+extern "C" int hyp_op_attn_decode_step(const hyp_attn_shape* shape, int32_t n_seqs, const float* qkv, int32_t stride,
+                                       void* kv_pages, const int32_t* block_table, int32_t max_pages_per_seq,
+                                       const int32_t* ctx_lens, const float* rope_table, int32_t n_splits, void* out,
+                                       void* stream) {
+  if (!attn_shape_ok(shape) || !qkv || !kv_pages || !block_table || !ctx_lens || !rope_table || !out) return HYP_EINVAL;
+  if (n_seqs < 1 || n_seqs > 65535 || max_pages_per_seq < 1 || n_splits < 0 || n_splits > 8) return HYP_EINVAL;
+  if (stride < (shape->n_q_heads + 2 * shape->n_kv_heads) * shape->head_dim) return HYP_EINVAL;
+  if (((uintptr_t)kv_pages & 15) != 0 || ((uintptr_t)rope_table & 7) != 0) return HYP_EINVAL;
+  int rc = tc_prepare();
+  if (rc) return rc;
+  BatchMeta bm{};
+  bm.n_seqs = n_seqs;
+  bm.n_tokens = n_seqs;
+  bm.max_pages_per_seq = max_pages_per_seq;
+  bm.ctx_lens = ctx_lens;
+  bm.block_table = block_table;
+  const ModelDims d = attn_dims(shape, stride);
+  if (n_splits == 0) n_splits = attn_decode_fused_splits(n_seqs, shape->n_kv_heads, 16 * max_pages_per_seq);
+  return finish(launch_attn_decode_fused(qkv, stride, (__half*)kv_pages, (const float2*)rope_table, (__half*)out, n_splits,
+                                         2, tc_err_flag_ptr(), bm, d, (cudaStream_t)stream));
+}
+
 extern "C" int hyp_op_attn_prefill(const hyp_attn_shape* shape, int32_t n_seqs, int32_t M, const void* q,
                                    int32_t q_stride, const void* kv_pages, const int32_t* block_table,
                                    int32_t max_pages_per_seq, const int32_t* cu_q, const int32_t* ctx_lens, void* out,

@@ -87,6 +87,9 @@ SIGNATURES = {
                                      C.c_void_p, C.c_void_p]),
     "hyp_op_attn_decode_static": (C.c_int, [C.POINTER(hyp_attn_shape), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
                                             C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
+    "hyp_op_attn_decode_step": (C.c_int, [C.POINTER(hyp_attn_shape), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
+                                          C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                          C.c_void_p]),
     "hyp_op_attn_prefill": (C.c_int, [C.POINTER(hyp_attn_shape), C.c_int32, C.c_int32, C.c_void_p, C.c_int32,
                                       C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.c_void_p]),
@@ -322,6 +325,13 @@ def hyp_op_attn_decode_static(shape3, q, kv_pages, block_table, ctx_lens, n_spli
     _check(lib().hyp_op_attn_decode_static(C.byref(sh), q.shape[0], _ptr(q), q.stride(0), _ptr(kv_pages),
                                            _ptr(block_table), block_table.stride(0), _ptr(ctx_lens), n_splits,
                                            _ptr(out), _stream_handle(stream)), "hyp_op_attn_decode_static")
+
+
+def hyp_op_attn_decode_step(shape3, qkv, kv_pages, block_table, ctx_lens, rope_table, n_splits, out, stream=None):
+    sh = hyp_attn_shape(*shape3)
+    _check(lib().hyp_op_attn_decode_step(C.byref(sh), qkv.shape[0], _ptr(qkv), qkv.stride(0), _ptr(kv_pages),
+                                         _ptr(block_table), block_table.stride(0), _ptr(ctx_lens), _ptr(rope_table),
+                                         n_splits, _ptr(out), _stream_handle(stream)), "hyp_op_attn_decode_step")
 
 
 def hyp_op_attn_prefill(shape3, q, kv_pages, block_table, cu_q, ctx_lens, out, stream=None):

@@ -116,6 +116,54 @@ def test_attn_decode(Hq, Hkv, D, n_splits):
         assert np.max(np.abs(f64(out[i]) - want)) < 1.5e-2, (i, L)
 
 
+def rope_table(n_pos, D, theta=10000.0):
+    """(cos, sin) of pos * theta^(-2i/D), angles in double, stored fp32 [n_pos, D/2, 2]."""
+    ang = np.arange(n_pos, dtype=np.float64)[:, None] * theta ** (-2.0 * np.arange(D // 2, dtype=np.float64) / D)
+    return torch.from_numpy(np.stack([np.cos(ang), np.sin(ang)], axis=-1).astype(np.float32)).cuda()
+
+
+@pytest.mark.parametrize("Hq,Hkv,D", [(4, 2, 64), (40, 10, 128), (8, 8, 128), (8, 1, 64)])
+@pytest.mark.parametrize("n_splits", [0, 1, 3, 8])
+def test_attn_decode_step_rotates_appends_attends_and_merges(Hq, Hkv, D, n_splits):
+    """The one-launch decode step against the oracle's rope + attention, on context lengths that sit on, before
+    and after page boundaries (0 = the very first token, 16 = the new token opens a page), with more splits than
+    pages for the short ones, and a second step on top of the first (the appended key / value must be in the
+    cache, in its chunk-permuted place)."""
+    cached = [0, 1, 15, 16, 17, 100, 333]                  # tokens already in the cache
+    pool, table, ks, vs = build_cache([c + 2 for c in cached], Hkv, D, seed=Hq + 1)   # pages for two more tokens
+    n = len(cached)
+    tab = rope_table(400, D)
+    out = torch.empty(n, Hq * D, dtype=torch.float16, device="cuda")
+    stride = (Hq + 2 * Hkv) * D + 8
+    ks = [f64(k) for k in ks]
+    vs = [f64(v) for v in vs]
+    for step in range(2):
+        qkv = bf16_normal(70 + step, (n, stride)).float() * 1.5
+        ctx = torch.tensor([c + step for c in cached], dtype=torch.int32, device="cuda")
+        hyp.hyp_op_attn_decode_step((Hq, Hkv, D), qkv, pool, table, ctx, tab, n_splits, out)
+        torch.cuda.synchronize()
+        for i, c in enumerate(cached):
+            pos = c + step
+            row = f64(qkv[i])
+            q = od.rope(row[:Hq * D].reshape(1, Hq, D), np.array([pos]), 10000.0)
+            k_new = od.rope(row[Hq * D:(Hq + Hkv) * D].reshape(1, Hkv, D), np.array([pos]), 10000.0)
+            v_new = row[(Hq + Hkv) * D:(Hq + 2 * Hkv) * D].reshape(1, Hkv, D)
+            # what the cache holds after the step: the old rows (fp16 values) and the new one rounded to fp16
+            ks[i] = np.concatenate([ks[i][:pos], k_new.astype(np.float16).astype(np.float64)])
+            vs[i] = np.concatenate([vs[i][:pos], v_new.astype(np.float16).astype(np.float64)])
+            want = od.attention(q, ks[i], vs[i], q_pos0=pos).reshape(-1)
+            assert np.max(np.abs(f64(out[i]) - want)) < 1.5e-2, (step, i, pos)
+            # the appended row, read back from its page and un-permuted
+            page, slot = int(table[i, pos // 16]), pos % 16
+            got_k = f64(pool[page, 0, :, slot]).reshape(Hkv, D // 8, 8)
+            src = np.arange(D // 8) ^ (slot & 7)
+            # fp32 rotation on the device against the float64 one: at most one fp16 step apart after rounding
+            assert np.max(np.abs(got_k[:, src].reshape(Hkv, D) - ks[i][pos])) <= 8e-3, (step, i, "key row")
+            ks[i][pos] = got_k[:, src].reshape(Hkv, D)      # the next step attends to what the cache really holds
+            got_v = f64(pool[page, 1, :, slot]).reshape(Hkv, D // 8, 8)
+            assert np.max(np.abs(got_v[:, src].reshape(Hkv, D) - vs[i][pos])) == 0.0, (step, i, "value row")
+
+
 def test_attn_decode_rejects_small_scratch():
     pool, table, _, _ = build_cache([20], 2, 64, seed=1)
     q = bf16_normal(51, (1, 256)).half()
