@@ -274,7 +274,11 @@ int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, void* out, int
 
 template <int NB, bool F16>
 int launch_nb(const TcAct& act, const TcWeight& w, int M, int N, int epi, void* out, int ldo, cudaStream_t st, bool early) {
-  const bool wide = N > 8192;  // many rows: 32 columns per CTA keep the CTA count down
+  // 32 columns per CTA: for matrices with many rows (keeps the CTA count down), and for more than 8 tokens when
+  // that still leaves 1.5 CTAs per SM: every CTA re-reads the activations from L2, and from 16 tokens on those
+  // reads outweigh the weights (measured on B200 at 32 tokens: q/k/v projection 42 us with 16 columns per CTA,
+  // 24 us with 32; L2 -> SM traffic then tops out near 8.5 TB/s)
+  const bool wide = N > 8192 || (NB >= 2 && N >= 32 * 222);
   switch (epi) {
     case EPI_STORE_BF16:
       return wide ? launch_cfg<NB, EPI_STORE_BF16, 2, F16>(act, w, M, N, out, ldo, st, early)

@@ -33,6 +33,7 @@ def test_rmsnorm(M, H):
 GEMM_SHAPES = [  # (M, N, K)
     (1, 256, 256), (8, 512, 256), (32, 256, 688), (5, 1024, 64),          # weight-streaming kernel, K tail
     (8, 528, 1096), (3, 272, 2056), (20, 5120, 17920),                     # its 16-row mode (few rows, long K)
+    (24, 7680, 328), (9, 7120, 264),                                       # its 32-column mode for > 8 tokens
     (33, 512, 256), (128, 256, 256), (200, 1024, 688), (129, 272, 328),   # tile kernel: M, N and K tails
     (512, 7680, 5120),                                                     # QKV projection at full size
 ]
