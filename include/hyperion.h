@@ -104,7 +104,7 @@ enum {
 };
 
 #define HYP_BATCH_ALL_LOGITS 1 /* last stage, prefill: return logits of every row, not only last   */
-#define HYP_MAX_DECODE_BATCH 32
+#define HYP_MAX_DECODE_BATCH 128
 
 /* One call's batch.  All arrays are HOST memory, caller-owned, and fully read before the call
  * returns.  Rows of the batch are packed in sequence order: M = sum(q_lens). */

@@ -60,8 +60,9 @@ HYP_API int hyp_op_pack_weight(const void* w, int32_t N, int32_t K, int32_t swig
  * acc[m, n] = sum_k a[m, k] * w[n, k], bf16 inputs, fp32 accumulation, then `epilogue`.  (The same kernels
  * run inside hyp_stage_* with fp16 operands; this entry point exposes the bf16 instantiation.)
  * a bf16 [M, K] row-major; w_packed = the output of hyp_op_pack_weight for the same N, K and
- * swiglu = (epilogue == HYP_EPI_SWIGLU_BF16); K multiple of 8, N multiple of 16 unless M <= 32.
- * M <= 32 runs the weight-streaming kernel, larger M the tcgen05 tile kernel.
+ * swiglu = (epilogue == HYP_EPI_SWIGLU_BF16); K multiple of 8, N and ldo multiples of 16 and 8 unless M <= 8.
+ * M <= 8 runs the weight-streaming kernel, larger M the tcgen05 kernels (for 9-128 rows the plain-store
+ * epilogues of narrow matrices take the variant with the operands swapped and K split over a cluster).
  * The first call on a process allocates one device word for error reporting. */
 HYP_API int hyp_op_gemm(const void* a, const void* w_packed, int32_t M, int32_t N, int32_t K, int32_t epilogue,
                         void* out, int32_t ldo, void* stream);
@@ -75,9 +76,11 @@ HYP_API int hyp_op_gemm(const void* a, const void* w_packed, int32_t M, int32_t 
  *   HYP_TUNE_ATTN_SLOTS    ring slots per warp of that kernel, 2..4 (0 = built-in)
  *   HYP_TUNE_STREAM_ROTATION  CTA b of the weight-streaming kernel starts its K walk at copy (b * value) mod copies
  *                          (0 = all CTAs walk K in the same order)
+ *   HYP_TUNE_SWAP_MIN_ROWS / HYP_TUNE_SWAP_MAX_ROWS  row counts (1..128; min 129 or max 0 = never) for which a
+ *                          projection runs on the swapped-operand tensor-core kernel
  * Affects launches made after the call; decode graphs already captured keep their setting. */
 enum { HYP_TUNE_PDL = 0, HYP_TUNE_STREAM_SLOTS = 1, HYP_TUNE_ATTN_SPLITS = 2, HYP_TUNE_ATTN_SLOTS = 3,
-       HYP_TUNE_STREAM_ROTATION = 4 };
+       HYP_TUNE_STREAM_ROTATION = 4, HYP_TUNE_SWAP_MIN_ROWS = 5, HYP_TUNE_SWAP_MAX_ROWS = 6 };
 HYP_API int hyp_tune(int32_t key, int32_t value);
 
 /* Number of context splits hyp_op_attn_decode would pick for this batch, and the scratch bytes

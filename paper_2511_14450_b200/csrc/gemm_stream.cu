@@ -1,4 +1,4 @@
-// Weight-streaming projection for M <= 32 rows (decode): out[m, n] (+)= sum_k a[m, k] * w[n, k].
+// Weight-streaming projection for M <= 8 rows (decode): out[m, n] (+)= sum_k a[m, k] * w[n, k].
 //
 // HBM-bound: every weight byte is read exactly once.  Weights are held packed (see gemm_tc.cuh): all k-blocks of
 // a 16-row strip are contiguous, so a CTA, which owns one strip (or two), reads it as a sequential run of 4 KB
@@ -13,7 +13,7 @@
 // MMA's sixteen k slots are assigned to those k so that a lane's 16 bytes are exactly its fragment entries:
 // slots {2t, 2t+1, 2t+8, 2t+9} of the first MMA of a pair hold k = 8t .. 8t+3, the same slots of the second hold
 // 8t+4 .. 8t+7 (t = lane % 4); the weight fragments are read from shared memory with the same assignment (two
-// 128-bit loads per pair), which a dot product does not notice.  Batch 8-32 costs no more copy traffic than batch 1.
+// 128-bit loads per pair), which a dot product does not notice.
 // Each warp keeps a partial sum over its k-blocks; the warps meet in shared memory and the epilogue (16-bit store,
 // residual add, SiLU(gate) * up, fp32 store) is applied once.  Every mbarrier wait is bounded.
 #include "gemm_tc.cuh"
@@ -274,11 +274,7 @@ int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, void* out, int
 
 template <int NB, bool F16>
 int launch_nb(const TcAct& act, const TcWeight& w, int M, int N, int epi, void* out, int ldo, cudaStream_t st, bool early) {
-  // 32 columns per CTA: for matrices with many rows (keeps the CTA count down), and for more than 8 tokens when
-  // that still leaves 1.5 CTAs per SM: every CTA re-reads the activations from L2, and from 16 tokens on those
-  // reads outweigh the weights (measured on B200 at 32 tokens: q/k/v projection 42 us with 16 columns per CTA,
-  // 24 us with 32; L2 -> SM traffic then tops out near 8.5 TB/s)
-  const bool wide = N > 8192 || (NB >= 2 && N >= 32 * 222);
+  const bool wide = N > 8192;  // many rows: 32 columns per CTA keep the CTA count down
   switch (epi) {
     case EPI_STORE_BF16:
       return wide ? launch_cfg<NB, EPI_STORE_BF16, 2, F16>(act, w, M, N, out, ldo, st, early)
@@ -296,19 +292,17 @@ int launch_nb(const TcAct& act, const TcWeight& w, int M, int N, int epi, void* 
 
 template <bool F16>
 int launch_type(const TcAct& act, const TcWeight& w, int M, int N, int epi, void* out, int ldo, cudaStream_t st, bool early) {
-  switch ((M + 7) / 8) {
-    case 1: return launch_nb<1, F16>(act, w, M, N, epi, out, ldo, st, early);
-    case 2: return launch_nb<2, F16>(act, w, M, N, epi, out, ldo, st, early);
-    case 3: return launch_nb<3, F16>(act, w, M, N, epi, out, ldo, st, early);
-    default: return launch_nb<4, F16>(act, w, M, N, epi, out, ldo, st, early);
-  }
+  // One group of 8 tokens.  The kernel is written for NB groups (up to 32 rows), but from 9 rows on the tensor-memory
+  // kernels are faster (every CTA here re-reads the activations of its K range from L2, and at 16+ tokens those
+  // reads outweigh the weights), so only NB = 1 is built.
+  return launch_nb<1, F16>(act, w, M, N, epi, out, ldo, st, early);
 }
 
 }  // namespace
 
 int launch_gemm_stream(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
                        cudaStream_t st, bool early) {
-  if (M < 1 || M > 32 || N < 1 || K < 8 || act.K != K || w.K != K || !tc_err_flag_ptr()) return HYP_EINVAL;
+  if (M < 1 || M > 8 || N < 1 || K < 8 || act.K != K || w.K != K || !tc_err_flag_ptr()) return HYP_EINVAL;
   if (w.rows != N || w.halves != (epi == EPI_SWIGLU_BF16 ? 2 : 1)) return HYP_EINVAL;
   if (act.f16 != w.f16) return HYP_EINVAL;  // one instruction takes both operands in the same 16-bit type
   if (((uintptr_t)act.ptr & 15) != 0 || (K % 8) != 0) return HYP_EINVAL;  // 128-bit activation loads

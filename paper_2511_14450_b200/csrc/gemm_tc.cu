@@ -21,6 +21,7 @@
 
 #include "gemm_tc.cuh"
 #include "sm100_common.cuh"
+#include "tcgen05.cuh"
 #include "hyperion.h"
 
 namespace hyp {
@@ -32,38 +33,6 @@ constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTE
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
 constexpr int TC_THREADS = 192;
 
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, 8-row groups 1024 B apart.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)1 << 16;            // leading byte offset: not used by swizzled K-major layouts
-  d |= (uint64_t)(1024 >> 4) << 32;  // stride byte offset between 8-row groups
-  d |= (uint64_t)1 << 46;            // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;            // 128-byte swizzle
-  return d;
-}
 // Instruction descriptor: (bf16 x bf16 | fp16 x fp16) -> fp32, both operands K-major, M = 128, N = 256.
 constexpr uint32_t IDESC_BF16 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 constexpr uint32_t IDESC_F16 = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
@@ -593,7 +562,7 @@ int* g_err_flag = nullptr;  // one device word per process: first non-zero code 
 
 template <int EPI>
 int launch_pair(const TcAct& act, const TcWeight& w, int M, int N, int K, void* out, int ldo, cudaStream_t st,
-                int num_sms) {
+                int num_sms, bool early) {
   static bool configured = false;
   if (!configured) {
     HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_tc2_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
@@ -622,13 +591,17 @@ int launch_pair(const TcAct& act, const TcWeight& w, int M, int N, int K, void* 
   } else if (tiles < pairs) {
     pairs = tiles;
   }
-  HYP_CUDA_TRY(launch_pdl(gemm_tc2_kernel<EPI>, dim3((unsigned)(2 * pairs)), dim3(TC_THREADS), (size_t)SMEM2_BYTES, st, act.map,
-                          w.map, M, N, K, w.N16p, out, ldo, team, act.f16 ? IDESC2_F16 : IDESC2_BF16, g_err_flag));
+  if (early)
+    HYP_CUDA_TRY(launch_pdl<1>(gemm_tc2_kernel<EPI>, dim3((unsigned)(2 * pairs)), dim3(TC_THREADS), (size_t)SMEM2_BYTES, st,
+                               act.map, w.map, M, N, K, w.N16p, out, ldo, team, act.f16 ? IDESC2_F16 : IDESC2_BF16, g_err_flag));
+  else
+    HYP_CUDA_TRY(launch_pdl(gemm_tc2_kernel<EPI>, dim3((unsigned)(2 * pairs)), dim3(TC_THREADS), (size_t)SMEM2_BYTES, st,
+                            act.map, w.map, M, N, K, w.N16p, out, ldo, team, act.f16 ? IDESC2_F16 : IDESC2_BF16, g_err_flag));
   return 1;
 }
 
 template <int EPI>
-int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* out, int ldo, cudaStream_t st) {
+int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* out, int ldo, cudaStream_t st, bool early) {
   static bool configured = false;
   static int num_sms = 0;
   if (!configured) {
@@ -642,7 +615,7 @@ int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
   const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN_OUT - 1) / BN_OUT;
   // two-CTA tiles (a third less shared-memory fill per flop) from 129 rows on; the residual epilogue up to 4096 rows
   // (stream-K), beyond that whole one-CTA tiles balance by themselves
-  if (tiles_m >= 2 && (EPI != EPI_RESID_F32 || tiles_m <= 32)) return launch_pair<EPI>(act, w, M, N, K, out, ldo, st, num_sms);
+  if (tiles_m >= 2 && (EPI != EPI_RESID_F32 || tiles_m <= 32)) return launch_pair<EPI>(act, w, M, N, K, out, ldo, st, num_sms, early);
   int grid, team = 0;  // team 0 = whole tiles per CTA
   if (EPI == EPI_RESID_F32 && tiles_m <= 16) {
     // stream-K (up to 2048 rows; beyond that whole tiles already balance and reuse A better): pick the team size (a divisor of tiles_m) that keeps most SMs busy, larger teams preferred
@@ -662,8 +635,13 @@ int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
     const long tiles = (long)tiles_m * tiles_n;
     grid = (int)(tiles < num_sms ? tiles : num_sms);
   }
-  HYP_CUDA_TRY(launch_pdl(gemm_tc_kernel<EPI>, dim3(grid), dim3(TC_THREADS), (size_t)SMEM_BYTES, st, act.map, w.map, M, N,
-                          K, w.N16p, out, ldo, team, act.f16 ? IDESC_F16 : IDESC_BF16, g_err_flag));
+  // launched early (set-up under the predecessor's tail; every load waits for it) where the caller allows
+  if (early)
+    HYP_CUDA_TRY(launch_pdl<1>(gemm_tc_kernel<EPI>, dim3(grid), dim3(TC_THREADS), (size_t)SMEM_BYTES, st, act.map, w.map, M,
+                               N, K, w.N16p, out, ldo, team, act.f16 ? IDESC_F16 : IDESC_BF16, g_err_flag));
+  else
+    HYP_CUDA_TRY(launch_pdl(gemm_tc_kernel<EPI>, dim3(grid), dim3(TC_THREADS), (size_t)SMEM_BYTES, st, act.map, w.map, M, N,
+                            K, w.N16p, out, ldo, team, act.f16 ? IDESC_F16 : IDESC_BF16, g_err_flag));
   return 1;
 }
 
@@ -727,11 +705,11 @@ int tc_pack_weight(const void* src, void* dst, int rows, int halves, int K, bool
   return 1;
 }
 
-// Activations: 128-row boxes for the tile kernel, 8/16/24/32-row boxes for the weight-streaming kernel.
+// Activations: 128-row boxes for the tile kernels, 16/32/64-row boxes for the swapped-operand kernel.
 int tc_make_act(TcAct* a, const void* ptr, int rows, int K, bool f16) {
   a->ptr = ptr; a->rows = rows; a->K = K; a->f16 = f16;
   int rc = encode_map(&a->map, ptr, rows, K, 128, f16);
-  for (int nb = 1; nb <= 4 && !rc; ++nb) rc = encode_map(&a->map_small[nb - 1], ptr, rows, K, 8 * nb, f16);
+  for (int i = 0; i < 3 && !rc; ++i) rc = encode_map(&a->map_small[i], ptr, rows, K, 16 << i, f16);
   return rc;
 }
 
@@ -753,15 +731,15 @@ int tc_error_flag(int* value_out) {
 }
 
 int launch_gemm_tc(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
-                   cudaStream_t st) {
+                   cudaStream_t st, bool early) {
   if (M < 1 || N < 1 || K < 8 || act.K != K || w.K != K || M > act.rows || !g_err_flag) return HYP_EINVAL;
   if (w.rows != N || w.halves != (epi == EPI_SWIGLU_BF16 ? 2 : 1)) return HYP_EINVAL;
   if (act.f16 != w.f16) return HYP_EINVAL;  // one instruction takes both operands in the same 16-bit type
   switch (epi) {
-    case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16>(act, w, M, N, K, out, ldo, st);
-    case EPI_RESID_F32: return launch_epi<EPI_RESID_F32>(act, w, M, N, K, out, ldo, st);
-    case EPI_SWIGLU_BF16: return launch_epi<EPI_SWIGLU_BF16>(act, w, M, N, K, out, ldo, st);
-    case EPI_STORE_F32: return launch_epi<EPI_STORE_F32>(act, w, M, N, K, out, ldo, st);
+    case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16>(act, w, M, N, K, out, ldo, st, early);
+    case EPI_RESID_F32: return launch_epi<EPI_RESID_F32>(act, w, M, N, K, out, ldo, st, early);
+    case EPI_SWIGLU_BF16: return launch_epi<EPI_SWIGLU_BF16>(act, w, M, N, K, out, ldo, st, early);
+    case EPI_STORE_F32: return launch_epi<EPI_STORE_F32>(act, w, M, N, K, out, ldo, st, early);
     default: return HYP_EINVAL;
   }
 }

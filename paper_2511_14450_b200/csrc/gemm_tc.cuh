@@ -39,7 +39,7 @@ struct TcAct {
   const void* ptr = nullptr;
   int rows = 0, K = 0;
   bool f16 = false;
-  CUtensorMap map_small[4];  // weight-streaming kernel: [nb - 1] = boxes of 8 * nb rows
+  CUtensorMap map_small[3];  // boxes of 16, 32, 64 rows (swapped-operand kernel: the tokens are the N operand)
 };
 int tc_make_act(TcAct* a, const void* ptr, int rows, int K, bool f16 = false);
 
@@ -56,13 +56,26 @@ int& gemm_stream_slots_override();
 // Per-CTA stagger of the K walk of the weight-streaming kernel: CTA b starts at copy (b * rotation) mod copies.
 int& gemm_stream_rotation();
 
-// Weight-streaming projection for M <= 32 rows (decode); same contract as launch_gemm_tc.  `early`: the packed
+// Weight-streaming projection for M <= 8 rows (decode); same contract as launch_gemm_tc.  `early`: the packed
 // weights are long-lived (not written by the kernel launched just before), so the launch may overlap that kernel.
 int launch_gemm_stream(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
                        cudaStream_t st, bool early = false);
 
+// The same projection for 1..128 rows with the operands swapped on the tensor cores (128 weight rows = the M
+// operand, the tokens = the N operand, K split over a cluster): activation traffic per weight byte is rows / 128.
+// launch_projection routes the plain-store epilogues of row counts in [gemm_swap_min_rows(), gemm_swap_max_rows()]
+// (default 9..128) to it when the matrix has too few 256-column tiles for the tile kernel.
+int& gemm_swap_min_rows();
+int& gemm_swap_max_rows();
+int launch_gemm_swap(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
+                     cudaStream_t st, bool early = false);
+
 // out[m, n] (+)= sum_k act[m, k] * w[n, k] for m < M, n < N (SwiGLU: w holds two halves of N rows).
 int launch_gemm_tc(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
-                   cudaStream_t st);
+                   cudaStream_t st, bool early = false);
+
+// Picks the kernel by row count and epilogue (see its definition) and launches it.
+int launch_projection(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo, cudaStream_t st,
+                      bool early = false);
 
 }  // namespace hyp

@@ -66,6 +66,14 @@ extern "C" int hyp_tune(int32_t key, int32_t value) {
       if (value < 0 || value > 1024) return HYP_EINVAL;
       gemm_stream_rotation() = value;
       return HYP_OK;
+    case HYP_TUNE_SWAP_MIN_ROWS:
+      if (value < 1 || value > 129) return HYP_EINVAL;
+      gemm_swap_min_rows() = value;
+      return HYP_OK;
+    case HYP_TUNE_SWAP_MAX_ROWS:
+      if (value < 0 || value > 128) return HYP_EINVAL;
+      gemm_swap_max_rows() = value;
+      return HYP_OK;
     case HYP_TUNE_ATTN_SPLITS:
       if (value < 0 || value > 8) return HYP_EINVAL;
       attn_fused_splits_override() = value;
@@ -83,7 +91,7 @@ extern "C" int hyp_op_gemm(const void* a, const void* w, int32_t M, int32_t N, i
   if (!a || !w || !out || M < 1 || N < 1 || K < 8 || K % 8 || ldo < N || ((uintptr_t)w & 127) != 0) return HYP_EINVAL;
   if (epilogue < HYP_EPI_STORE_BF16 || epilogue > HYP_EPI_STORE_F32) return HYP_EINVAL;
   cudaStream_t st = (cudaStream_t)stream;
-  if (M > 32 && (N % 16 || ldo % 8)) return HYP_EINVAL;
+  if (M > 8 && (N % 16 || ldo % 8)) return HYP_EINVAL;
   int rc = tc_prepare();
   if (rc) return rc;
   TcAct ta;
@@ -92,8 +100,7 @@ extern "C" int hyp_op_gemm(const void* a, const void* w, int32_t M, int32_t N, i
   if (rc) return rc;
   rc = tc_make_weight(&tw, w, N, epilogue == HYP_EPI_SWIGLU_BF16 ? 2 : 1, K, false);
   if (rc) return rc;
-  if (M <= 32) return finish(launch_gemm_stream(ta, tw, M, N, K, epilogue, out, ldo, st));
-  return finish(launch_gemm_tc(ta, tw, M, N, K, epilogue, out, ldo, st));
+  return finish(launch_projection(ta, tw, M, N, K, epilogue, out, ldo, st));
 }
 
 extern "C" int hyp_op_attn_decode_splits(int32_t n_seqs, int32_t n_kv_heads, int32_t max_ctx) {

@@ -274,8 +274,7 @@ int check_ready(const hyp_stage* s) {
 int project(hyp_stage* s, const TcAct& act, const bf16* a, int lda, const TcWeight& tw, const bf16* w, int N, int K,
             int M, int epi, void* out, int ldo, cudaStream_t st) {
   (void)a; (void)lda; (void)w;
-  if (M <= 32) return launch_gemm_stream(act, tw, M, N, K, epi, out, ldo, st, /*early=*/true);
-  return launch_gemm_tc(act, tw, M, N, K, epi, out, ldo, st);
+  return launch_projection(act, tw, M, N, K, epi, out, ldo, st, /*early=*/true);
 }
 
 // The block sequence B_lo -> ... -> B_{hi-1} on rows already resident in s->x.

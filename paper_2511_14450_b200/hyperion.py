@@ -17,7 +17,7 @@ HYP_ETIMEOUT = -7
 (HYP_W_QKV, HYP_W_O, HYP_W_GATE_UP, HYP_W_DOWN, HYP_W_NORM1, HYP_W_NORM2, HYP_W_EMBED, HYP_W_FINAL_NORM,
  HYP_W_LM_HEAD) = range(9)
 HYP_BATCH_ALL_LOGITS = 1
-HYP_MAX_DECODE_BATCH = 32
+HYP_MAX_DECODE_BATCH = 128
 
 
 class hyp_cfg(C.Structure):
@@ -271,7 +271,8 @@ def hyp_op_rmsnorm(x, g, out, eps: float, stream=None):
     _check(lib().hyp_op_rmsnorm(_ptr(x), _ptr(g), _ptr(out), M, H, eps, _stream_handle(stream)), "hyp_op_rmsnorm")
 
 
-HYP_TUNE_PDL, HYP_TUNE_STREAM_SLOTS, HYP_TUNE_ATTN_SPLITS, HYP_TUNE_ATTN_SLOTS, HYP_TUNE_STREAM_ROTATION = range(5)
+(HYP_TUNE_PDL, HYP_TUNE_STREAM_SLOTS, HYP_TUNE_ATTN_SPLITS, HYP_TUNE_ATTN_SLOTS, HYP_TUNE_STREAM_ROTATION,
+ HYP_TUNE_SWAP_MIN_ROWS, HYP_TUNE_SWAP_MAX_ROWS) = range(7)
 
 
 def hyp_tune(key: int, value: int):

@@ -75,6 +75,32 @@ def kv_rows(x):
     return out.reshape(slots, Hkv, D).permute(1, 0, 2)
 
 
+@pytest.mark.parametrize("N,K,swiglu", [(48, 128, False), (272, 328, True), (1000, 72, False)])
+def test_pack_weight_layout(N, K, swiglu):
+    """The packed copy against the layout the header states, built with numpy: tile (t, kb) at (t * KBp + kb) * 2 KB,
+    t = half * strips + n // 16; inside a tile row r, 16-byte chunk c at chunk position c ^ (r & 7); zero padding."""
+    rows = 2 * N if swiglu else N
+    w = bf16_normal(8, (rows, K))
+    packed = hyp.hyp_op_pack_weight(w, N, swiglu).cpu().numpy().view(np.uint16)
+    bits = w.cpu().view(torch.int16).numpy().view(np.uint16)
+    strips = -(-N // 16)
+    strips += strips & 1
+    kbp = -(-K // 64)
+    kbp += kbp & 1
+    want = np.zeros(((2 if swiglu else 1) * strips, kbp, 16, 8, 8), np.uint16)
+    for half in range(2 if swiglu else 1):
+        for n in range(N):
+            t, r = half * strips + n // 16, n % 16
+            for kb in range(-(-K // 64)):
+                blk = np.zeros(64, np.uint16)
+                seg = bits[half * N + n, kb * 64:min(K, kb * 64 + 64)]
+                blk[:len(seg)] = seg
+                chunks = blk.reshape(8, 8)
+                want[t, kb, r, np.arange(8) ^ (r & 7)] = chunks
+    assert packed.size == want.size
+    assert np.array_equal(packed, want.reshape(-1))
+
+
 def build_cache(seq_lens, Hkv, D, seed):
     """Random rotated keys / values (fp16) for each sequence, scattered into a shuffled page pool."""
     n = len(seq_lens)

@@ -125,3 +125,19 @@ def test_strerror_covers_all_codes():
     seen = {L.hyp_strerror(c).decode() for c in range(0, -8, -1)}
     assert len(seen) == 8 and "unknown status" not in seen
     assert L.hyp_strerror(-99).decode() == "unknown status"
+
+
+def test_packed_weight_size_and_tuning_switch_ranges():
+    """Host-only parts of the single-kernel API: the packed size is whole 2 KB tiles with an even number of 16-row
+    strips and 64-k blocks per half, and the tuning switches refuse values outside their range."""
+    L = hyp.lib()
+    for N, K, sw in [(5120, 5120, 0), (17920, 5120, 1), (256, 688, 0), (272, 328, 1), (1, 8, 0)]:
+        strips = -(-N // 16)
+        strips += strips & 1
+        kblocks = -(-K // 64)
+        kblocks += kblocks & 1
+        assert L.hyp_op_weight_packed_bytes(N, K, sw) == (2 if sw else 1) * strips * kblocks * 2048
+    assert L.hyp_op_weight_packed_bytes(0, 64, 0) == 0 and L.hyp_op_weight_packed_bytes(16, 12, 0) == 0
+    assert L.hyp_tune(hyp.HYP_TUNE_PDL, 4) == hyp.HYP_EINVAL and L.hyp_tune(hyp.HYP_TUNE_STREAM_SLOTS, 9) == hyp.HYP_EINVAL
+    assert L.hyp_tune(hyp.HYP_TUNE_ATTN_SPLITS, 9) == hyp.HYP_EINVAL and L.hyp_tune(99, 0) == hyp.HYP_EINVAL
+    assert L.hyp_tune(hyp.HYP_TUNE_STREAM_SLOTS, 0) == hyp.HYP_OK
