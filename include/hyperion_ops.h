@@ -77,10 +77,13 @@ HYP_API int hyp_op_gemm(const void* a, const void* w_packed, int32_t M, int32_t 
  *   HYP_TUNE_STREAM_ROTATION  CTA b of the weight-streaming kernel starts its K walk at copy (b * value) mod copies
  *                          (0 = all CTAs walk K in the same order)
  *   HYP_TUNE_SWAP_MIN_ROWS / HYP_TUNE_SWAP_MAX_ROWS  row counts (1..128; min 129 or max 0 = never) for which a
- *                          projection runs on the swapped-operand tensor-core kernel
+ *                          projection may run on the swapped-operand tensor-core kernel (a minimum below 9
+ *                          also takes those row counts away from the weight-streaming kernel)
+ *   HYP_TUNE_SWAP_EPILOGUES  bit mask over the HYP_EPI_* values: which epilogues may take that kernel
+ *                          (default: the two plain stores; it is only chosen for matrices of < 100 tiles of 256 rows)
  * Affects launches made after the call; decode graphs already captured keep their setting. */
 enum { HYP_TUNE_PDL = 0, HYP_TUNE_STREAM_SLOTS = 1, HYP_TUNE_ATTN_SPLITS = 2, HYP_TUNE_ATTN_SLOTS = 3,
-       HYP_TUNE_STREAM_ROTATION = 4, HYP_TUNE_SWAP_MIN_ROWS = 5, HYP_TUNE_SWAP_MAX_ROWS = 6 };
+       HYP_TUNE_STREAM_ROTATION = 4, HYP_TUNE_SWAP_MIN_ROWS = 5, HYP_TUNE_SWAP_MAX_ROWS = 6, HYP_TUNE_SWAP_EPILOGUES = 7 };
 HYP_API int hyp_tune(int32_t key, int32_t value);
 
 /* Number of context splits hyp_op_attn_decode would pick for this batch, and the scratch bytes

@@ -33,6 +33,11 @@ int& gemm_swap_max_rows() {
 }
 
 
+int& gemm_swap_epilogues() {
+  static int v = (1 << EPI_STORE_BF16) | (1 << EPI_STORE_F32);
+  return v;
+}
+
 namespace {
 
 constexpr int SW_ROWS = 128, SW_BK = 64, SW_THREADS = 192, SW_MAX_STAGES = 8;
@@ -331,8 +336,8 @@ int launch_gemm_swap(const TcAct& act, const TcWeight& w, int M, int N, int K, i
 //   above            the tile kernels.
 int launch_projection(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo, cudaStream_t st,
                       bool early) {
-  if (M <= 8) return launch_gemm_stream(act, w, M, N, K, epi, out, ldo, st, early);
-  const bool store = epi == EPI_STORE_BF16 || epi == EPI_STORE_F32;
+  if (M <= 8 && M < gemm_swap_min_rows()) return launch_gemm_stream(act, w, M, N, K, epi, out, ldo, st, early);
+  const bool store = epi >= 0 && epi < 4 && ((gemm_swap_epilogues() >> epi) & 1);
   if (store && M >= gemm_swap_min_rows() && M <= gemm_swap_max_rows() && (N + 255) / 256 < 100)
     return launch_gemm_swap(act, w, M, N, K, epi, out, ldo, st, early);
   return launch_gemm_tc(act, w, M, N, K, epi, out, ldo, st, early && M <= 128);

@@ -67,6 +67,7 @@ int launch_gemm_stream(const TcAct& act, const TcWeight& w, int M, int N, int K,
 // (default 9..128) to it when the matrix has too few 256-column tiles for the tile kernel.
 int& gemm_swap_min_rows();
 int& gemm_swap_max_rows();
+int& gemm_swap_epilogues();  // bit e set: epilogue e may take the swapped kernel (default: the two plain stores)
 int launch_gemm_swap(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
                      cudaStream_t st, bool early = false);
 

@@ -74,6 +74,10 @@ extern "C" int hyp_tune(int32_t key, int32_t value) {
       if (value < 0 || value > 128) return HYP_EINVAL;
       gemm_swap_max_rows() = value;
       return HYP_OK;
+    case HYP_TUNE_SWAP_EPILOGUES:
+      if (value < 0 || value > 15) return HYP_EINVAL;
+      gemm_swap_epilogues() = value;
+      return HYP_OK;
     case HYP_TUNE_ATTN_SPLITS:
       if (value < 0 || value > 8) return HYP_EINVAL;
       attn_fused_splits_override() = value;

@@ -75,6 +75,22 @@ def kv_rows(x):
     return out.reshape(slots, Hkv, D).permute(1, 0, 2)
 
 
+@pytest.mark.parametrize("M,N,K", [(1, 256, 256), (8, 528, 1096), (20, 5120, 17920), (33, 512, 256), (128, 272, 328),
+                                   (100, 1024, 688), (16, 17920, 512)])
+@pytest.mark.parametrize("epi", [hyp.HYP_EPI_STORE_BF16, hyp.HYP_EPI_RESID_F32, hyp.HYP_EPI_SWIGLU_BF16,
+                                 hyp.HYP_EPI_STORE_F32])
+def test_gemm_swapped_operand_kernel_all_epilogues(M, N, K, epi):
+    """Every epilogue and 1-128 rows forced through the swapped-operand kernel (by default it only takes the plain
+    stores of 9-128 rows): ragged N (not a multiple of 128), K tails, clusters of 1-8 K shares, all four token tiles."""
+    hyp.hyp_tune(hyp.HYP_TUNE_SWAP_MIN_ROWS, 1)
+    hyp.hyp_tune(hyp.HYP_TUNE_SWAP_EPILOGUES, 15)
+    try:
+        test_gemm_all_epilogues(M, N, K, epi)
+    finally:
+        hyp.hyp_tune(hyp.HYP_TUNE_SWAP_MIN_ROWS, 9)
+        hyp.hyp_tune(hyp.HYP_TUNE_SWAP_EPILOGUES, (1 << hyp.HYP_EPI_STORE_BF16) | (1 << hyp.HYP_EPI_STORE_F32))
+
+
 @pytest.mark.parametrize("N,K,swiglu", [(48, 128, False), (272, 328, True), (1000, 72, False)])
 def test_pack_weight_layout(N, K, swiglu):
     """The packed copy against the layout the header states, built with numpy: tile (t, kb) at (t * KBp + kb) * 2 KB,
