@@ -74,20 +74,30 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
   const size_t v_off = (size_t)d.Hkv * AF_PT * D;
   const uint32_t my_bars = smem_u32(bars) + 8u * (warp * AF_MAX_SLOTS);
   const uint32_t my_ring = ring0 + (uint32_t)(warp * S) * SLOT_BYTES;
-  auto issue = [&](int i, int slot) {  // this warp's i-th page
-    const int pi = p_begin + warp + AF_WARPS * i;
-    const __half* src = a.kv_layer + (size_t)bt[pi] * page_elems + (size_t)kvh * AF_PT * D;
+  const int my_n = p_begin + warp < p_end ? (p_end - p_begin - warp + AF_WARPS - 1) / AF_WARPS : 0;
+  // the block-table entries of this warp's pages, one per lane (two rounds): a refill then needs no dependent
+  // global load in front of its copy
+  const int32_t bt_lo = lane < my_n ? bt[p_begin + warp + AF_WARPS * lane] : 0;
+  const int32_t bt_hi = lane + 32 < my_n ? bt[p_begin + warp + AF_WARPS * (lane + 32)] : 0;
+  auto page_of = [&](int i) {  // all lanes call; page id of this warp's i-th page
+    const int32_t lo = __shfl_sync(0xffffffffu, bt_lo, i & 31), hi = __shfl_sync(0xffffffffu, bt_hi, i & 31);
+    return i < 32 ? lo : i < 64 ? hi : bt[p_begin + warp + AF_WARPS * i];
+  };
+  auto issue = [&](int page, int slot) {  // lane 0: copy one page's keys and values of this head into a slot
+    const __half* src = a.kv_layer + (size_t)page * page_elems + (size_t)kvh * AF_PT * D;
     const uint32_t dst = my_ring + slot * SLOT_BYTES, bar = my_bars + 8u * slot;
     mbar_expect_tx(bar, SLOT_BYTES);
     bulk_load(dst, src, PAGE_BYTES, bar);
     bulk_load(dst + PAGE_BYTES, src + v_off, PAGE_BYTES, bar);
   };
-  const int my_n = p_begin + warp < p_end ? (p_end - p_begin - warp + AF_WARPS - 1) / AF_WARPS : 0;
   pdl_trigger();
   if (lane == 0) {
     for (int sl = 0; sl < S; ++sl) mbar_init(my_bars + 8u * sl, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    for (int sl = 0; sl < S && sl < my_n; ++sl) issue(sl, sl);
+  }
+  for (int sl = 0; sl < S && sl < my_n; ++sl) {
+    const int page = page_of(sl);
+    if (lane == 0) issue(page, sl);
   }
   pdl_wait();  // the projection's output
 
@@ -215,9 +225,12 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
     }
     // all reads of the slot are consumed by issued MMAs; hand it back to the copy engine
     __syncwarp();
-    if (lane == 0 && i + S < my_n) {
-      if (patched) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      issue(i + S, slot);
+    if (i + S < my_n) {
+      const int page = page_of(i + S);
+      if (lane == 0) {
+        if (patched) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        issue(page, slot);
+      }
     }
     if (++slot == S) { slot = 0; phase ^= 1u; }
   }
