@@ -212,6 +212,25 @@ HYP_API void hyp_stage_destroy(hyp_stage* s);
 HYP_API int hyp_split_dp(int32_t N, int32_t T, const double* f, const double* m, const double* C,
                  const double* Mcap, double eps, int32_t* p_out, double* tau_out);
 
+/* The partitioning steps of the two systems the paper compares against (Section V, "HEFT" and "GPipe"), on the
+ * same inputs as hyp_split_dp, so that their bottleneck max_j L_j(p) can be set beside HypSplit-DP's on measured
+ * per-block costs.  The paper names the strategies and gives no algorithm; the readings taken here:
+ *   hyp_split_even   ("classic static, load balanced partitioning" of GPipe into contiguous segments):
+ *                    segments of equal block count, the N mod T leading tiers one block longer; costs,
+ *                    capacities and memory limits play no part.  p_out and tau_out are always written for valid
+ *                    arguments with N >= T; the return value is HYP_EINFEASIBLE if a segment exceeds its tier's
+ *                    memory limit (the partition is reported, not repaired).
+ *   hyp_split_greedy ("memory aware greedy strategy" that precedes HEFT's scheduling): tiers are filled in order;
+ *                    tier j keeps taking the next block while its memory limit holds and its load stays within
+ *                    its capacity-proportional share S_f[N] * C_j / sum(C), takes at least one block, and leaves
+ *                    one block for every later tier; the last tier takes the rest.  HYP_EINFEASIBLE (outputs
+ *                    untouched) if a tier cannot hold its first block or the last tier cannot hold the rest.
+ * Arguments, units and the other errors: as hyp_split_dp (no eps).  Pure host functions, thread-safe. */
+HYP_API int hyp_split_even(int32_t N, int32_t T, const double* f, const double* m, const double* C,
+                           const double* Mcap, int32_t* p_out, double* tau_out);
+HYP_API int hyp_split_greedy(int32_t N, int32_t T, const double* f, const double* m, const double* C,
+                             const double* Mcap, int32_t* p_out, double* tau_out);
+
 /* Real-time state of one node of a tier, as Algorithm 2 (HypSched-RT) reads it. */
 typedef struct {
   double C;        /* computing capacity C_{j,k} (> 0)                                             */

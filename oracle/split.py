@@ -19,6 +19,16 @@ Readings where the paper is silent (each is restated in the library's header):
   - initial bounds: tau_low = 0, tau_high = S_f[N] / min_j C_j;
   - the returned tau* is max_j L_j(p*) of the returned partition, not the last probe value.
 
+* `split_even`, `split_greedy` - the inter-tier partitioning halves of the paper's two comparison
+  systems (Section V, baselines), which it only names: the "classic static, load balanced
+  partitioning" of GPipe into contiguous segments, and the "memory aware greedy strategy" that
+  precedes HEFT.  Readings taken (the paper gives no algorithm for either):
+  - even: contiguous segments of equal block count, the N mod T leading tiers one block longer;
+    blind to costs, capacities and memory (a violated memory limit is reported, not repaired);
+  - greedy: tiers are filled in order; tier j keeps taking the next block while its memory limit
+    holds and its load stays within its capacity-proportional share S_f[N] * C_j / sum(C), takes at
+    least one block, and always leaves one block for every later tier; the last tier takes the rest.
+
 The block allocations printed in the paper's utilisation table: parity unpinned (the f_i, m_i
 and capacities that produced them are not published).
 """
@@ -162,3 +172,60 @@ def hypsched_rt_scan(F_new, m_act, nodes):
             if cost < min_cost:
                 min_cost, k_star = cost, k
     return k_star
+
+
+def split_even(N, T):
+    """GPipe-style static partition (Section V, second baseline): contiguous segments of equal
+    block count; the first N mod T tiers get one block more.  Returns p (1-based last block of
+    tiers 1..T-1)."""
+    base, extra = divmod(N, T)
+    p, cut = [], 0
+    for j in range(T - 1):
+        cut += base + (1 if j < extra else 0)
+        p.append(cut)
+    return tuple(p)
+
+
+def split_greedy(f, m, C, Mcap):
+    """Memory-aware greedy contiguous partition (Section V, first baseline, its partitioning step).
+    Returns p, or None if some tier's first block, or the remainder left to the last tier, breaks
+    a memory limit."""
+    N, T = len(f), len(C)
+    total = 0.0
+    for x in f:
+        total += float(x)
+    csum = 0.0
+    for c in C:
+        csum += float(c)
+    p, nxt = [], 0                      # nxt = 0-based index of the next unassigned block
+    for j in range(T - 1):
+        share = total * float(C[j]) / csum
+        load, mem, taken = 0.0, 0.0, 0
+        while nxt < N - (T - 1 - j):    # leave one block for every later tier
+            nl, nm = load + float(f[nxt]), mem + float(m[nxt])
+            if nm > Mcap[j]:
+                break
+            if taken >= 1 and nl > share:
+                break
+            load, mem, taken, nxt = nl, nm, taken + 1, nxt + 1
+        if taken == 0:
+            return None
+        p.append(nxt)
+    rest = 0.0
+    for i in range(nxt, N):
+        rest += float(m[i])
+    if nxt >= N or rest > Mcap[T - 1]:
+        return None
+    return tuple(p)
+
+
+def memory_feasible(p, m, Mcap):
+    """Does every tier's segment of the partition p fit its memory limit?"""
+    cuts = [0] + list(p) + [len(m)]
+    for j in range(len(Mcap)):
+        u = 0.0
+        for i in range(cuts[j], cuts[j + 1]):
+            u += float(m[i])
+        if u > Mcap[j]:
+            return False
+    return True

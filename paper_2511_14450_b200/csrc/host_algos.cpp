@@ -145,3 +145,94 @@ extern "C" int hyp_sched_rt(double F_new, double m_act, const hyp_node_state* no
   *k_out = k_star;
   return HYP_OK;
 }
+
+// -------------------------------------------------------------------------------------------------
+// The partitioning halves of the paper's two comparison systems (Section V names them, gives no algorithm;
+// the readings are stated in hyperion.h).  They exist to show, on measured per-block costs, the bottleneck
+// gap that HypSplit-DP closes.
+// -------------------------------------------------------------------------------------------------
+namespace {
+
+int check_split_args(int32_t N, int32_t T, const double* f, const double* m, const double* C, const double* Mcap,
+                     const int32_t* p_out, const double* tau_out) {
+  if (N < 1 || T < 1 || !f || !m || !C || !Mcap || !tau_out) return HYP_EINVAL;
+  if (T > 1 && !p_out) return HYP_EINVAL;
+  for (int i = 0; i < N; ++i)
+    if (!(f[i] >= 0.0) || !(m[i] >= 0.0) || std::isinf(f[i]) || std::isinf(m[i])) return HYP_EINVAL;
+  for (int j = 0; j < T; ++j)
+    if (!(C[j] > 0.0) || std::isinf(C[j]) || !(Mcap[j] >= 0.0)) return HYP_EINVAL;
+  return N < T ? HYP_EINFEASIBLE : HYP_OK;
+}
+
+// max_j load and memory feasibility of a partition given as cut points (1-based last blocks of tiers 1..T-1)
+bool evaluate_partition(const std::vector<int32_t>& p, int N, int T, const double* f, const double* m, const double* C,
+                        const double* Mcap, double* tau) {
+  bool fits = true;
+  double worst = 0.0;
+  int first = 0;
+  for (int j = 0; j < T; ++j) {
+    const int last = j == T - 1 ? N : p[j];
+    double load = 0.0, mem = 0.0;
+    for (int i = first; i < last; ++i) {
+      load += f[i];
+      mem += m[i];
+    }
+    if (mem > Mcap[j]) fits = false;
+    if (load / C[j] > worst) worst = load / C[j];
+    first = last;
+  }
+  *tau = worst;
+  return fits;
+}
+
+}  // namespace
+
+extern "C" int hyp_split_even(int32_t N, int32_t T, const double* f, const double* m, const double* C,
+                              const double* Mcap, int32_t* p_out, double* tau_out) {
+  int rc = check_split_args(N, T, f, m, C, Mcap, p_out, tau_out);
+  if (rc) return rc;
+  std::vector<int32_t> p(std::max(T - 1, 1), 0);
+  const int base = N / T, extra = N % T;
+  int cut = 0;
+  for (int j = 0; j < T - 1; ++j) {
+    cut += base + (j < extra ? 1 : 0);
+    p[j] = cut;
+  }
+  double tau = 0.0;
+  const bool fits = evaluate_partition(p, N, T, f, m, C, Mcap, &tau);
+  for (int j = 0; j < T - 1; ++j) p_out[j] = p[j];
+  *tau_out = tau;
+  return fits ? HYP_OK : HYP_EINFEASIBLE;
+}
+
+extern "C" int hyp_split_greedy(int32_t N, int32_t T, const double* f, const double* m, const double* C,
+                                const double* Mcap, int32_t* p_out, double* tau_out) {
+  int rc = check_split_args(N, T, f, m, C, Mcap, p_out, tau_out);
+  if (rc) return rc;
+  double total = 0.0, csum = 0.0;
+  for (int i = 0; i < N; ++i) total += f[i];
+  for (int j = 0; j < T; ++j) csum += C[j];
+  std::vector<int32_t> p(std::max(T - 1, 1), 0);
+  int next = 0;  // first block not yet assigned
+  for (int j = 0; j < T - 1; ++j) {
+    const double share = total * C[j] / csum;  // what the tier would carry if load followed capacity
+    double load = 0.0, mem = 0.0;
+    int taken = 0;
+    while (next < N - (T - 1 - j)) {  // every later tier keeps at least one block
+      const double nl = load + f[next], nm = mem + m[next];
+      if (nm > Mcap[j]) break;
+      if (taken >= 1 && nl > share) break;
+      load = nl;
+      mem = nm;
+      ++taken;
+      ++next;
+    }
+    if (taken == 0) return HYP_EINFEASIBLE;  // the tier cannot even hold its first block
+    p[j] = next;
+  }
+  double tau = 0.0;
+  if (next >= N || !evaluate_partition(p, N, T, f, m, C, Mcap, &tau)) return HYP_EINFEASIBLE;
+  for (int j = 0; j < T - 1; ++j) p_out[j] = p[j];
+  *tau_out = tau;
+  return HYP_OK;
+}

@@ -73,6 +73,12 @@ SIGNATURES = {
     "hyp_split_dp": (C.c_int, [C.c_int32, C.c_int32, C.POINTER(C.c_double), C.POINTER(C.c_double),
                                C.POINTER(C.c_double), C.POINTER(C.c_double), C.c_double, C.POINTER(C.c_int32),
                                C.POINTER(C.c_double)]),
+    "hyp_split_even": (C.c_int, [C.c_int32, C.c_int32, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                 C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int32),
+                                 C.POINTER(C.c_double)]),
+    "hyp_split_greedy": (C.c_int, [C.c_int32, C.c_int32, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                   C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int32),
+                                   C.POINTER(C.c_double)]),
     "hyp_sched_rt": (C.c_int, [C.c_double, C.c_double, C.POINTER(hyp_node_state), C.c_int32, C.POINTER(C.c_int32)]),
     "hyp_op_rmsnorm": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_float, C.c_void_p]),
     "hyp_op_weight_packed_bytes": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int32]),
@@ -250,6 +256,27 @@ def hyp_split_dp(f, m, Cap, Mcap, eps: float = 0.0):
     tau = C.c_double()
     _check(lib().hyp_split_dp(N, T, _f64(f), _f64(m), _f64(Cap), _f64(Mcap), eps, p, C.byref(tau)), "hyp_split_dp")
     return tuple(p[j] for j in range(T - 1)), tau.value
+
+
+def _split_baseline(name, f, m, Cap, Mcap, tolerate_infeasible):
+    N, T = len(f), len(Cap)
+    p = (C.c_int32 * max(T - 1, 1))()
+    tau = C.c_double()
+    code = getattr(lib(), name)(N, T, _f64(f), _f64(m), _f64(Cap), _f64(Mcap), p, C.byref(tau))
+    if not (tolerate_infeasible and code == HYP_EINFEASIBLE and N >= T):
+        _check(code, name)
+    return tuple(p[j] for j in range(T - 1)), tau.value, code == HYP_OK
+
+
+def hyp_split_even(f, m, Cap, Mcap):
+    """Equal-count contiguous partition.  Returns (p, tau, fits): fits is False if a memory limit is exceeded."""
+    return _split_baseline("hyp_split_even", f, m, Cap, Mcap, True)
+
+
+def hyp_split_greedy(f, m, Cap, Mcap):
+    """Memory-aware greedy contiguous partition.  Returns (p, tau); raises HYP_EINFEASIBLE if it finds none."""
+    p, tau, _ = _split_baseline("hyp_split_greedy", f, m, Cap, Mcap, False)
+    return p, tau
 
 
 def hyp_sched_rt(F_new: float, m_act: float, nodes) -> int:

@@ -195,6 +195,12 @@ def phi3_medium_shape(n_layers=40):
     return ModelShape(n_layers, 5120, 40, 10, 128, 17920, 32064)
 
 
+def llama3_8b_shape(n_layers=32):
+    """The paper's second evaluation model (its hardware / model table): 32 blocks, hidden 4096, grouped-query
+    attention with 32 query and 8 KV heads of 128, SwiGLU width 14336, vocabulary 128256, rotary base 500000."""
+    return ModelShape(n_layers, 4096, 32, 8, 128, 14336, 128256, rope_theta=500000.0)
+
+
 def layer_weights(shape: ModelShape, layer: int, seed: int = SEED_WEIGHTS, device="cpu",
                   random_gains: bool = False) -> dict:
     """bf16 tensors of one decoder layer, each stored [out, in] row-major.

@@ -5,6 +5,7 @@
     python -m paper_2511_14450_b200.opbench attn_prefill --batch 1 --ctx 512
     python -m paper_2511_14450_b200.opbench layer_gemms --M 512
     python -m paper_2511_14450_b200.opbench decode_stage --layers 2 --batch 8 --ctx 1024
+    python -m paper_2511_14450_b200.opbench decode_stage --shape llama3 --layers 11 --batch 8 --ctx 1024
 
 Times with CUDA events after warm-up; weights / KV pools are rotated so that no launch finds its
 operands in L2.  Prints one JSON line per case.
@@ -80,20 +81,29 @@ def attn_prefill(batch, ctx, Hq=40, Hkv=10, D=128, iters=10):
             "tflops_causal": 4.0 * batch * (ctx * (ctx + 1) / 2) * Hq * D / ms / 1e9}
 
 
-def layer_gemms(M):
-    """The four projections of one Phi-3-medium-shaped block at M rows."""
-    cases = [(7680, 5120, "bf16"), (5120, 5120, "resid"), (17920, 5120, "swiglu"), (5120, 17920, "resid")]
+def _shape(name):
+    from paper_2511_14450_b200 import inputs
+    return inputs.llama3_8b_shape() if name == "llama3" else inputs.phi3_medium_shape()
+
+
+def layer_gemms(M, shape="phi3"):
+    """The four projections of one block of the given model shape at M rows."""
+    sh = _shape(shape)
+    H, F, HD = sh.hidden, sh.ffn, sh.n_q_heads * sh.head_dim
+    cases = [(sh.qkv_rows, H, "bf16"), (H, HD, "resid"), (F, H, "swiglu"), (H, F, "resid")]
     res = [gemm(M, n, k, e) for n, k, e in cases]
     us = sum(r["us"] for r in res)
-    flops = 2.0 * M * 340_787_200
+    flops = 2.0 * M * sh.layer_linear_params
     return res + [{"op": "layer_gemms", "M": M, "us": us, "tflops": flops / us / 1e6}]
 
 
-def decode_stage(layers, batch, ctx, iters=20):
+def decode_stage(layers, batch, ctx, iters=20, shape="phi3"):
     """Decode steps of a short stage of Phi-3-medium-shaped blocks (the library's own kernel sequence, graph
     replay): a small stand-in for the benchmark's 14-block stage, e.g. for profiling one of its kernels."""
     from paper_2511_14450_b200 import inputs
-    sh = inputs.phi3_medium_shape()
+    sh = _shape(shape)
+    if shape == "llama3":
+        sh.vocab = 32768      # only the embedding gather sees it; keeps the table small
     chunk = min(ctx, 2048)
     st = hyp.Stage(sh, 0, layers, max_seqs=batch, max_ctx=ctx + iters + 16, max_tokens=chunk)
     for layer in range(layers):
@@ -119,7 +129,7 @@ def decode_stage(layers, batch, ctx, iters=20):
     ms = _time(step, iters, warmup=4)
     st.close()
     kv = layers * batch * (ctx + iters // 2) * 2 * sh.n_kv_heads * sh.head_dim * 2
-    return {"op": "decode_stage", "layers": layers, "batch": batch, "ctx": ctx, "us_per_step": ms * 1e3,
+    return {"op": "decode_stage", "shape": shape, "layers": layers, "batch": batch, "ctx": ctx, "us_per_step": ms * 1e3,
             "us_per_layer": ms * 1e3 / layers,
             "gbs": (layers * sh.layer_linear_params * 2 + kv) / ms / 1e6}
 
@@ -128,6 +138,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("op", choices=["gemm", "attn_decode", "attn_prefill", "layer_gemms", "decode_stage"])
     ap.add_argument("--layers", type=int, default=2)
+    ap.add_argument("--shape", default="phi3", choices=["phi3", "llama3"], help="model shape of layer_gemms / decode_stage")
     ap.add_argument("--M", type=int, default=8)
     ap.add_argument("--N", type=int, default=17920)
     ap.add_argument("--K", type=int, default=5120)
@@ -144,9 +155,9 @@ def main():
     elif a.op == "attn_prefill":
         out = [attn_prefill(a.batch, a.ctx, iters=a.iters)]
     elif a.op == "decode_stage":
-        out = [decode_stage(a.layers, a.batch, a.ctx, iters=a.iters)]
+        out = [decode_stage(a.layers, a.batch, a.ctx, iters=a.iters, shape=a.shape)]
     else:
-        out = layer_gemms(a.M)
+        out = layer_gemms(a.M, a.shape)
     for r in out:
         print(json.dumps(r))
 

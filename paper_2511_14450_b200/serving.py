@@ -67,6 +67,38 @@ def plan_stages(shape, n_tiers: int, batch: int = 8, ctx: int = 1024, capacity=N
     return [0] + list(p) + [N], tau, ms, nbytes
 
 
+# Relative compute capacity and memory of the paper's three device tiers (its hardware table: 67 / 157 / 200 TOPS,
+# 8 / 16 / 32 GB); the two- and four-tier rows extend the ladder the same way.
+TIER_LADDERS = {2: ([67.0, 200.0], [8.0, 32.0]), 3: ([67.0, 157.0, 200.0], [8.0, 16.0, 32.0]),
+                4: ([67.0, 157.0, 200.0, 275.0], [8.0, 16.0, 32.0, 64.0])}
+
+
+def compare_splits(f, m, n_tiers: int, slack: float = 1.25):
+    """HypSplit-DP beside the two comparison partitioners on the same per-block costs f (ms) and bytes m.
+
+    Tiers follow TIER_LADDERS; the memory limits keep the ladder's ratios and sum to `slack` x the model's bytes,
+    so that the small tier's limit can bind.  Returns one record per method: boundaries, bottleneck
+    max_j L_j(p) (in units of f / capacity) and the bottleneck relative to HypSplit-DP's."""
+    cap, mem = TIER_LADDERS[n_tiers]
+    total = float(sum(m))
+    limits = [slack * total * g / sum(mem) for g in mem]
+    mb = [float(v) for v in m]
+    N = len(f)
+    out = {}
+    p, tau = hyp.hyp_split_dp(f, mb, cap, limits)
+    out["hypsplit_dp"] = {"boundaries": [0] + list(p) + [N], "bottleneck": tau, "fits_memory": True}
+    try:
+        pg, tg = hyp.hyp_split_greedy(f, mb, cap, limits)
+        out["greedy_memory_aware"] = {"boundaries": [0] + list(pg) + [N], "bottleneck": tg, "fits_memory": True}
+    except hyp.HyperionError:
+        out["greedy_memory_aware"] = {"boundaries": None, "bottleneck": None, "fits_memory": False}
+    pe, te, fits = hyp.hyp_split_even(f, mb, cap, limits)
+    out["even_count"] = {"boundaries": [0] + list(pe) + [N], "bottleneck": te, "fits_memory": fits}
+    for rec in out.values():
+        rec["vs_hypsplit_dp"] = rec["bottleneck"] / tau if rec["bottleneck"] is not None else None
+    return {"tiers": n_tiers, "capacity": cap, "memory_limits_bytes": limits, "methods": out}
+
+
 class PipelineEngine:
     def __init__(self, shape, boundaries, max_seqs: int, max_ctx: int, max_tokens: int, random_gains: bool = False):
         assert boundaries[0] == 0 and boundaries[-1] == shape.n_layers_total
@@ -233,7 +265,8 @@ def synthetic_requests(shape, n: int, rate: float, len_lo: int, len_hi: int, n_o
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--mode", choices=["closed", "replay"], default="closed")
+    ap.add_argument("--mode", choices=["closed", "replay", "compare-splits"], default="closed")
+    ap.add_argument("--shape", choices=["phi3", "llama3"], default="phi3")
     ap.add_argument("--requests", type=int, default=32)
     ap.add_argument("--rate", type=float, default=4.0)
     ap.add_argument("--len-lo", type=int, default=128)
@@ -242,6 +275,13 @@ def main():
     ap.add_argument("--tiers", type=int, default=3)
     ap.add_argument("--layers", type=int, default=40)
     a = ap.parse_args()
+    if a.mode == "compare-splits":
+        # measured per-block decode cost of the whole model, then the three partitioners on 2, 3 and 4 tiers
+        shape = inputs.llama3_8b_shape() if a.shape == "llama3" else inputs.phi3_medium_shape()
+        _, _, ms, nbytes = plan_stages(shape, 1)
+        print(json.dumps({"shape": a.shape, "blocks": shape.n_layers_total, "block_ms_min_max": [min(ms), max(ms)],
+                          "splits": [compare_splits(ms, nbytes, t) for t in (2, 3, 4)]}))
+        return
     shape = inputs.phi3_medium_shape(a.layers)
     bounds, tau, ms, nbytes = plan_stages(shape, a.tiers)
     eng = PipelineEngine(shape, bounds, max_seqs=a.requests, max_ctx=a.len_hi + a.n_out + 16, max_tokens=2048)

@@ -122,3 +122,41 @@ def test_config4_shape_40_blocks_with_head_prompt_512():
 def test_config4_full_size_prompt_2048():
     """configs[4] at full size: batch 4, 2048-token prompts (8192 rows in one prefill call), first decode steps."""
     _full_model_case(prompt_len=2048, steps=2)
+
+
+def test_llama3_8b_shaped_blocks_prefill_and_batched_decode():
+    """The paper's other model shape (32 blocks, hidden 4096, 32 / 8 heads, FFN 14336, rotary base 500000): two
+    blocks, two ragged prompts in one prefill call, then three batched decode steps; stage output against the
+    oracle, and the logits criterion through a seeded 4096-way probe head."""
+    sh = inputs.llama3_8b_shape()
+    sh.vocab = 16384          # only the embedding gather sees it: a 128256-row table would cost the oracle 4 GB
+    lens, steps = [300, 77], 3
+    st = H.gpu_stage(sh, 0, 2, max_seqs=2, max_ctx=320, max_tokens=sum(lens))
+    seqs = [inputs.token_ids(inputs.SEED_PROMPTS, 600 + i, lens[i] + steps, sh.vocab) for i in range(2)]
+    want = [H.oracle_stage(sh, 0, 2, s.numpy()) for s in seqs]
+    out = torch.empty(sum(lens), sh.hidden, dtype=torch.float32, device="cuda")
+    st.prefill([0, 1], lens, [0, 0], torch.cat([s[:l] for s, l in zip(seqs, lens)]).cuda(), out,
+               flags=hyp.HYP_BATCH_ALL_LOGITS)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy().astype(np.float64)
+    probe = inputs.ModelShape(32, sh.hidden, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.ffn, 4096)
+    gf, wlm = (inputs.bf16_bits_to_f64(t) for t in inputs.head_weights(probe))
+    row = 0
+    for i, l in enumerate(lens):
+        H.assert_hidden_close(got[row:row + l], want[i][:l], f"llama3 prefill seq {i}")
+        pick = np.arange(row, row + l, 9)
+        H.assert_logits_close(od.lm_head(got[pick], gf, wlm, sh.rms_eps),
+                              od.lm_head(want[i][pick - row], gf, wlm, sh.rms_eps), f"llama3 prefill probe seq {i}")
+        row += l
+    dec = torch.empty(2, sh.hidden, dtype=torch.float32, device="cuda")
+    for s_ in range(steps):
+        tok = torch.stack([seqs[i][lens[i] + s_] for i in range(2)]).cuda()
+        st.decode([0, 1], [l + s_ for l in lens], tok, dec)
+        torch.cuda.synchronize()
+        g = dec.cpu().numpy().astype(np.float64)
+        for i in range(2):
+            w = want[i][lens[i] + s_][None]
+            H.assert_hidden_close(g[i:i + 1], w, f"llama3 decode step {s_} seq {i}")
+            H.assert_logits_close(od.lm_head(g[i:i + 1], gf, wlm, sh.rms_eps), od.lm_head(w, gf, wlm, sh.rms_eps),
+                                  f"llama3 decode probe step {s_} seq {i}")
+    st.close()

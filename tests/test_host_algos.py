@@ -141,3 +141,51 @@ def test_packed_weight_size_and_tuning_switch_ranges():
     assert L.hyp_tune(hyp.HYP_TUNE_PDL, 4) == hyp.HYP_EINVAL and L.hyp_tune(hyp.HYP_TUNE_STREAM_SLOTS, 9) == hyp.HYP_EINVAL
     assert L.hyp_tune(hyp.HYP_TUNE_ATTN_SPLITS, 9) == hyp.HYP_EINVAL and L.hyp_tune(99, 0) == hyp.HYP_EINVAL
     assert L.hyp_tune(hyp.HYP_TUNE_STREAM_SLOTS, 0) == hyp.HYP_OK
+
+
+def test_baseline_partitioners_equal_the_oracle():
+    """hyp_split_even / hyp_split_greedy against the oracle's versions on seeded instances (bit-exact boundaries),
+    infeasible cases included, and never better than hyp_split_dp."""
+    r = np.random.default_rng(11)
+    n_inf = 0
+    for trial in range(400):
+        N, T = int(r.integers(1, 13)), int(r.integers(1, 5))
+        if N < T:
+            continue
+        f = [float(x) for x in np.floor(r.uniform(1, 9, N))]
+        m = [float(x) for x in np.floor(r.uniform(1, 4, N))]
+        Cp = [float(x) for x in np.floor(r.uniform(1, 4, T))]
+        M = [float(x) for x in np.floor(r.uniform(3, 20, T))]
+        p, tau, fits = hyp.hyp_split_even(f, m, Cp, M)
+        assert p == osp.split_even(N, T) and fits == osp.memory_feasible(p, m, M)
+        assert tau == max(osp.tier_loads(p, f, Cp))
+        want = osp.split_greedy(f, m, Cp, M)
+        if want is None:
+            n_inf += 1
+            with pytest.raises(hyp.HyperionError) as ei:
+                hyp.hyp_split_greedy(f, m, Cp, M)
+            assert ei.value.code == hyp.HYP_EINFEASIBLE
+        else:
+            pg, tg = hyp.hyp_split_greedy(f, m, Cp, M)
+            assert pg == want and tg == max(osp.tier_loads(pg, f, Cp))
+            assert tg >= hyp.hyp_split_dp(f, m, Cp, M)[1]
+    assert n_inf > 10
+    with pytest.raises(hyp.HyperionError):
+        hyp.hyp_split_greedy([1.0, 2.0], [1.0, 1.0], [1.0, 0.0], [9.0, 9.0])      # zero capacity
+
+
+def test_compare_splits_report_on_uneven_costs():
+    """The serving tool's comparison of the three partitioners (host logic only): HypSplit-DP is never worse, the
+    ratios are reported against it, and a first block heavier than the small tier's share shows the greedy gap."""
+    from paper_2511_14450_b200 import serving
+    f = [9.0, 1.0, 1.0, 1.0, 5.0, 1.0, 1.0, 1.0, 1.0, 3.0, 1.0, 1.0]
+    m = [1.0] * 12
+    for tiers in (2, 3, 4):
+        rep = serving.compare_splits(f, m, tiers)
+        meth = rep["methods"]
+        assert meth["hypsplit_dp"]["vs_hypsplit_dp"] == 1.0 and len(meth["hypsplit_dp"]["boundaries"]) == tiers + 1
+        for name in ("greedy_memory_aware", "even_count"):
+            if meth[name]["bottleneck"] is not None and meth[name]["fits_memory"]:
+                assert meth[name]["vs_hypsplit_dp"] >= 1.0
+        assert abs(sum(rep["memory_limits_bytes"]) - 1.25 * 12) < 1e-9
+    assert serving.compare_splits(f, m, 3)["methods"]["even_count"]["vs_hypsplit_dp"] > 1.0

@@ -154,3 +154,42 @@ def test_sched_rt_scan_equals_argmin_definition_and_hand_cases():
                "F_wait": [float(v) for v in r.integers(0, 6, int(r.integers(0, 4)))],
                "available": bool(r.integers(0, 4))} for _ in range(K)]
         assert osp.hypsched_rt_scan(3.0, 2.0, nd) == osp.sched_rt_argmin(3.0, 2.0, nd)
+
+
+def test_baseline_partitioners_hand_worked_and_dominated_by_the_optimum():
+    """The two comparison partitioners (Section V names them; the readings are in the oracle's header).
+    Hand-worked cases, structural properties, and: neither can beat the exact optimum."""
+    # even: sizes differ by at most one, longer segments first
+    assert osp.split_even(40, 3) == (14, 27) and osp.split_even(8, 3) == (3, 6) and osp.split_even(6, 3) == (2, 4)
+    assert osp.split_even(5, 1) == () and osp.split_even(4, 4) == (1, 2, 3)
+    # greedy by hand: f = 4,1,1,4,1,1; C = (1,1,1): share 4 each.  Tier 1 takes block 1 (load 4; a second
+    # block would exceed 4).  Tier 2 takes 1,1 (load 2; the next block, 4, would exceed).  p = (1, 3).
+    assert osp.split_greedy([4, 1, 1, 4, 1, 1], [1] * 6, [1, 1, 1], [9, 9, 9]) == (1, 3)
+    # capacities 1:3 -> shares 3 and 9 of a total of 12: tier 1 stops after 3 unit blocks
+    assert osp.split_greedy([1] * 12, [1] * 12, [1, 3], [99, 99]) == (3,)
+    # memory binds before the share does: tier 1 may hold only 2 blocks
+    assert osp.split_greedy([1] * 12, [1] * 12, [3, 1], [2, 99]) == (2,)
+    # the last tier cannot hold what is left -> no partition; a first block that does not fit -> none
+    assert osp.split_greedy([1] * 12, [1] * 12, [1, 1], [6, 3]) is None
+    assert osp.split_greedy([1, 1, 1], [5, 1, 1], [1, 1], [4, 9]) is None
+    # every later tier keeps a block even when the shares would starve it
+    assert osp.split_greedy([1, 1, 1], [1, 1, 1], [100, 1, 1], [9, 9, 9]) == (1, 2)
+    # uniform blocks, equal tiers, N divisible by T: greedy = even = optimal
+    for N, T in [(6, 3), (12, 4), (10, 5)]:
+        f, m, C, M = [2.0] * N, [1.0] * N, [1.0] * T, [1e9] * T
+        assert osp.split_greedy(f, m, C, M) == osp.split_even(N, T) == osp.enumerate_split(f, m, C, M)[0]
+    r = np.random.default_rng(5)
+    for trial in range(200):
+        N, T = int(r.integers(3, 11)), int(r.integers(2, 4))
+        f = list(np.floor(r.uniform(1, 9, N)))
+        m = list(np.floor(r.uniform(1, 4, N)))
+        C = list(np.floor(r.uniform(1, 4, T)))
+        M = list(np.floor(r.uniform(4, 20, T)))
+        opt = osp.enumerate_split(f, m, C, M)
+        for p in (osp.split_greedy(f, m, C, M), osp.split_even(N, T)):
+            if p is None or not osp.memory_feasible(p, m, M):
+                continue
+            assert list(p) == sorted(set(p)) and 1 <= p[0] and p[-1] < N     # a valid partition vector
+            assert opt is not None and max(osp.tier_loads(p, f, C)) >= opt[1]
+        g = osp.split_greedy(f, m, C, M)
+        assert g is None or osp.memory_feasible(g, m, M)                      # greedy never breaks a limit
