@@ -160,3 +160,29 @@ def test_llama3_8b_shaped_blocks_prefill_and_batched_decode():
             H.assert_logits_close(od.lm_head(g[i:i + 1], gf, wlm, sh.rms_eps), od.lm_head(w, gf, wlm, sh.rms_eps),
                                   f"llama3 decode probe step {s_} seq {i}")
     st.close()
+
+
+@pytest.mark.parametrize("B", [12, 24, 40])
+def test_phi3_shaped_blocks_decode_batches_beyond_8(B):
+    """Decode batches that leave the weight-streaming kernel (9-128 rows: tile kernel with stream-K, swapped-operand
+    kernel for q/k/v) at the Phi-3-medium shape, through the stage path and its graph replay: two blocks, ragged
+    prompt lengths, four steps; three sampled sequences against the oracle."""
+    sh = inputs.phi3_medium_shape()
+    steps = 4
+    lens = [17 + (11 * b) % 90 for b in range(B)]
+    st = H.gpu_stage(sh, 0, 2, max_seqs=B, max_ctx=128, max_tokens=sum(lens))
+    seqs = [inputs.token_ids(inputs.SEED_PROMPTS, 700 + b, lens[b] + steps, sh.vocab) for b in range(B)]
+    hid = torch.empty(sum(lens), sh.hidden, dtype=torch.float32, device="cuda")
+    st.prefill(list(range(B)), lens, [0] * B, torch.cat([s[:l] for s, l in zip(seqs, lens)]).cuda(), hid)
+    out = torch.empty(B, sh.hidden, dtype=torch.float32, device="cuda")
+    got = []
+    for s_ in range(steps):
+        tok = torch.stack([seqs[b][lens[b] + s_] for b in range(B)]).cuda()
+        st.decode(list(range(B)), [l + s_ for l in lens], tok, out)
+        torch.cuda.synchronize()
+        got.append(out.cpu().numpy().astype(np.float64))
+    st.close()
+    for b in (0, B // 2, B - 1):
+        want = H.oracle_stage(sh, 0, 2, seqs[b].numpy())
+        for s_ in range(steps):
+            H.assert_hidden_close(got[s_][b:b + 1], want[lens[b] + s_][None], f"batch {B} seq {b} step {s_}")
