@@ -1,14 +1,16 @@
 // Prefill attention over the paged KV cache: causal, grouped-query, fp32 online softmax.
 //
 // Flash-attention tiling on tensor cores: one CTA = 64 query rows of one sequence and one query head
-// (4 warps x 16 rows); keys/values stream through shared memory in 64-token tiles (4 pages) with
-// double-buffered cp.async; S = Q K^T and O += P V run on mma.sync.m16n8k16 (fp16 in, fp32 accumulate: q, k,
+// (4 warps x 16 rows); keys/values stream through shared memory in 64-token tiles (4 pages), double-buffered,
+// one bulk copy per page and operand (the cache keeps a page's rows in the tile's chunk-permuted order); S = Q K^T and O += P V run on mma.sync.m16n8k16 (fp16 in, fp32 accumulate: q, k,
 // v and the softmax weights carry 11 mantissa bits - bf16's 8 bits alone cost ~0.5 % error in the softmax
 // weights), the probabilities never leave registers.  New rows of a sequence sit at positions
 // ctx_len .. ctx_len + q_len - 1 and see every cached position up to their own (their k, v were
 // appended by the RoPE / KV-write kernel beforehand), so chunked prefill needs no special case.
 #include "attn_common.cuh"
 #include "hyperion.h"
+#include "gemm_tc.cuh"
+#include "sm100_common.cuh"
 
 namespace hyp {
 
@@ -17,9 +19,9 @@ namespace {
 constexpr int FA_BQ = 64, FA_BKV = 64, FA_THREADS = 128, PT = 16;
 
 template <int D>
-__global__ void __launch_bounds__(FA_THREADS)
+__global__ void __launch_bounds__(FA_THREADS, 3)
 attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict__ kv_layer,
-                       __half* __restrict__ out, BatchMeta bm, ModelDims d) {
+                       __half* __restrict__ out, BatchMeta bm, ModelDims d, int* __restrict__ err) {
   constexpr int KS = D / 16;       // k-steps of the QK^T contraction
   constexpr int DN = D / 8;        // 8-wide output column tiles of O
   constexpr int CPR = D / 8;       // 16-byte chunks per K/V row
@@ -30,10 +32,12 @@ attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict_
   auto k_tile = [&](int buf) { return smem0 + buf * TILE_BYTES; };
   auto v_tile = [&](int buf) { return smem0 + (2 + buf) * TILE_BYTES; };
 
+  __shared__ uint64_t kv_bars[2];
+  constexpr int PAGE_BYTES = PT * D * 2;  // the 16 keys (or values) of one page and KV head: contiguous in the cache
   pdl_trigger();
   pdl_wait();
-  // which (sequence, query tile) is this CTA?
-  int t = blockIdx.x, seq = -1, q0 = 0, q_len = 0;
+  // which (sequence, query tile) is this CTA?  The last tiles of a sequence see the most keys: they go first.
+  int t = (int)gridDim.x - 1 - (int)blockIdx.x, seq = -1, q0 = 0, q_len = 0;
   for (int i = 0; i < bm.n_seqs; ++i) {
     const int ql = bm.cu_q[i + 1] - bm.cu_q[i];
     const int nt = (ql + FA_BQ - 1) / FA_BQ;
@@ -55,24 +59,38 @@ attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, tq = lane & 3;
 
+  // One tile = 4 pages.  The cache stores a page's rows with the tile's own chunk permutation, so thread 0 brings a
+  // tile in with one bulk copy per page for the keys and one for the values; pages past the sequence's last one
+  // are not copied but cleared (their probabilities are zero, and 0 x stale bits must not become NaN).
+  const int n_pages_seq = (kv_total + PT - 1) / PT;
+  const uint32_t bar0 = smem_u32(kv_bars);
+  if (threadIdx.x == 0) {
+    mbar_init(bar0, 1);
+    mbar_init(bar0 + 8, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
   auto load_kv_tile = [&](int j, int buf) {
-    // 64 keys x CPR chunks for K and the same for V; 128 threads
-    for (int idx = threadIdx.x; idx < FA_BKV * CPR; idx += FA_THREADS) {
-      const int r = idx / CPR, c = idx % CPR;
-      const int key = j * FA_BKV + r;
-      const bool ok = key < kv_total;
-      const int kk = ok ? key : 0;
-      const __half* src =
-          kv_layer + (size_t)bt[kk / PT] * page_elems + ((size_t)kvh * PT + (kk % PT)) * D + c * 8;
-      // the cache row is stored with the tile's own chunk permutation (tiles start on page boundaries, so
-      // r & 7 is the token's slot & 7): chunk positions copy one to one
-      cp_async16(k_tile(buf) + r * (D * 2) + c * 16, src, ok);
-      cp_async16(v_tile(buf) + r * (D * 2) + c * 16, src + v_off, ok);
+    const int p0 = j * (FA_BKV / PT);
+    const int n_valid = min(FA_BKV / PT, n_pages_seq - p0);
+    if (threadIdx.x == 0) {
+      mbar_expect_tx(bar0 + 8u * buf, (uint32_t)(2 * n_valid * PAGE_BYTES));
+      for (int pi = 0; pi < n_valid; ++pi) {
+        const __half* src = kv_layer + (size_t)bt[p0 + pi] * page_elems + (size_t)kvh * PT * D;
+        bulk_load(k_tile(buf) + pi * PAGE_BYTES, src, PAGE_BYTES, bar0 + 8u * buf);
+        bulk_load(v_tile(buf) + pi * PAGE_BYTES, src + v_off, PAGE_BYTES, bar0 + 8u * buf);
+      }
+    }
+    if (n_valid < FA_BKV / PT) {
+      const int bytes = (FA_BKV / PT - n_valid) * PAGE_BYTES;
+      for (int o = threadIdx.x * 16; o < bytes; o += FA_THREADS * 16) {
+        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(k_tile(buf) + n_valid * PAGE_BYTES + o), "r"(0u) : "memory");
+        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(v_tile(buf) + n_valid * PAGE_BYTES + o), "r"(0u) : "memory");
+      }
     }
   };
 
   load_kv_tile(0, 0);
-  cp_async_commit();
 
   // Q fragments of this warp's 16 rows, straight from global memory
   uint32_t qf[KS][4];
@@ -100,12 +118,14 @@ attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict_
   for (int i = 0; i < DN; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
   float m_lo = -1e30f, m_hi = -1e30f, l_lo = 0.f, l_hi = 0.f;
 
+  bool ok = true;
   for (int j = 0; j < n_kv_tiles; ++j) {
     const int buf = j & 1;
     if (j + 1 < n_kv_tiles) load_kv_tile(j + 1, buf ^ 1);
-    cp_async_commit();
-    cp_async_wait<1>();
-    __syncthreads();
+    const bool landed = mbar_wait(bar0 + 8u * buf, (uint32_t)((j >> 1) & 1), nullptr);
+    // one decision for the whole CTA (a bounded wait could expire for some threads only); as a barrier it also
+    // makes the cleared pages of a last tile visible
+    if (!__syncthreads_and(landed)) { ok = false; break; }
 
     // ---- S = Q K^T (16 rows x 64 keys per warp) ----
     float s[8][4];
@@ -183,7 +203,11 @@ attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict_
     }
     __syncthreads();  // everyone is done with `buf` before the next iteration's loads overwrite it
   }
-  cp_async_wait<0>();
+  if (!ok) {
+    // a copy never landed (bounded wait expired): record it; the rows of this tile are not written
+    if (threadIdx.x == 0) atomicCAS(err, 0, 12);
+    return;
+  }
 
   // row sums live spread over the 4 lanes of a quad
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
@@ -208,6 +232,8 @@ int launch_fa(const __half* qkv, const __half* kv_layer, __half* attn_out, const
               const ModelDims& d, cudaStream_t st) {
   static bool configured = false;
   constexpr int smem = 4 * FA_BKV * D * 2;
+  int rc = tc_prepare();  // the device word that bounded waits report to
+  if (rc) return rc;
   if (!configured) {
     HYP_CUDA_TRY(cudaFuncSetAttribute(attn_prefill_fa_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     configured = true;
@@ -215,7 +241,7 @@ int launch_fa(const __half* qkv, const __half* kv_layer, __half* attn_out, const
   // every sequence adds at most one ragged tile on top of floor(rows / 64)
   const int max_tiles = bm.n_tokens / FA_BQ + bm.n_seqs;
   HYP_CUDA_TRY(launch_pdl(attn_prefill_fa_kernel<D>, dim3(max_tiles, d.Hq), dim3(FA_THREADS), smem, st, qkv, kv_layer,
-                          attn_out, bm, d));
+                          attn_out, bm, d, tc_err_flag_ptr()));
   return 1;
 }
 
