@@ -31,7 +31,7 @@
  *    the softmax weights are fp16 (values saturate at +-65504).  With bf16 activations instead, their
  *    8 mantissa bits alone put the per-step logits of the 5120-wide 40-block model outside the 5e-2
  *    tolerance.
- *  - Prefill rows: the residual projections split K across CTAs for row counts up to 4096 and add
+ *  - Prefill rows: the residual projections split K across CTAs for row counts up to 2048 and add
  *    partial sums with floating-point atomics, so the last bits of a prefill result may differ from
  *    run to run; decode is bit-reproducible.
  */

@@ -613,9 +613,10 @@ int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
   }
   constexpr int BN_OUT = EPI == EPI_SWIGLU_BF16 ? BN / 2 : BN;
   const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN_OUT - 1) / BN_OUT;
-  // two-CTA tiles (a third less shared-memory fill per flop) from 129 rows on; the residual epilogue up to 4096 rows
-  // (stream-K), beyond that whole one-CTA tiles balance by themselves
-  if (tiles_m >= 2 && (EPI != EPI_RESID_F32 || tiles_m <= 32)) return launch_pair<EPI>(act, w, M, N, K, out, ldo, st, num_sms, early);
+  // two-CTA tiles (a third less shared-memory fill per flop) from 129 rows on; the residual epilogue only up to 1024
+  // rows: measured on B200 (N 5120, K 17920) the pair kernel's stream-K takes 75 / 154 us at 512 / 1024 rows against
+  // 79 / 161 for one-CTA stream-K, but 359 / 679 against 299 / 590 at 2048 / 4096 rows
+  if (tiles_m >= 2 && (EPI != EPI_RESID_F32 || tiles_m <= 8)) return launch_pair<EPI>(act, w, M, N, K, out, ldo, st, num_sms, early);
   int grid, team = 0;  // team 0 = whole tiles per CTA
   if (EPI == EPI_RESID_F32 && tiles_m <= 16) {
     // stream-K (up to 2048 rows; beyond that whole tiles already balance and reuse A better): pick the team size (a divisor of tiles_m) that keeps most SMs busy, larger teams preferred
