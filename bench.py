@@ -306,7 +306,7 @@ def run_ours(args):
                          "frac": (achieved / peak) if achieved else None, "peak_source": f"of {peak_src}",
                          "bytes_per_launch": gu_bytes, "launches_timed": n_k,
                          "avg_launch_us": (k_ms / n_k * 1e3) if n_k else None,
-                         "traffic": 371.5e6,   # dram read + write per launch, profiles/gemm_stream_gateup_M8.md
+                         "traffic": 371.2e6,   # dram read + write per launch, profiles/gemm_stream_gateup_M8.md
                          "timed_in": "second pass of K steps with per-launch events (kernel-by-kernel launches)",
                          "kernel_pass_ms_per_step": kernel_pass_ms},
             "step_roofline": {"bound": "hbm", "bytes_per_step": step_bytes, "achieved": step_gbs, "peak": peak,
@@ -377,7 +377,7 @@ def prefill_config1(torch, hyp, inputs, stream, iters=10):
                      "peak_source": "of measured (burst)" if peaks else "of fallback",
                      "frac_of_nominal_2250": achieved / 2250.0, "flops": gemm_flops,
                      "dominant_kernel_tflops": gu, "dominant_kernel_frac": gu / peak,
-                     "traffic": 401.0e6},  # gate/up launch, dram read + write, profiles/gemm_tc2_gateup_M512.md
+                     "traffic": 401.7e6},  # gate/up launch, dram read + write, profiles/gemm_tc2_gateup_M512.md
     }
 
 
