@@ -39,14 +39,6 @@ __device__ __forceinline__ float warp_max(float v) {
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
   return v;
 }
-// 128-bit streaming load that does not pollute L1 (weights are read exactly once per step).
-__device__ __forceinline__ uint4 ldg_stream(const void* p) {
-  uint4 r;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-               : "l"(p));
-  return r;
-}
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
                                                uint32_t a3, uint32_t b0, uint32_t b1) {
   asm volatile(
@@ -158,8 +150,6 @@ int launch_copy_f32(const float* src, float* dst, size_t n, cudaStream_t st);
 int launch_rmsnorm(const float* x, const __nv_bfloat16* g, void* h, bool out_f16, int M, int H, float eps,
                    const int32_t* row_index /* optional gather of rows, may be null */, cudaStream_t st,
                    bool gains_are_constant = false /* true: g is a loaded weight, never a predecessor's output */);
-// dst[i] = fp16(src[i]) (exact for |x| >= 2^-17, saturating at +-65504)
-int launch_bf16_to_f16(const __nv_bfloat16* src, __half* dst, size_t n, cudaStream_t st);
 // rotate q, k of every row (fp32 in), write q as fp16 [M, Hq*D] and append k, v as fp16 to the pages
 int launch_rope_kv_write(const float* qkv, __half* q16, __half* kv_layer, const float2* rope_table,
                          const BatchMeta& bm, const ModelDims& d, cudaStream_t st);

@@ -120,19 +120,6 @@ int launch_rmsnorm(const float* x, const __nv_bfloat16* g, void* h, bool out_f16
   return 1;
 }
 
-__global__ void bf16_to_f16_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n8) {
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x) {
-    const uint4 v = src[i];
-    dst[i] = make_uint4(pack_f16_sat(bf16_lo(v.x), bf16_hi(v.x)), pack_f16_sat(bf16_lo(v.y), bf16_hi(v.y)),
-                        pack_f16_sat(bf16_lo(v.z), bf16_hi(v.z)), pack_f16_sat(bf16_lo(v.w), bf16_hi(v.w)));
-  }
-}
-
-int launch_bf16_to_f16(const __nv_bfloat16* src, __half* dst, size_t n, cudaStream_t st) {
-  bf16_to_f16_kernel<<<148 * 8, 256, 0, st>>>(reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(dst), n / 8);
-  return 1;
-}
-
 // Rotate q and k of every new row by its position and append k, v to the sequence's pages.
 // Input row layout (fp32, straight from the projection's accumulators): [Q heads | K heads | V heads],
 // each head D wide.  Outputs are fp16 (rounded once): q to its own [M, Hq*D] buffer, k and v to the pages.
