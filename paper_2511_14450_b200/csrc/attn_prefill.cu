@@ -37,7 +37,7 @@ attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict_
   pdl_trigger();
   pdl_wait();
   // which (sequence, query tile) is this CTA?  The last tiles of a sequence see the most keys: they go first.
-  int t = (int)gridDim.x - 1 - (int)blockIdx.x, seq = -1, q0 = 0, q_len = 0;
+  int t = (int)gridDim.y - 1 - (int)blockIdx.y, seq = -1, q0 = 0, q_len = 0;
   for (int i = 0; i < bm.n_seqs; ++i) {
     const int ql = bm.cu_q[i + 1] - bm.cu_q[i];
     const int nt = (ql + FA_BQ - 1) / FA_BQ;
@@ -45,7 +45,7 @@ attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict_
     t -= nt;
   }
   if (seq < 0) return;
-  const int hq = blockIdx.y;
+  const int hq = blockIdx.x;  // heads vary fastest: every head's heaviest tile is scheduled before any lighter one
   const int kvh = hq / (d.Hq / d.Hkv);
   const int ctx = bm.ctx_lens[seq];
   const int row_base = bm.cu_q[seq] + q0;               // first packed row of this tile
@@ -240,7 +240,7 @@ int launch_fa(const __half* qkv, const __half* kv_layer, __half* attn_out, const
   }
   // every sequence adds at most one ragged tile on top of floor(rows / 64)
   const int max_tiles = bm.n_tokens / FA_BQ + bm.n_seqs;
-  HYP_CUDA_TRY(launch_pdl(attn_prefill_fa_kernel<D>, dim3(max_tiles, d.Hq), dim3(FA_THREADS), smem, st, qkv, kv_layer,
+  HYP_CUDA_TRY(launch_pdl(attn_prefill_fa_kernel<D>, dim3(d.Hq, max_tiles), dim3(FA_THREADS), smem, st, qkv, kv_layer,
                           attn_out, bm, d, tc_err_flag_ptr()));
   return 1;
 }

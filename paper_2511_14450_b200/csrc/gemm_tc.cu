@@ -706,6 +706,27 @@ int tc_pack_weight(const void* src, void* dst, int rows, int halves, int K, bool
   return 1;
 }
 
+// One block's KV page pool [pages][K, V][Hkv][16 tokens][D] fp16 seen as a matrix of D-wide rows; box = 16 rows (one
+// page of one head) x 64 columns.  The rows are stored chunk-permuted inside each 128-byte half, so such a box lands
+// in shared memory as a 128-byte-swizzled operand tile without any swizzle in the copy.
+int tc_make_kv_map(CUtensorMap* map, const void* kv_layer, size_t n_pages, int Hkv, int D) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return HYP_ECUDA;
+  if (D != 128 || ((uintptr_t)kv_layer & 15) != 0 || n_pages < 1) return HYP_EINVAL;
+  const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)(n_pages * 2 * (size_t)Hkv * 16)};
+  const cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+  const cuuint32_t box[2] = {64u, 16u};
+  const cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, (void*)kv_layer, dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error((int)r);
+    return HYP_ECUDA;
+  }
+  return HYP_OK;
+}
+
 // Activations: 128-row boxes for the tile kernels, 16/32/64-row boxes for the swapped-operand kernel.
 int tc_make_act(TcAct* a, const void* ptr, int rows, int K, bool f16) {
   a->ptr = ptr; a->rows = rows; a->K = K; a->f16 = f16;

@@ -43,6 +43,13 @@ struct TcAct {
 };
 int tc_make_act(TcAct* a, const void* ptr, int rows, int K, bool f16 = false);
 
+// Tensor map over one block's KV page pool for the tcgen05 prefill attention (head_dim 128).
+int tc_make_kv_map(CUtensorMap* map, const void* kv_layer, size_t n_pages, int Hkv, int D);
+// Prefill attention on tcgen05 (head_dim 128); q_map = TcAct::map of the rotated-query buffer.
+int& attn_prefill_tc_enabled();
+int launch_attn_prefill_tc(const CUtensorMap& q_map, const CUtensorMap& kv_map, __half* attn_out, const BatchMeta& bm,
+                           const ModelDims& d, cudaStream_t st);
+
 // One-time set-up of the device-side error word (allocates; call from stage creation, not from the hot path).
 int tc_prepare();
 // Reads the error word (synchronises the device): 0 = no kernel gave up on a wait.

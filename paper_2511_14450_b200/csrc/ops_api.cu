@@ -78,6 +78,9 @@ extern "C" int hyp_tune(int32_t key, int32_t value) {
       if (value < 0 || value > 15) return HYP_EINVAL;
       gemm_swap_epilogues() = value;
       return HYP_OK;
+    case HYP_TUNE_PREFILL_ATTN_TC:
+      attn_prefill_tc_enabled() = value != 0;
+      return HYP_OK;
     case HYP_TUNE_ATTN_SPLITS:
       if (value < 0 || value > 8) return HYP_EINVAL;
       attn_fused_splits_override() = value;
@@ -174,6 +177,16 @@ extern "C" int hyp_op_attn_prefill(const hyp_attn_shape* shape, int32_t n_seqs, 
   bm.ctx_lens = ctx_lens;
   bm.block_table = block_table;
   const ModelDims d = attn_dims(shape, q_stride);
+  if (attn_prefill_tc_enabled() && d.D == 128 && ((uintptr_t)q & 15) == 0) {
+    // descriptors over the caller's buffers; the pool's size is not known here and only bounds the descriptor
+    TcAct qa;
+    CUtensorMap kvm;
+    int rc = tc_make_act(&qa, q, M, q_stride, true);
+    if (!rc) rc = tc_make_kv_map(&kvm, kv_pages, (size_t)1 << 20, d.Hkv, d.D);
+    if (rc) return rc;
+    ModelDims dd = d;
+    return finish(launch_attn_prefill_tc(qa.map, kvm, (__half*)out, bm, dd, (cudaStream_t)stream));
+  }
   return finish(launch_attn_prefill((const __half*)q, q_stride, (const __half*)kv_pages, (__half*)out, bm, d,
                                     (cudaStream_t)stream));
 }

@@ -56,7 +56,8 @@ struct hyp_stage {
   float* qkv32 = nullptr;             // q | k | v straight from the projection's accumulators
   __half* q16 = nullptr;              // rotated queries
   __half *h = nullptr, *attn = nullptr, *u = nullptr;  // projection inputs (fp16)
-  TcAct tc_h, tc_attn, tc_u;
+  TcAct tc_h, tc_attn, tc_u, tc_q16;
+  std::vector<CUtensorMap> kv_maps;  // per block: the page pool as rows (tcgen05 prefill attention, head_dim 128)
   int max_splits = 8;
   float2* rope_table = nullptr;
   size_t workspace_bytes = 0;
@@ -297,7 +298,10 @@ int run_blocks(hyp_stage* s, const BatchMeta& bm, bool decode, int n_splits, cud
                                                         2, tc_err_flag_ptr(), bm, d, st));
     } else {
       HYP_LAUNCH_T(HYP_K_ROPE, launch_rope_kv_write(s->qkv32, s->q16, kv_layer, s->rope_table, bm, d, st));
-      HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_prefill(s->q16, d.Hq * d.D, kv_layer, s->attn, bm, d, st));
+      if (attn_prefill_tc_enabled() && !s->kv_maps.empty())
+        HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_prefill_tc(s->tc_q16.map, s->kv_maps[li], s->attn, bm, d, st));
+      else
+        HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_prefill(s->q16, d.Hq * d.D, kv_layer, s->attn, bm, d, st));
     }
     HYP_LAUNCH_T(HYP_K_GEMM_O, project(s, s->tc_attn, nullptr, d.Hq * d.D, lw.tc_o, nullptr, d.H, d.Hq * d.D, M,
                                        EPI_RESID_F32, s->x, d.H, st));
@@ -609,6 +613,12 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
   TRY(tc_make_act(&s->tc_h, s->h, (int)rows_pad, d.H, true));
   TRY(tc_make_act(&s->tc_attn, s->attn, (int)rows_pad, d.Hq * d.D, true));
   TRY(tc_make_act(&s->tc_u, s->u, (int)rows_pad, d.F, true));
+  TRY(tc_make_act(&s->tc_q16, s->q16, (int)rows_pad, d.Hq * d.D, true));
+  if (d.D == 128) {
+    s->kv_maps.resize(s->L);
+    for (int li = 0; li < s->L; ++li)
+      TRY(tc_make_kv_map(&s->kv_maps[li], s->kv_pool + (size_t)li * s->kv_layer_elems, (size_t)s->n_pages, d.Hkv, d.D));
+  }
   for (LayerW& lw : s->layers) {
     // all projection matrices are held packed as fp16, see hyp_stage_load
     TRY(tc_make_weight(&lw.tc_qkv, lw.wqkv, d.qkv_rows, 1, d.H, true));

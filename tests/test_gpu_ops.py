@@ -217,6 +217,26 @@ def test_attn_decode_rejects_small_scratch():
     assert ei.value.code == hyp.HYP_ECAPACITY
 
 
+@pytest.mark.parametrize("Hq,Hkv", [(40, 10), (8, 8), (8, 1)])
+@pytest.mark.parametrize("lens,new", [([37, 5, 64], [37, 2, 20]), ([300, 129, 1, 64], [300, 65, 1, 64]),
+                                      ([700, 128, 257], [700, 128, 130])])
+def test_attn_prefill_tensor_memory_kernel(Hq, Hkv, lens, new):
+    """The tcgen05 prefill attention (head_dim 128, the default there) on the cases of test_attn_prefill plus prompts
+    of several key tiles: ragged query tiles, chunked prefill, pages past a sequence's end inside a tile."""
+    test_attn_prefill(Hq, Hkv, 128, lens, new)
+
+
+@pytest.mark.parametrize("lens,new", [([37, 5, 64], [37, 2, 20]), ([300, 129, 1, 64], [300, 65, 1, 64]),
+                                      ([700, 128, 257], [700, 128, 130])])
+def test_attn_prefill_mma_sync_kernel_head_dim_128(lens, new):
+    """head_dim 128 on the mma.sync kernel (otherwise only reached by the other head sizes)."""
+    hyp.hyp_tune(hyp.HYP_TUNE_PREFILL_ATTN_TC, 0)
+    try:
+        test_attn_prefill(40, 10, 128, lens, new)
+    finally:
+        hyp.hyp_tune(hyp.HYP_TUNE_PREFILL_ATTN_TC, 1)
+
+
 @pytest.mark.parametrize("Hq,Hkv,D", [(4, 2, 64), (40, 10, 128), (8, 8, 64)])
 @pytest.mark.parametrize("lens,new", [([37, 5, 64], [37, 2, 20]), ([300, 129, 1, 64], [300, 65, 1, 64])])
 def test_attn_prefill(Hq, Hkv, D, lens, new):
