@@ -57,6 +57,7 @@ struct hyp_stage {
   __half* q16 = nullptr;              // rotated queries
   __half *h = nullptr, *attn = nullptr, *u = nullptr;  // projection inputs (fp16)
   TcAct tc_h, tc_attn, tc_u, tc_q16;
+  int* err_host = nullptr;  // pinned: the device error word, copied behind a host-buffer call's last kernel
   std::vector<CUtensorMap> kv_maps;  // per block: the page pool as rows (tcgen05 prefill attention, head_dim 128)
   int max_splits = 8;
   float2* rope_table = nullptr;
@@ -456,11 +457,12 @@ int run_stage_host(hyp_stage* s, const hyp_batch* b, const void* in, void* out, 
   }
   int rc = run_stage(s, b, in, out, st, decode, /*io_on_host=*/true);
   if (rc) return rc;
+  // the error word rides behind the last kernel, so one synchronisation covers the outputs and the status
+  *s->err_host = 0;
+  if (tc_err_flag_ptr())
+    HYP_CUDA_TRY(cudaMemcpyAsync(s->err_host, tc_err_flag_ptr(), sizeof(int), cudaMemcpyDeviceToHost, st));
   HYP_CUDA_TRY(cudaStreamSynchronize(st));
-  int dev_err = 0;
-  rc = tc_error_flag(&dev_err);
-  if (rc) return rc;
-  return dev_err ? HYP_ETIMEOUT : HYP_OK;
+  return *s->err_host ? HYP_ETIMEOUT : HYP_OK;
 }
 
 __global__ void fill_pattern_kernel(float* x, size_t n) {
@@ -505,6 +507,7 @@ extern "C" void hyp_stage_destroy(hyp_stage* s) {
     if (s->meta_host[i]) cudaFreeHost(s->meta_host[i]);
     if (s->meta_ev[i]) cudaEventDestroy(s->meta_ev[i]);
   }
+  if (s->err_host) cudaFreeHost(s->err_host);
   for (cudaEvent_t e : s->time_ev) cudaEventDestroy(e);
   for (auto& g : s->graphs)
     if (g.exec) cudaGraphExecDestroy(g.exec);
@@ -599,6 +602,7 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
     TRY_CUDA(cudaMallocHost((void**)&s->meta_host[i], s->meta_ints * sizeof(int32_t)));
     TRY_CUDA(cudaEventCreateWithFlags(&s->meta_ev[i], cudaEventDisableTiming));
   }
+  TRY_CUDA(cudaMallocHost((void**)&s->err_host, sizeof(int)));
   // staging for host-buffer calls
   s->io_in_bytes = (size_t)s->max_rows * (s->first ? sizeof(int32_t) : d.H * sizeof(float));
   s->io_out_bytes = s->last ? (size_t)std::max(c.max_seqs, std::min(s->max_rows, 64)) * d.V * sizeof(float)

@@ -111,19 +111,32 @@ def test_two_stages_chained_equal_oracle_and_hidden_boundary():
 
 
 def test_host_buffer_entry_points_match_device_ones():
+    """Same kernels behind both kinds of entry point.  Calls of up to 8 rows take the weight-streaming projections,
+    which are bit-reproducible, so there the two paths must agree exactly; a larger prefill adds its split-K
+    partial sums with floating-point atomics, whose order (and with it the last bits, amplified by the fp16
+    roundings that follow) may change from run to run, on either path."""
     sh = inputs.tiny_shape()
-    ids = inputs.token_ids(inputs.SEED_PROMPTS, 40, 20, sh.vocab)
-    st = H.gpu_stage(sh, 0, 2, 2, 32, 32)
+    ids = inputs.token_ids(inputs.SEED_PROMPTS, 40, 29, sh.vocab)
+    st = H.gpu_stage(sh, 0, 2, 2, 48, 32)
     out_d = torch.empty(1, sh.vocab, dtype=torch.float32, device="cuda")
-    st.prefill([0], [19], [0], dev(ids[:19]), out_d)
     out_h = torch.empty(1, sh.vocab, dtype=torch.float32).pin_memory()
-    hyp.hyp_stage_prefill_host(st.handle, [1], [19], [0], ids[:19].pin_memory(), out_h)
+    st.prefill([0], [8], [0], dev(ids[:8]), out_d)
+    hyp.hyp_stage_prefill_host(st.handle, [1], [8], [0], ids[:8].pin_memory(), out_h)
     torch.cuda.synchronize()
     assert torch.equal(out_d.cpu(), out_h)
-    st.decode([0], [19], dev(ids[19:20]), out_d)
-    hyp.hyp_stage_decode_host(st.handle, [1], [19], ids[19:20].pin_memory(), out_h)
+    st.decode([0], [8], dev(ids[8:9]), out_d)
+    hyp.hyp_stage_decode_host(st.handle, [1], [8], ids[8:9].pin_memory(), out_h)
     torch.cuda.synchronize()
     assert torch.equal(out_d.cpu(), out_h)
+    # a 19-row chunk behind the 9 cached tokens, then one more decode step
+    st.prefill([0], [19], [9], dev(ids[9:28]), out_d)
+    hyp.hyp_stage_prefill_host(st.handle, [1], [19], [9], ids[9:28].pin_memory(), out_h)
+    torch.cuda.synchronize()
+    assert torch.allclose(out_d.cpu(), out_h, rtol=0, atol=5e-3)
+    st.decode([0], [28], dev(ids[28:29]), out_d)
+    hyp.hyp_stage_decode_host(st.handle, [1], [28], ids[28:29].pin_memory(), out_h)
+    torch.cuda.synchronize()
+    assert torch.allclose(out_d.cpu(), out_h, rtol=0, atol=5e-3)
     st.close()
 
 
