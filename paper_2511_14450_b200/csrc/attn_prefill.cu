@@ -240,7 +240,7 @@ int launch_fa(const __half* qkv, const __half* kv_layer, __half* attn_out, const
   }
   // every sequence adds at most one ragged tile on top of floor(rows / 64)
   const int max_tiles = bm.n_tokens / FA_BQ + bm.n_seqs;
-  HYP_CUDA_TRY(launch_pdl(attn_prefill_fa_kernel<D>, dim3(d.Hq, max_tiles), dim3(FA_THREADS), smem, st, qkv, kv_layer,
+  HYP_CUDA_TRY(launch_pdl<2>(attn_prefill_fa_kernel<D>, dim3(d.Hq, max_tiles), dim3(FA_THREADS), smem, st, qkv, kv_layer,
                           attn_out, bm, d, tc_err_flag_ptr()));
   return 1;
 }

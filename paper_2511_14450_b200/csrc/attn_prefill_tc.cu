@@ -371,7 +371,7 @@ int launch_attn_prefill_tc(const CUtensorMap& q_map, const CUtensorMap& kv_map, 
     configured = true;
   }
   const int max_tiles = bm.n_tokens / PT_Q + bm.n_seqs;  // every sequence adds at most one ragged tile
-  HYP_CUDA_TRY(launch_pdl(attn_prefill_tc_kernel, dim3(d.Hq, max_tiles), dim3(PT_THREADS), (size_t)PT_SMEM, st, q_map, kv_map,
+  HYP_CUDA_TRY(launch_pdl<2>(attn_prefill_tc_kernel, dim3(d.Hq, max_tiles), dim3(PT_THREADS), (size_t)PT_SMEM, st, q_map, kv_map,
                           attn_out, bm, d, tc_err_flag_ptr()));
   return 1;
 }

@@ -177,7 +177,7 @@ int launch_rope_kv_write(const float* qkv, __half* q16, __half* kv_layer, const 
   const int work = (d.Hq + 2 * d.Hkv) * (d.D / 16);
   int threads = ((work + 31) / 32) * 32;
   if (threads > 512) threads = 512;
-  HYP_CUDA_TRY(launch_pdl(rope_kv_write_kernel, dim3(bm.n_tokens), dim3(threads), 0, st, qkv, q16, kv_layer, rope_table,
+  HYP_CUDA_TRY(launch_pdl<2>(rope_kv_write_kernel, dim3(bm.n_tokens), dim3(threads), 0, st, qkv, q16, kv_layer, rope_table,
                           bm, d));
   return 1;
 }
