@@ -203,7 +203,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t tmem_s = tmem_slot, tmem_o = tmem_slot + 128u;
 
   if (warp == 0) {
-    // ---------------- TMA producer: one box per lane and tile (a single thread issues a box every ~250 cycles) ----
+    // ---------------- TMA producer: one box per lane and tile, the sixteen boxes of a tile side by side ----------
     // lanes 0-7 bring the keys, 8-15 the values; within each, lane = page (0-3) x half of head_dim
     if (lane == 0) {
       mbar_expect_tx(q_full, 2 * PT_TILE);
