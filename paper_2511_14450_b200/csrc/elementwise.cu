@@ -48,9 +48,10 @@ int launch_copy_f32(const float* src, float* dst, size_t n, cudaStream_t st) {
 // row = row_index ? row_index[r] : r.  fp32 statistics; output bf16, or fp16 for the q/k/v projection
 // (whose inputs need fp16's 11 mantissa bits to keep the softmax weights inside the logit tolerance).
 template <int THREADS, bool F16>
-__global__ void rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ g, void* __restrict__ h,
+__global__ void __launch_bounds__(THREADS, 1280 / THREADS)  // <= 51 registers: five 256-thread CTAs per SM
+rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ g, void* __restrict__ h,
                                int H, float eps, const int32_t* __restrict__ row_index) {
-  constexpr int CACHE = 8;  // float4 per thread kept in registers: rows up to THREADS * 32 wide are read once
+  constexpr int CACHE = 5;  // float4 per thread kept in registers: rows up to THREADS * 20 wide are read once
   __shared__ float red[THREADS / 32];
   const int r = blockIdx.x;
   const int n4 = H / 4;
@@ -124,59 +125,78 @@ int launch_rmsnorm(const float* x, const __nv_bfloat16* g, void* h, bool out_f16
 // Input row layout (fp32, straight from the projection's accumulators): [Q heads | K heads | V heads],
 // each head D wide.  Outputs are fp16 (rounded once): q to its own [M, Hq*D] buffer, k and v to the pages.
 // One thread handles 8 rotation pairs (i .. i+7, i+D/2 .. i+D/2+7) of one head of one row.
-__global__ void rope_kv_write_kernel(const float* __restrict__ qkv, __half* __restrict__ q16,
-                                     __half* __restrict__ kv_layer, const float2* __restrict__ rope_table,
-                                     BatchMeta bm, ModelDims d) {
+__global__ void __launch_bounds__(256, 4)
+rope_kv_write_kernel(const float* __restrict__ qkv, __half* __restrict__ q16, __half* __restrict__ kv_layer,
+                     const float2* __restrict__ rope_table, BatchMeta bm, ModelDims d) {
   pdl_trigger();
   pdl_wait();
+  constexpr int ITEMS = 2;  // work items of a thread whose loads are issued together
   const int t = blockIdx.x;
   const int vec_per_head = d.D / 16;
   const int n_heads = d.Hq + 2 * d.Hkv;
-  const int pos = bm.tok_pos[t];
-  const int sq = bm.tok_seq[t];
-  const int page = bm.block_table[(size_t)sq * bm.max_pages_per_seq + pos / d.page_tokens];
-  const int slot = pos % d.page_tokens;
-  const size_t page_base = (size_t)page * kv_page_elems(d.Hkv, d.page_tokens, d.D);
+  const int n_work = n_heads * vec_per_head;
   const float* row = qkv + (size_t)t * d.qkv_rows;
-  for (int w = threadIdx.x; w < n_heads * vec_per_head; w += blockDim.x) {
-    const int head = w / vec_per_head;
-    const int i0 = (w % vec_per_head) * 8;
-    const float* hp = row + (size_t)head * d.D;
-    float a[8], b[8];
-    *reinterpret_cast<float4*>(a) = *reinterpret_cast<const float4*>(hp + i0);
-    *reinterpret_cast<float4*>(a + 4) = *reinterpret_cast<const float4*>(hp + i0 + 4);
-    *reinterpret_cast<float4*>(b) = *reinterpret_cast<const float4*>(hp + d.D / 2 + i0);
-    *reinterpret_cast<float4*>(b + 4) = *reinterpret_cast<const float4*>(hp + d.D / 2 + i0 + 4);
-    __half* dst;
-    if (head < d.Hq + d.Hkv) {
-      const float2* cs = rope_table + (size_t)pos * (d.D / 2) + i0;
+  for (int w0 = threadIdx.x; w0 < n_work; w0 += ITEMS * blockDim.x) {
+    // the projection's rows first: they depend on nothing, the token's position and page are a chain of two loads
+    float4 a[ITEMS][2], b[ITEMS][2];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float2 c = cs[j];
-        const float x1 = a[j], x2 = b[j];
-        a[j] = x1 * c.x - x2 * c.y;
-        b[j] = x2 * c.x + x1 * c.y;
+    for (int it = 0; it < ITEMS; ++it) {
+      const int w = w0 + it * blockDim.x;
+      if (w < n_work) {
+        const float* hp = row + (size_t)(w / vec_per_head) * d.D + (w % vec_per_head) * 8;
+        a[it][0] = *reinterpret_cast<const float4*>(hp);
+        a[it][1] = *reinterpret_cast<const float4*>(hp + 4);
+        b[it][0] = *reinterpret_cast<const float4*>(hp + d.D / 2);
+        b[it][1] = *reinterpret_cast<const float4*>(hp + d.D / 2 + 4);
       }
-      dst = head < d.Hq ? q16 + (size_t)t * d.Hq * d.D + (size_t)head * d.D
-                        : kv_layer + page_base + ((size_t)(head - d.Hq) * d.page_tokens + slot) * d.D;
-    } else {
-      dst = kv_layer + page_base + (size_t)d.Hkv * d.page_tokens * d.D +
-            ((size_t)(head - d.Hq - d.Hkv) * d.page_tokens + slot) * d.D;
     }
-    // cache rows keep their 16-byte chunks XOR-permuted by the token's slot (see kv_chunk_pos); q rows are plain
-    const int sw = head < d.Hq ? 0 : (slot & 7);
-    *reinterpret_cast<uint4*>(dst + (((i0 >> 3) ^ sw) << 3)) =
-        make_uint4(pack_f16_sat(a[0], a[1]), pack_f16_sat(a[2], a[3]), pack_f16_sat(a[4], a[5]), pack_f16_sat(a[6], a[7]));
-    *reinterpret_cast<uint4*>(dst + ((((d.D / 2 + i0) >> 3) ^ sw) << 3)) =
-        make_uint4(pack_f16_sat(b[0], b[1]), pack_f16_sat(b[2], b[3]), pack_f16_sat(b[4], b[5]), pack_f16_sat(b[6], b[7]));
+    const int pos = bm.tok_pos[t];
+    const int sq = bm.tok_seq[t];
+    const int page = bm.block_table[(size_t)sq * bm.max_pages_per_seq + pos / d.page_tokens];
+    const int slot = pos % d.page_tokens;
+    const size_t page_base = (size_t)page * kv_page_elems(d.Hkv, d.page_tokens, d.D);
+#pragma unroll
+    for (int it = 0; it < ITEMS; ++it) {
+      const int w = w0 + it * blockDim.x;
+      if (w >= n_work) break;
+      const int head = w / vec_per_head;
+      const int i0 = (w % vec_per_head) * 8;
+      float x1[8] = {a[it][0].x, a[it][0].y, a[it][0].z, a[it][0].w, a[it][1].x, a[it][1].y, a[it][1].z, a[it][1].w};
+      float x2[8] = {b[it][0].x, b[it][0].y, b[it][0].z, b[it][0].w, b[it][1].x, b[it][1].y, b[it][1].z, b[it][1].w};
+      __half* dst;
+      if (head < d.Hq + d.Hkv) {
+        const float4* cs = reinterpret_cast<const float4*>(rope_table + (size_t)pos * (d.D / 2) + i0);  // (cos, sin) pairs
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float4 c = cs[j];
+          const float u0 = x1[2 * j], v0 = x2[2 * j], u1 = x1[2 * j + 1], v1 = x2[2 * j + 1];
+          x1[2 * j] = u0 * c.x - v0 * c.y;
+          x2[2 * j] = v0 * c.x + u0 * c.y;
+          x1[2 * j + 1] = u1 * c.z - v1 * c.w;
+          x2[2 * j + 1] = v1 * c.z + u1 * c.w;
+        }
+        dst = head < d.Hq ? q16 + (size_t)t * d.Hq * d.D + (size_t)head * d.D
+                          : kv_layer + page_base + ((size_t)(head - d.Hq) * d.page_tokens + slot) * d.D;
+      } else {
+        dst = kv_layer + page_base + (size_t)d.Hkv * d.page_tokens * d.D +
+              ((size_t)(head - d.Hq - d.Hkv) * d.page_tokens + slot) * d.D;
+      }
+      // cache rows keep their 16-byte chunks XOR-permuted by the token's slot (see kv_chunk_pos); q rows are plain
+      const int sw = head < d.Hq ? 0 : (slot & 7);
+      *reinterpret_cast<uint4*>(dst + (((i0 >> 3) ^ sw) << 3)) = make_uint4(
+          pack_f16_sat(x1[0], x1[1]), pack_f16_sat(x1[2], x1[3]), pack_f16_sat(x1[4], x1[5]), pack_f16_sat(x1[6], x1[7]));
+      *reinterpret_cast<uint4*>(dst + ((((d.D / 2 + i0) >> 3) ^ sw) << 3)) = make_uint4(
+          pack_f16_sat(x2[0], x2[1]), pack_f16_sat(x2[2], x2[3]), pack_f16_sat(x2[4], x2[5]), pack_f16_sat(x2[6], x2[7]));
+    }
   }
 }
 
 int launch_rope_kv_write(const float* qkv, __half* q16, __half* kv_layer, const float2* rope_table,
                          const BatchMeta& bm, const ModelDims& d, cudaStream_t st) {
   const int work = (d.Hq + 2 * d.Hkv) * (d.D / 16);
-  int threads = ((work + 31) / 32) * 32;
-  if (threads > 512) threads = 512;
+  int threads = ((work / 2 + 31) / 32) * 32;  // two work items per thread
+  if (threads > 256) threads = 256;
+  if (threads < 32) threads = 32;
   HYP_CUDA_TRY(launch_pdl<2>(rope_kv_write_kernel, dim3(bm.n_tokens), dim3(threads), 0, st, qkv, q16, kv_layer, rope_table,
                           bm, d));
   return 1;
