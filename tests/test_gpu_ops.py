@@ -219,7 +219,7 @@ def test_attn_decode_rejects_small_scratch():
 
 @pytest.mark.parametrize("Hq,Hkv", [(40, 10), (8, 8), (8, 1)])
 @pytest.mark.parametrize("lens,new", [([37, 5, 64], [37, 2, 20]), ([300, 129, 1, 64], [300, 65, 1, 64]),
-                                      ([700, 128, 257], [700, 128, 130])])
+                                      ([700, 128, 257], [700, 128, 130]), ([1500, 90, 64], [300, 90, 1])])
 def test_attn_prefill_tensor_memory_kernel(Hq, Hkv, lens, new):
     """The tcgen05 prefill attention (head_dim 128, the default there) on the cases of test_attn_prefill plus prompts
     of several key tiles: ragged query tiles, chunked prefill, pages past a sequence's end inside a tile."""
