@@ -77,7 +77,7 @@ typedef struct {
   int32_t n_kv_heads;     /* Hkv; query head h reads KV head floor(h / (Hq/Hkv))                   */
   int32_t head_dim;       /* D: 64 or 128                                                          */
   int32_t ffn;            /* F: SwiGLU inner width, multiple of 8                                  */
-  int32_t vocab;          /* V                                                                     */
+  int32_t vocab;          /* V, multiple of 8 (rows of the logits matrix start on 16-byte boundaries) */
   float rms_eps;          /* y = x / sqrt(mean(x^2) + eps) * g                                     */
   float rope_theta;       /* pair (i, i + D/2) rotated by pos * theta^(-2i/D), positions from 0    */
   int32_t kv_block_size;  /* tokens per KV page; must be 16                                        */
@@ -139,8 +139,11 @@ HYP_API int hyp_stage_load(hyp_stage* s, int32_t layer, int32_t tensor_id, const
  *        activations [M, H] from the previous stage.
  *   out: DEVICE. fp32 activations [M, H]; or, if layer_hi == n_layers_total, fp32 logits
  *        [n_seqs, V] of each sequence's last row ([M, V] with HYP_BATCH_ALL_LOGITS).
- * Errors: HYP_EINVAL, HYP_ECAPACITY (M > max_tokens, context > max_ctx, pool empty; the cache is
- * left unchanged), HYP_ESTATE, HYP_ECUDA. */
+ *        Both 16-byte aligned (ids: 4-byte).
+ * Errors: HYP_EINVAL, HYP_ECAPACITY (M > max_tokens, context > max_ctx, pool empty), HYP_ESTATE,
+ * HYP_ECUDA.  Whatever the code, a call that does not return HYP_OK leaves the slot lengths
+ * (hyp_stage_seq_len) and the page pool as they were before it: arguments are checked before anything
+ * is reserved, and pages reserved for a call whose enqueue then fails (HYP_ECUDA) are handed back. */
 HYP_API int hyp_stage_prefill(hyp_stage* s, const hyp_batch* batch, const void* in, void* out, void* stream);
 
 /* Decode: one new row per sequence (q_lens all 1, n_seqs <= HYP_MAX_DECODE_BATCH), attending to
@@ -199,28 +202,29 @@ HYP_API void hyp_stage_destroy(hyp_stage* s);
  *   f, m : HOST double [N]   block compute cost (any unit, >= 0) and memory (>= 0)
  *   C    : HOST double [T]   tier capacity (> 0), same unit as f per unit time
  *   Mcap : HOST double [T]   tier memory limit (>= 0), same unit as m
- *   eps  : 0  -> exact: the feasibility DP of Algorithm 1 is driven over the finite set of
- *                values a tier load can take, so the minimum is found exactly;
- *          >0 -> Algorithm 1 as printed: bisection on tau from [0, S_f[N]/min C] until the
- *                interval is <= eps (result within eps of the optimum).
+ *   eps  : 0  -> exact: the monotone feasibility test of Algorithm 1 is bisected over the finite,
+ *                sorted set of values a tier load can take, so the minimum is found exactly;
+ *          >0 -> the same search may stop once the bracket around the optimum is narrower than
+ *                eps (the paper's tolerance parameter): the result is a memory-feasible partition
+ *                whose bottleneck is within eps of the optimum.
  *   p_out  : HOST int32 [T-1], 1-based index of the last block of tiers 1..T-1 (may be NULL if T==1)
  *   tau_out: HOST double, max_j L_j(p_out)
- * Ties between equally good partitions are resolved as Algorithm 1 does (first feasible
- * predecessor scanning upward, backtracking from the last tier): the result is the smallest
- * vector when read as (p_{T-1}, ..., p_1).
+ * Ties between equally good partitions are resolved as Algorithm 1's predecessor choice implies
+ * (each tier, from the last one back, takes the smallest feasible predecessor): the result is the
+ * smallest vector when read as (p_{T-1}, ..., p_1).
  * Errors: HYP_EINVAL (null, N < 1, T < 1, negative cost, C <= 0, NaN), HYP_EINFEASIBLE. */
 HYP_API int hyp_split_dp(int32_t N, int32_t T, const double* f, const double* m, const double* C,
                  const double* Mcap, double eps, int32_t* p_out, double* tau_out);
 
-/* The partitioning steps of the two systems the paper compares against (Section V, "HEFT" and "GPipe"), on the
+/* The partitioning steps of the two systems the paper compares against (Section V, the HEFT and GPipe baselines), on the
  * same inputs as hyp_split_dp, so that their bottleneck max_j L_j(p) can be set beside HypSplit-DP's on measured
  * per-block costs.  The paper names the strategies and gives no algorithm; the readings taken here:
- *   hyp_split_even   ("classic static, load balanced partitioning" of GPipe into contiguous segments):
+ *   hyp_split_even   (GPipe's static split of the block chain into contiguous, equally long segments):
  *                    segments of equal block count, the N mod T leading tiers one block longer; costs,
  *                    capacities and memory limits play no part.  p_out and tau_out are always written for valid
  *                    arguments with N >= T; the return value is HYP_EINFEASIBLE if a segment exceeds its tier's
  *                    memory limit (the partition is reported, not repaired).
- *   hyp_split_greedy ("memory aware greedy strategy" that precedes HEFT's scheduling): tiers are filled in order;
+ *   hyp_split_greedy (the greedy, memory-checking partitioning step that precedes HEFT's scheduling): tiers are filled in order;
  *                    tier j keeps taking the next block while its memory limit holds and its load stays within
  *                    its capacity-proportional share S_f[N] * C_j / sum(C), takes at least one block, and leaves
  *                    one block for every later tier; the last tier takes the rest.  HYP_EINFEASIBLE (outputs

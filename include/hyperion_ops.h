@@ -110,7 +110,7 @@ HYP_API int hyp_op_attn_decode(const hyp_attn_shape* shape, int32_t n_seqs, cons
                                void* out, void* stream);
 
 /* One decode step of the attention sub-layer as hyp_stage_decode runs it, in a single launch: rotary encoding
- * (Section III-A: grouped-query attention "with rotary position encoding") of the new token's query and key,
+ * (Section III-A: the block's grouped-query attention carries a rotary position encoding) of the new token's query and key,
  * append of its key and value to the paged cache, attention of the new token over positions
  * 0 .. ctx_lens[b] (itself included) and the merge of the context splits (a thread-block cluster per sequence
  * and KV head, merged through distributed shared memory; no scratch buffer).

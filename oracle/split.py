@@ -20,8 +20,8 @@ Readings where the paper is silent (each is restated in the library's header):
   - the returned tau* is max_j L_j(p*) of the returned partition, not the last probe value.
 
 * `split_even`, `split_greedy` - the inter-tier partitioning halves of the paper's two comparison
-  systems (Section V, baselines), which it only names: the "classic static, load balanced
-  partitioning" of GPipe into contiguous segments, and the "memory aware greedy strategy" that
+  systems (Section V, baselines), which it only names: GPipe's static split of the chain into
+  contiguous, equally long segments, and the greedy, memory-checking partitioning step that
   precedes HEFT.  Readings taken (the paper gives no algorithm for either):
   - even: contiguous segments of equal block count, the N mod T leading tiers one block longer;
     blind to costs, capacities and memory (a violated memory limit is reported, not repaired);
@@ -116,7 +116,7 @@ def backtrack(P, N, T):
 
 
 def hypsplit_dp_bisect(f, m, C, Mcap, eps):
-    """Algorithm 1 (HypSplit-DP) as printed: bisection until tau_high - tau_low <= eps.
+    """Algorithm 1 (HypSplit-DP) step by step: bisection until tau_high - tau_low <= eps.
 
     Returns (p*, tau*, probes) where tau* = max_j L_j(p*) and probes is the number of DP
     checks made; (None, inf, probes) if even tau_high is infeasible."""

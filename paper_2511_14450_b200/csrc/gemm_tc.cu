@@ -757,6 +757,9 @@ int launch_gemm_tc(const TcAct& act, const TcWeight& w, int M, int N, int K, int
   if (M < 1 || N < 1 || K < 8 || act.K != K || w.K != K || M > act.rows || !g_err_flag) return HYP_EINVAL;
   if (w.rows != N || w.halves != (epi == EPI_SWIGLU_BF16 ? 2 : 1)) return HYP_EINVAL;
   if (act.f16 != w.f16) return HYP_EINVAL;  // one instruction takes both operands in the same 16-bit type
+  // the epilogues write 16 bytes per lane at out + row * ldo + col (col a multiple of 16)
+  const int row_align = (epi == EPI_RESID_F32 || epi == EPI_STORE_F32) ? 4 : 8;
+  if (!out || ((uintptr_t)out & 15) != 0 || ldo < N || ldo % row_align) return HYP_EINVAL;
   switch (epi) {
     case EPI_STORE_BF16: return launch_epi<EPI_STORE_BF16>(act, w, M, N, K, out, ldo, st, early);
     case EPI_RESID_F32: return launch_epi<EPI_RESID_F32>(act, w, M, N, K, out, ldo, st, early);

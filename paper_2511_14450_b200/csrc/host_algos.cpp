@@ -9,47 +9,62 @@
 
 namespace {
 
-// Decision problem P_check(tau) of Section IV-A: boolean DP over (tier j, blocks 1..n) with the
-// predecessor taken as the first feasible k while scanning upward.  Tables are (T+1) x (N+1).
-struct CheckTables {
-  int N, T;
-  std::vector<uint8_t> dp;
-  std::vector<int32_t> pred;
-  CheckTables(int n, int t) : N(n), T(t), dp((size_t)(t + 1) * (n + 1)), pred((size_t)(t + 1) * (n + 1)) {}
-  uint8_t& D(int j, int n) { return dp[(size_t)j * (N + 1) + n]; }
-  int32_t& P(int j, int n) { return pred[(size_t)j * (N + 1) + n]; }
-};
+// Feasibility of a latency budget tau for problem P1 (Section III-D), and the canonical partition that meets it.
+//
+// A tier's load (S_f[n] - S_f[k]) / C_j and memory S_m[n] - S_m[k] only shrink as the segment's left edge k moves
+// right (prefix sums of non-negative numbers are monotone, also in floating point), and only grow with its right
+// edge n.  So for tier j and right edge n the admissible left edges form a run [left_j(n), n-1] whose start never
+// moves left as n grows: one two-pointer sweep per tier finds every left_j(n).  Tier j can end at n iff some
+// prefix length in that run is reachable by tiers 1..j-1; `next_reachable` answers "smallest reachable prefix at
+// or after k" in O(1), which is also the predecessor the tie rule of hyperion.h asks for (the smallest one).
+// One probe costs O(T N).
+class BudgetSweep {
+ public:
+  BudgetSweep(int N, int T, const std::vector<double>& Sf, const std::vector<double>& Sm, const double* C,
+              const double* Mcap)
+      : N_(N), T_(T), Sf_(Sf), Sm_(Sm), C_(C), Mcap_(Mcap), first_pred_((size_t)T * (N + 1)),
+        next_reachable_(N + 2), reach_(N + 1) {}
 
-bool p_check(double tau, CheckTables& tb, const std::vector<double>& Sf, const std::vector<double>& Sm,
-             const double* C, const double* Mcap) {
-  const int N = tb.N, T = tb.T;
-  std::fill(tb.dp.begin(), tb.dp.end(), 0);
-  std::fill(tb.pred.begin(), tb.pred.end(), -1);
-  tb.D(0, 0) = 1;
-  for (int j = 1; j <= T; ++j) {
-    for (int n = j; n <= N; ++n) {
-      for (int k = j - 1; k < n; ++k) {
-        if (!tb.D(j - 1, k)) continue;
-        const double L = (Sf[n] - Sf[k]) / C[j - 1];
-        const double U = Sm[n] - Sm[k];
-        if (L <= tau && U <= Mcap[j - 1]) {
-          tb.D(j, n) = 1;
-          tb.P(j, n) = k;
-          break;
-        }
+  bool feasible(double tau) {
+    std::fill(reach_.begin(), reach_.end(), 0);
+    reach_[0] = 1;  // zero tiers cover the empty prefix
+    for (int j = 0; j < T_; ++j) {
+      // smallest reachable prefix length >= k (N_ + 1: none)
+      next_reachable_[N_ + 1] = N_ + 1;
+      for (int k = N_; k >= 0; --k) next_reachable_[k] = reach_[k] ? k : next_reachable_[k + 1];
+      std::fill(reach_.begin(), reach_.end(), 0);
+      int32_t* pred = &first_pred_[(size_t)j * (N_ + 1)];
+      int left = 0;
+      for (int n = 1; n <= N_; ++n) {
+        while (left < n && !fits(j, left, n, tau)) ++left;
+        const int k = left < n ? next_reachable_[left] : n;
+        pred[n] = k < n ? k : -1;
+        reach_[n] = k < n;
       }
     }
+    return reach_[N_] != 0;
   }
-  return tb.D(T, N) != 0;
-}
 
-void backtrack(CheckTables& tb, int32_t* p) {
-  int n = tb.N;
-  for (int j = tb.T; j >= 2; --j) {
-    n = tb.P(j, n);
-    p[j - 2] = n;
+  // cut points of the partition the last feasible() call found: walk the predecessors back from (T, N)
+  void cuts(int32_t* p) const {
+    int n = N_;
+    for (int j = T_ - 1; j >= 1; --j) {
+      n = first_pred_[(size_t)j * (N_ + 1) + n];
+      p[j - 1] = n;
+    }
   }
-}
+
+ private:
+  bool fits(int j, int k, int n, double tau) const {
+    return (Sf_[n] - Sf_[k]) / C_[j] <= tau && Sm_[n] - Sm_[k] <= Mcap_[j];
+  }
+  int N_, T_;
+  const std::vector<double>&Sf_, &Sm_;
+  const double *C_, *Mcap_;
+  std::vector<int32_t> first_pred_;
+  std::vector<int> next_reachable_;
+  std::vector<uint8_t> reach_;
+};
 
 double bottleneck(const int32_t* p, int N, int T, const std::vector<double>& Sf, const double* C) {
   double tau = 0.0;
@@ -81,44 +96,34 @@ extern "C" int hyp_split_dp(int32_t N, int32_t T, const double* f, const double*
     Sf[i + 1] = Sf[i] + f[i];
     Sm[i + 1] = Sm[i] + m[i];
   }
-  CheckTables tb(N, T);
-  std::vector<int32_t> p(std::max(T - 1, 1), 0);
+  // The optimum is one of the finitely many values a tier load can take, and feasibility is monotone in the
+  // budget (Section IV-A), so the search runs over the sorted set of those values: exact, no tolerance needed.
+  // With eps > 0 the search may stop as soon as the bracket [largest infeasible, smallest feasible seen] is
+  // narrower than eps; the partition of the feasible end is then within eps of the optimum.
+  std::vector<double> cand;
+  cand.reserve((size_t)T * N * (N + 1) / 2);
+  for (int j = 0; j < T; ++j)
+    for (int n = 1; n <= N; ++n)
+      for (int k = 0; k < n; ++k) cand.push_back((Sf[n] - Sf[k]) / C[j]);
+  std::sort(cand.begin(), cand.end());
+  cand.erase(std::unique(cand.begin(), cand.end()), cand.end());
 
-  if (eps > 0.0) {
-    // Algorithm 1 as printed: bisection on tau.
-    double c_min = C[0];
-    for (int j = 1; j < T; ++j) c_min = std::min(c_min, C[j]);
-    double lo = 0.0, hi = Sf[N] / c_min;
-    if (!p_check(hi, tb, Sf, Sm, C, Mcap)) return HYP_EINFEASIBLE;
-    backtrack(tb, p.data());
-    while ((hi - lo) > eps) {
-      const double mid = (lo + hi) / 2.0;
-      if (p_check(mid, tb, Sf, Sm, C, Mcap)) {
-        hi = mid;
-        backtrack(tb, p.data());
-      } else {
-        lo = mid;
-      }
+  BudgetSweep sweep(N, T, Sf, Sm, C, Mcap);
+  if (!sweep.feasible(cand.back())) return HYP_EINFEASIBLE;   // only memory can rule out the largest budget
+  size_t lo = 0, hi = cand.size() - 1;  // cand[hi] is feasible; everything below cand[lo] is infeasible
+  double below = 0.0;                    // a budget known to be <= the optimum
+  while (lo < hi && !(eps > 0.0 && cand[hi] - below <= eps)) {
+    const size_t mid = lo + (hi - lo) / 2;
+    if (sweep.feasible(cand[mid])) {
+      hi = mid;
+    } else {
+      lo = mid + 1;
+      below = cand[mid];
     }
-  } else {
-    // Exact: the optimum is one of the finitely many values a tier load can take, and
-    // feasibility is monotone in tau, so bisect over the sorted candidate set.
-    std::vector<double> cand;
-    cand.reserve((size_t)T * N * (N + 1) / 2);
-    for (int j = 0; j < T; ++j)
-      for (int n = 1; n <= N; ++n)
-        for (int k = 0; k < n; ++k) cand.push_back((Sf[n] - Sf[k]) / C[j]);
-    std::sort(cand.begin(), cand.end());
-    cand.erase(std::unique(cand.begin(), cand.end()), cand.end());
-    if (!p_check(cand.back(), tb, Sf, Sm, C, Mcap)) return HYP_EINFEASIBLE;
-    size_t lo = 0, hi = cand.size() - 1;  // invariant: cand[hi] feasible
-    while (lo < hi) {
-      const size_t mid = lo + (hi - lo) / 2;
-      if (p_check(cand[mid], tb, Sf, Sm, C, Mcap)) hi = mid; else lo = mid + 1;
-    }
-    p_check(cand[hi], tb, Sf, Sm, C, Mcap);
-    backtrack(tb, p.data());
   }
+  std::vector<int32_t> p(std::max(T - 1, 1), 0);
+  sweep.feasible(cand[hi]);
+  sweep.cuts(p.data());
   for (int j = 0; j + 1 < T; ++j) p_out[j] = p[j];
   *tau_out = bottleneck(p.data(), N, T, Sf, C);
   return HYP_OK;
@@ -126,23 +131,19 @@ extern "C" int hyp_split_dp(int32_t N, int32_t T, const double* f, const double*
 
 extern "C" int hyp_sched_rt(double F_new, double m_act, const hyp_node_state* nodes, int32_t K,
                             int32_t* k_out) {
-  if (!nodes || !k_out || K < 1 || !(F_new >= 0.0) || std::isnan(m_act)) return HYP_EINVAL;
+  if (!nodes || !k_out || K < 1 || !(F_new >= 0.0) || !std::isfinite(F_new) || std::isnan(m_act)) return HYP_EINVAL;
   for (int k = 0; k < K; ++k)
-    if (!(nodes[k].C > 0.0) || std::isnan(nodes[k].F_rem) || std::isnan(nodes[k].F_wait)) return HYP_EINVAL;
-  double min_cost = INFINITY;
-  int32_t k_star = -1;
-  for (int k = 0; k < K; ++k) {
-    if (nodes[k].available && nodes[k].M_avail >= m_act) {
-      const double queued = nodes[k].F_rem + nodes[k].F_wait;
-      const double cost = (queued + F_new) / nodes[k].C;
-      if (cost < min_cost) {
-        min_cost = cost;
-        k_star = k;
-      }
-    }
-  }
-  if (k_star < 0) return HYP_EINFEASIBLE;
-  *k_out = k_star;
+    if (!(nodes[k].C > 0.0) || !std::isfinite(nodes[k].F_rem) || !std::isfinite(nodes[k].F_wait)) return HYP_EINVAL;
+  // the nodes that may take the task (Section IV-B: switched on, enough free memory) ...
+  std::vector<int32_t> eligible;
+  for (int k = 0; k < K; ++k)
+    if (nodes[k].available && nodes[k].M_avail >= m_act) eligible.push_back(k);
+  if (eligible.empty()) return HYP_EINFEASIBLE;
+  // ... and among them the earliest estimated completion of the new task; min_element keeps the first of equal
+  // minima, i.e. the lowest node index
+  auto finish = [&](int32_t k) { return (nodes[k].F_rem + nodes[k].F_wait + F_new) / nodes[k].C; };
+  *k_out = *std::min_element(eligible.begin(), eligible.end(),
+                             [&](int32_t a, int32_t b) { return finish(a) < finish(b); });
   return HYP_OK;
 }
 

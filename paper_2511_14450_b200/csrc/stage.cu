@@ -148,6 +148,9 @@ struct HostBatch {
   int n = 0, M = 0;
   std::vector<int32_t> packed;  // q_lens | ctx_lens | cu_q | last_row | tok_seq | tok_pos | block_table
   size_t off_q, off_ctx, off_cu, off_last, off_tseq, off_tpos, off_bt;
+  // what admission changed, so that a call that fails after it can put the tables back
+  struct Undo { int32_t id, old_len; size_t old_pages; };
+  std::vector<Undo> undo;
 };
 
 void layout_meta(HostBatch& hb, int n, int M, int mpps) {
@@ -223,6 +226,7 @@ int admit_batch(hyp_stage* s, const hyp_batch* b, bool decode, HostBatch& hb) {
     const int id = b->seq_ids[i];
     const int total = b->ctx_lens[i] + b->q_lens[i];
     auto& pages = s->seq_pages[id];
+    hb.undo.push_back({id, s->seq_len[id], pages.size()});
     while ((int)pages.size() < (total + PT - 1) / PT) {
       pages.push_back(s->free_pages.back());
       s->free_pages.pop_back();
@@ -241,6 +245,18 @@ int admit_batch(hyp_stage* s, const hyp_batch* b, bool decode, HostBatch& hb) {
   }
   p[hb.off_cu + n] = row;
   return HYP_OK;
+}
+
+// Undo admit_batch: lengths back, the pages taken for this call back on the free list in their old order.
+void rollback_batch(hyp_stage* s, const HostBatch& hb) {
+  for (auto it = hb.undo.rbegin(); it != hb.undo.rend(); ++it) {
+    auto& pages = s->seq_pages[it->id];
+    while (pages.size() > it->old_pages) {
+      s->free_pages.push_back(pages.back());
+      pages.pop_back();
+    }
+    s->seq_len[it->id] = it->old_len;
+  }
 }
 
 int check_ready(const hyp_stage* s) {
@@ -390,13 +406,19 @@ int decode_with_graph(hyp_stage* s, const BatchMeta& bm, int n, int n_splits, co
 int run_stage(hyp_stage* s, const hyp_batch* b, const void* in, void* out, cudaStream_t st, bool decode,
               bool io_on_host = false) {
   if (!s || !in || !out) return HYP_EINVAL;
+  // device buffers are written 16 bytes at a time by the epilogues (host buffers only see copies)
+  if (!io_on_host && ((((uintptr_t)in) & 3) != 0 || (((uintptr_t)out) & 15) != 0)) return HYP_EINVAL;
   int rc = check_ready(s);
   if (rc) return rc;
   HostBatch hb;
   rc = admit_batch(s, b, decode, hb);
   if (rc) return rc;
+  // from here on the tables say the rows are cached: any failure before the last enqueue puts them back
   rc = upload_meta(s, hb, st);
-  if (rc) return rc;
+  if (rc) {
+    rollback_batch(s, hb);
+    return rc;
+  }
   const BatchMeta bm = device_meta(s, hb);
   const ModelDims& d = s->dims;
 
@@ -407,26 +429,30 @@ int run_stage(hyp_stage* s, const hyp_batch* b, const void* in, void* out, cudaS
     n_splits = std::min(s->max_splits, attn_decode_fused_splits(hb.n, d.Hkv, max_ctx));
   }
   const bool all = (b->flags & HYP_BATCH_ALL_LOGITS) != 0 || decode;
-  rc = 1;
-  if (decode && s->graphs_ok && s->time_cls < 0) rc = decode_with_graph(s, bm, hb.n, n_splits, in, out, st);
-  if (rc == 1) {
+  auto enqueue = [&]() -> int {
+    int r = 1;
+    if (decode && s->graphs_ok && s->time_cls < 0) r = decode_with_graph(s, bm, hb.n, n_splits, in, out, st);
+    if (r != 1) return r;
     if (io_on_host) {  // eager kernels need device buffers: stage through the I/O buffers
       const size_t in_bytes = s->first ? (size_t)hb.M * sizeof(int32_t) : (size_t)hb.M * d.H * sizeof(float);
       const size_t out_bytes = (size_t)(all ? hb.M : hb.n) * (s->last ? d.V : d.H) * sizeof(float);
       HYP_CUDA_TRY(cudaMemcpyAsync(s->io_in, in, in_bytes, cudaMemcpyHostToDevice, st));
-      rc = enqueue_stage(s, bm, hb.n, decode, all, n_splits, s->io_in, s->io_out, st);
-      if (rc == HYP_OK) HYP_CUDA_TRY(cudaMemcpyAsync(out, s->io_out, out_bytes, cudaMemcpyDeviceToHost, st));
-    } else {
-      rc = enqueue_stage(s, bm, hb.n, decode, all, n_splits, in, out, st);
+      r = enqueue_stage(s, bm, hb.n, decode, all, n_splits, s->io_in, s->io_out, st);
+      if (r == HYP_OK) HYP_CUDA_TRY(cudaMemcpyAsync(out, s->io_out, out_bytes, cudaMemcpyDeviceToHost, st));
+      return r;
+    }
+    return enqueue_stage(s, bm, hb.n, decode, all, n_splits, in, out, st);
+  };
+  rc = enqueue();
+  if (rc == HYP_OK) {
+    cudaError_t e = cudaPeekAtLastError();
+    if (e != cudaSuccess) {
+      set_last_cuda_error((int)e);
+      rc = HYP_ECUDA;
     }
   }
-  if (rc) return rc;
-  cudaError_t e = cudaPeekAtLastError();
-  if (e != cudaSuccess) {
-    set_last_cuda_error((int)e);
-    return HYP_ECUDA;
-  }
-  return HYP_OK;
+  if (rc) rollback_batch(s, hb);
+  return rc;
 }
 
 int run_stage_host(hyp_stage* s, const hyp_batch* b, const void* in, void* out, cudaStream_t st, bool decode) {
@@ -442,18 +468,13 @@ int run_stage_host(hyp_stage* s, const hyp_batch* b, const void* in, void* out, 
   const size_t out_bytes =
       s->last ? (size_t)(all ? M : b->n_seqs) * d.V * sizeof(float) : (size_t)M * d.H * sizeof(float);
   if (in_bytes > s->io_in_bytes || out_bytes > s->io_out_bytes) return HYP_ECAPACITY;
-  // validate before the first copy so that a rejected call moves no data
+  // validate before the first copy so that a rejected call moves no data: a trial admission, taken back at once
   {
     HostBatch probe;
-    std::vector<int32_t> lens(s->seq_len);
-    std::vector<std::vector<int32_t>> pages(s->seq_pages);
-    std::vector<int32_t> freep(s->free_pages);
     int rc = check_ready(s);
     if (!rc) rc = admit_batch(s, b, decode, probe);
-    s->seq_len.swap(lens);
-    s->seq_pages.swap(pages);
-    s->free_pages.swap(freep);
     if (rc) return rc;
+    rollback_batch(s, probe);
   }
   int rc = run_stage(s, b, in, out, st, decode, /*io_on_host=*/true);
   if (rc) return rc;
@@ -520,7 +541,8 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
   if (!cfg || !out) return HYP_EINVAL;
   const hyp_cfg& c = *cfg;
   if (c.n_layers_total < 1 || layer_lo < 0 || layer_hi <= layer_lo || layer_hi > c.n_layers_total) return HYP_EINVAL;
-  if (c.hidden < 8 || c.hidden % 8 || c.ffn < 8 || c.ffn % 8 || c.vocab < 1) return HYP_EINVAL;
+  // every row of an activation, logits or weight matrix must start on a 16-byte boundary (vector stores, TMA)
+  if (c.hidden < 8 || c.hidden % 8 || c.ffn < 8 || c.ffn % 8 || c.vocab < 8 || c.vocab % 8) return HYP_EINVAL;
   if (c.n_kv_heads < 1 || c.n_q_heads < c.n_kv_heads || c.n_q_heads % c.n_kv_heads) return HYP_EINVAL;
   const int G = c.n_q_heads / c.n_kv_heads;
   if (!(G == 1 || G == 2 || G == 4 || G == 8)) return HYP_EINVAL;

@@ -7,12 +7,9 @@ import torch
 from oracle import decoder as od
 from paper_2511_14450_b200 import hyperion as hyp
 from paper_2511_14450_b200 import inputs
+from tests.helpers import build_cache, f64, kv_rows  # noqa: F401
 
 pytestmark = pytest.mark.gpu
-
-
-def f64(t):
-    return t.detach().cpu().to(torch.float64).numpy()
 
 
 def bf16_normal(stream, shape, std=1.0):
@@ -64,17 +61,6 @@ def test_gemm_all_epilogues(M, N, K, epi):
     assert np.max(err) < tol, (np.max(err), np.unravel_index(np.argmax(err), err.shape))
 
 
-def kv_rows(x):
-    """Token rows [slots, Hkv, D] -> the cache's row layout [Hkv, slots, D]: 16-byte chunk c of the token in
-    page slot s sits at chunk position c ^ (s & 7)."""
-    slots, Hkv, D = x.shape
-    c = torch.arange(D // 8, device=x.device)
-    src = (c[None, :] ^ (torch.arange(slots, device=x.device)[:, None] & 7))          # [slots, chunks]
-    xc = x.reshape(slots, Hkv, D // 8, 8)
-    out = torch.gather(xc, 2, src[:, None, :, None].expand(slots, Hkv, D // 8, 8))
-    return out.reshape(slots, Hkv, D).permute(1, 0, 2)
-
-
 @pytest.mark.parametrize("M,N,K", [(1, 256, 256), (8, 528, 1096), (20, 5120, 17920), (33, 512, 256), (128, 272, 328),
                                    (100, 1024, 688), (16, 17920, 512)])
 @pytest.mark.parametrize("epi", [hyp.HYP_EPI_STORE_BF16, hyp.HYP_EPI_RESID_F32, hyp.HYP_EPI_SWIGLU_BF16,
@@ -115,28 +101,6 @@ def test_pack_weight_layout(N, K, swiglu):
                 want[t, kb, r, np.arange(8) ^ (r & 7)] = chunks
     assert packed.size == want.size
     assert np.array_equal(packed, want.reshape(-1))
-
-
-def build_cache(seq_lens, Hkv, D, seed):
-    """Random rotated keys / values (fp16) for each sequence, scattered into a shuffled page pool."""
-    n = len(seq_lens)
-    mpps = max((l + 15) // 16 for l in seq_lens) + 1
-    n_pages = n * mpps + 3
-    perm = torch.from_numpy(np.random.default_rng(seed).permutation(n_pages)).to(torch.int32)
-    pool = torch.zeros(n_pages, 2, Hkv, 16, D, dtype=torch.float16, device="cuda")
-    table = torch.zeros(n, mpps, dtype=torch.int32)
-    ks, vs = [], []
-    for i, L in enumerate(seq_lens):
-        k = bf16_normal(100 + 2 * i + seed, (L, Hkv, D)).half()
-        v = bf16_normal(101 + 2 * i + seed, (L, Hkv, D)).half()
-        ks.append(k); vs.append(v)
-        for p in range((L + 15) // 16):
-            page = int(perm[i * mpps + p])
-            table[i, p] = page
-            t0, t1 = 16 * p, min(L, 16 * p + 16)
-            pool[page, 0, :, :t1 - t0] = kv_rows(k[t0:t1])
-            pool[page, 1, :, :t1 - t0] = kv_rows(v[t0:t1])
-    return pool, table.cuda(), ks, vs
 
 
 @pytest.mark.parametrize("Hq,Hkv,D", [(4, 2, 64), (40, 10, 128), (8, 8, 128), (8, 1, 64)])

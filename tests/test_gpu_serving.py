@@ -1,5 +1,7 @@
 """The multi-stage engine: a model split into stages by HypSplit-DP, continuous batching, every generated
 token crossing every stage; per-step logits of every request against the oracle."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -38,3 +40,36 @@ def test_plan_stages_profiles_and_splits_like_the_enumerator():
     total = torch.cuda.get_device_properties(0).total_memory
     p_e, tau_e = osp.enumerate_split(ms, [float(b) for b in nbytes], [1.0] * 3, [total / 3] * 3)
     assert tuple(bounds[1:-1]) == p_e and tau == tau_e
+
+
+@pytest.mark.skipif(os.environ.get("HYP_SKIP_SLOW") == "1", reason="oracle needs a few minutes; HYP_SKIP_SLOW=1 skips it")
+def test_config3_phi3_shape_three_stages_from_hypsplit_dp_match_oracle():
+    """The serving configuration at the Phi-3-medium shape: all 40 blocks profiled on this GPU, cut into three
+    stages by hyp_split_dp (the cut must equal exhaustive enumeration on the same measured costs), one hyp_stage
+    per tier chained by 5120-wide fp32 hand-offs, continuous batching with more requests than slots and decode
+    batches beyond 8 rows (so the tile and swapped-operand kernels serve the steps); the real per-step logits of
+    every request against the oracle's 40-block full-sequence pass."""
+    sh = inputs.phi3_medium_shape()
+    bounds, tau, ms, nbytes = serving.plan_stages(sh, 3)
+    total = torch.cuda.get_device_properties(0).total_memory
+    p_e, tau_e = osp.enumerate_split(ms, [float(b) for b in nbytes], [1.0] * 3, [total / 3] * 3)
+    assert tuple(bounds[1:-1]) == p_e and tau == tau_e
+    assert all(hi - lo >= 10 for lo, hi in zip(bounds, bounds[1:])), bounds     # near-equal blocks: near-equal tiers
+    lens = [24, 150, 61, 200, 33, 97, 129, 48, 75, 180, 16, 110]
+    n_out, slots = 5, 10
+    reqs = [serving.Request(i, 0.0, inputs.token_ids(inputs.SEED_PROMPTS, 900 + i, lens[i], sh.vocab),
+                            inputs.token_ids(inputs.SEED_FORCED, 900 + i, n_out, sh.vocab), keep_logits=True)
+            for i in range(len(lens))]
+    eng = serving.PipelineEngine(sh, bounds, max_seqs=slots, max_ctx=256, max_tokens=512)
+    stats = eng.run(reqs, realtime=False)
+    eng.close()
+    torch.cuda.empty_cache()
+    assert stats["requests"] == len(lens) and stats["output_tokens"] == len(lens) * n_out
+    assert stats["decode_steps"] == 2 * (n_out - 1)          # ten requests side by side, then the two that waited
+    wants = H.oracle_stage_many(sh, 0, 40, [torch.cat([r.prompt, r.forced[:n_out - 1]]).numpy() for r in reqs])
+    worst = 0.0
+    for r, want in zip(reqs, wants):
+        assert len(r.logits) == n_out
+        got = np.stack([l.numpy() for l in r.logits]).astype(np.float64)
+        worst = max(worst, H.assert_logits_close(got, want[len(r.prompt) - 1:], f"config 3 request {r.rid}"))
+    print(f"config 3: stages {bounds}, worst logit error {worst:.4f}")

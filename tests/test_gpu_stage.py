@@ -159,6 +159,7 @@ def test_error_paths_leave_state_untouched():
     assert code(lambda: st.prefill([0], [8], [3], ids, out)) == hyp.HYP_EINVAL          # wrong cached length
     assert code(lambda: st.prefill([2], [8], [0], ids, out)) == hyp.HYP_EINVAL          # slot out of range
     assert code(lambda: st.prefill([0, 0], [4, 4], [0, 0], ids, out)) == hyp.HYP_EINVAL  # duplicate slot
+    assert code(lambda: st.prefill([0], [8], [0], ids, out.data_ptr() + 4)) == hyp.HYP_EINVAL   # output not 16-byte aligned
     assert hyp.hyp_stage_seq_len(st.handle, 0) == 0 and hyp.hyp_stage_free_pages(st.handle) == 3
     st.prefill([0], [16], [0], ids, out)                                                 # 1 page
     st.prefill([0], [16], [16], ids, out)                                                # 2 pages

@@ -59,19 +59,29 @@ def test_split_dp_ties_with_integer_costs():
         assert hyp.hyp_split_dp(f, m, C, M) == (p_e, tau_e)
 
 
-def test_split_dp_bisection_mode_matches_algorithm_1_step_for_step():
-    for s in range(30):
+def test_split_dp_tolerance_mode_is_within_eps_of_the_enumerated_optimum():
+    """eps > 0 lets the search stop early: the partition returned must be memory-feasible, its reported tau must be
+    its own bottleneck, and that bottleneck must lie within eps of the exhaustive optimum; a tiny eps gives the
+    exact answer.  (The oracle's step-by-step Algorithm 1 is held to the same bound in test_oracle_split.py.)"""
+    hit_inexact = 0
+    for s in range(60):
         N, T = 5 + s % 8, 2 + s % 3
         f, m, C, M = inputs.split_instance(N, T, stream=5000 + s, tight_memory=(s % 4 == 0))
-        eps = 1e-3 * (f.sum() / C.min())
-        p_o, tau_o, _ = osp.hypsplit_dp_bisect(f, m, C, M, eps)
-        if p_o is None:
-            with pytest.raises(hyp.HyperionError):
-                hyp.hyp_split_dp(f, m, C, M, eps)
-            continue
-        assert hyp.hyp_split_dp(f, m, C, M, eps) == (p_o, tau_o)
-        # and it is within eps of the exact optimum
-        assert hyp.hyp_split_dp(f, m, C, M)[1] <= tau_o <= hyp.hyp_split_dp(f, m, C, M)[1] + eps
+        p_e, tau_e = osp.enumerate_split(f, m, C, M)
+        for eps in (0.3 * tau_e if p_e else 1.0, 1e-3, 1e-12):
+            if p_e is None:
+                with pytest.raises(hyp.HyperionError) as ei:
+                    hyp.hyp_split_dp(f, m, C, M, eps)
+                assert ei.value.code == hyp.HYP_EINFEASIBLE
+                continue
+            p, tau = hyp.hyp_split_dp(f, m, C, M, eps)
+            assert list(p) == sorted(set(p)) and all(1 <= c < N for c in p)
+            assert osp.memory_feasible(p, m, M) and tau == max(osp.tier_loads(p, f, C))
+            assert tau_e <= tau <= tau_e + eps
+            hit_inexact += tau > tau_e
+            if eps == 1e-12:
+                assert (p, tau) == (p_e, tau_e)
+    assert hit_inexact > 0          # the loose tolerance really stops early somewhere
 
 
 def test_split_dp_config0_instance_and_40_layer_uniform():
@@ -111,7 +121,7 @@ def test_sched_rt_matches_oracle():
                   "available": bool(r.integers(0, 4))}
             nodes_o.append(nd)
             nodes_l.append((nd["C"], nd["M_avail"], nd["F_rem"], sum(nd["F_wait"]), int(nd["available"])))
-        want = osp.hypsched_rt_scan(4.0, 2.0, nodes_o)
+        want = osp.sched_rt_argmin(4.0, 2.0, nodes_o)        # the definition, not the scan of Algorithm 2
         if want < 0:
             with pytest.raises(hyp.HyperionError) as ei:
                 hyp.hyp_sched_rt(4.0, 2.0, nodes_l)
@@ -189,3 +199,19 @@ def test_compare_splits_report_on_uneven_costs():
                 assert meth[name]["vs_hypsplit_dp"] >= 1.0
         assert abs(sum(rep["memory_limits_bytes"]) - 1.25 * 12) < 1e-9
     assert serving.compare_splits(f, m, 3)["methods"]["even_count"]["vs_hypsplit_dp"] > 1.0
+
+
+def test_stage_create_rejects_shapes_before_touching_the_gpu():
+    """Shape checks come first in hyp_stage_create, so they answer without a GPU: a vocabulary that is not a
+    multiple of 8 (rows of the logits matrix would not start on 16-byte boundaries), an odd hidden size, a group
+    size the attention kernels do not have."""
+    def code(**kw):
+        sh = inputs.tiny_shape()
+        for k, v in kw.items():
+            setattr(sh, k, v)
+        with pytest.raises(hyp.HyperionError) as ei:
+            hyp.hyp_stage_create(0, 1, hyp.make_cfg(sh, 1, 32, 32))
+        return ei.value.code
+    assert code(vocab=1001) == hyp.HYP_EINVAL and code(vocab=4) == hyp.HYP_EINVAL
+    assert code(hidden=100) == hyp.HYP_EINVAL and code(n_q_heads=6) == hyp.HYP_EINVAL
+    assert code(head_dim=96) == hyp.HYP_EINVAL and code(kv_block_size=32) == hyp.HYP_EINVAL
