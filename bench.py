@@ -9,13 +9,17 @@ teacher-forced token ids.  With N > 1 every rank runs an independent replica of 
 GPU (request-level replication, no data-path collective); the value is all ranks' tokens divided by
 the slowest rank's time.
 
-Prints ONE JSON line on rank 0.
+With --gpus N > 1 and no launcher around it (WORLD_SIZE unset) the script starts its own N ranks through
+`python -m torch.distributed.run` on 127.0.0.1.  Prints ONE JSON line on rank 0.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import re
+import socket
 import statistics
 import subprocess
 import sys
@@ -51,6 +55,25 @@ def measured_peaks():
             d = json.load(fh)
         return float(d["hbm_gbs"]), "measured", d
     return FALLBACK_HBM_GBS, "fallback", {}
+
+
+def measured_traffic(profile_name: str):
+    """DRAM bytes per launch (read + write) from a committed ncu summary, or None.  The summary carries two
+    lines, `traffic_bytes_per_launch: N` and `kernel_source: <file> sha256/16 <hex>`; the figure only counts
+    while the kernel's source file still has that hash, i.e. the kernel has not changed since the capture."""
+    path = os.path.join(ROOT, "profiles", profile_name)
+    try:
+        text = open(path).read()
+        n = re.search(r"traffic_bytes_per_launch:\s*([0-9.eE+]+)", text)
+        k = re.search(r"kernel_source:\s*(\S+)\s+sha256/16\s+([0-9a-f]{16})", text)
+        if not n or not k:
+            return None
+        src = os.path.join(ROOT, "paper_2511_14450_b200", "csrc", k.group(1))
+        if hashlib.sha256(open(src, "rb").read()).hexdigest()[:16] != k.group(2):
+            return None
+        return float(n.group(1))
+    except OSError:
+        return None
 
 
 # ------------------------------------------------------------------------------------------
@@ -124,11 +147,14 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------
 # CPU baseline: the oracle, as it stands, on a bounded sample
 # ------------------------------------------------------------------------------------------
+REF_BLOCKS = 2      # blocks of the stage the oracle's step covers (of N_LAYERS_STAGE)
+
+
 def oracle_decode_sample(steps: int, warmup: int):
-    """Time the oracle's literal KV-cached decode on a sample of the workload: ONE sequence through
-    ONE block with a 1024-token cache (seeded random K/V), `steps` single-token steps.  Returns
-    (tokens/s scaled to the 14-block stage, seconds per token-block, threads used, description)."""
-    import numpy as np
+    """Time the oracle's literal KV-cached decode loop on a slice of the workload: the whole batch (8 sequences, a
+    1024-token cache each, seeded random K/V) through REF_BLOCKS of the stage's 14 blocks, `warmup` untimed and
+    `steps` timed steps; a step feeds one new token per sequence.  Returns (seconds per slice step, threads
+    used, description)."""
     from oracle import decoder as od
     from paper_2511_14450_b200 import inputs
     try:
@@ -138,40 +164,94 @@ def oracle_decode_sample(steps: int, warmup: int):
         cores = os.cpu_count() or 1
     sh = inputs.phi3_medium_shape()
     osh = od.Shape(sh.hidden, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.ffn, sh.vocab, sh.rms_eps, sh.rope_theta)
-    w = {k: inputs.bf16_bits_to_f64(v) for k, v in inputs.layer_weights(sh, 0).items()}
-    cs = od.CachedStage([w], osh)
-    cs.k[0] = inputs.bf16_bits_to_f64(inputs.normal_bf16(7, 1, (CTX0, sh.n_kv_heads, sh.head_dim), std=1.0))
-    cs.v[0] = inputs.bf16_bits_to_f64(inputs.normal_bf16(7, 2, (CTX0, sh.n_kv_heads, sh.head_dim), std=1.0))
-    cs.n_cached = CTX0
-    x = inputs.bf16_bits_to_f64(inputs.normal_bf16(7, 3, (warmup + steps, sh.hidden), std=1.0))
-    for i in range(warmup):
-        cs.step(x[i:i + 1])
-    t0 = time.perf_counter()
-    for i in range(warmup, warmup + steps):
-        cs.step(x[i:i + 1])
+    layers = [{k: inputs.bf16_bits_to_f64(v) for k, v in inputs.layer_weights(sh, l).items()} for l in range(REF_BLOCKS)]
+    seqs = []
+    for b in range(BATCH):
+        cs = od.CachedStage(layers, osh)
+        for l in range(REF_BLOCKS):
+            cs.k[l] = inputs.bf16_bits_to_f64(inputs.normal_bf16(7, 10 * b + 2 * l, (CTX0, sh.n_kv_heads, sh.head_dim), std=1.0))
+            cs.v[l] = inputs.bf16_bits_to_f64(inputs.normal_bf16(7, 10 * b + 2 * l + 1, (CTX0, sh.n_kv_heads, sh.head_dim), std=1.0))
+        cs.n_cached = CTX0
+        seqs.append(cs)
+    x = inputs.bf16_bits_to_f64(inputs.normal_bf16(7, 999, (warmup + steps, BATCH, sh.hidden), std=1.0))
+    t0 = 0.0
+    for i in range(warmup + steps):
+        if i == warmup:
+            t0 = time.perf_counter()
+        for b in range(BATCH):
+            seqs[b].step(x[i, b:b + 1])
     dt = (time.perf_counter() - t0) / steps
-    desc = (f"{steps} decode steps of 1 sequence through 1 of the {N_LAYERS_STAGE} blocks at a {CTX0}-token cache "
-            f"(float64 numpy oracle); tokens/s = 1 / ({N_LAYERS_STAGE} x seconds per token-block)")
-    return 1.0 / (N_LAYERS_STAGE * dt), dt, cores, desc
+    desc = (f"{steps} timed decode steps (after {warmup} untimed) of the whole batch ({BATCH} sequences, {CTX0}-token "
+            f"caches) through {REF_BLOCKS} of the stage's {N_LAYERS_STAGE} blocks, float64 numpy oracle, literal "
+            f"KV-cached loop; ms_per_step is that slice step as timed; tokens/s = {BATCH} / (slice step x "
+            f"{N_LAYERS_STAGE}/{REF_BLOCKS})")
+    return dt, cores, desc
+
+
+def oracle_tokens_per_s(dt_slice: float) -> float:
+    return BATCH / (dt_slice * N_LAYERS_STAGE / REF_BLOCKS)
 
 
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    steps = max(1, min(args.steps, 16))
-    warm = max(1, min(args.warmup, 3))
-    tps, dt, cores, desc = oracle_decode_sample(steps, warm)
+    dt, cores, desc = oracle_decode_sample(args.steps, args.warmup)
+    tps = oracle_tokens_per_s(dt)
     line = {
-        "impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-        "warmup": warm, "ms_per_step": dt * 1e3 * N_LAYERS_STAGE * BATCH, "higher_is_better": True,
+        "impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(steps, warm),
+        "config": workload_config(args.steps, args.warmup),
         "cpu_baseline": {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------
+# launch path: N ranks on one node
+# ------------------------------------------------------------------------------------------
+def free_port() -> int:
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def relaunch_with_ranks(n: int, argv) -> int:
+    """`bench.py --gpus N` outside any launcher: start N ranks of this script under torch.distributed.run
+    (one per GPU, rendezvous on 127.0.0.1) and return their exit status."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + list(argv)
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "WARN")
+    return subprocess.call(cmd, env=env)
+
+
+def run_stand_in(args):
+    """The multi-rank bookkeeping of the library arm with the GPU work replaced by a host-side sleep (gloo ranks,
+    no CUDA): used by the CPU test of the launch path, selected by HYP_BENCH_STAND_IN=1.  Same barriers, same
+    max-over-ranks / sum-over-ranks aggregation, same single JSON line on rank 0; `stand_in` marks the line."""
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time.sleep(0.001 * (1 + rank))          # ranks differ, so the max over ranks is visible
+    local_ms = (time.perf_counter() - t0) * 1e3
+    if world > 1:
+        dist.barrier()
+    ms, tokens = aggregate_over_ranks(local_ms, BATCH * args.steps, dist if world > 1 else None, "cpu")
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": tokens / (ms / 1e3), "unit": UNIT, "n_gpus": world,
+                          "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+                          "higher_is_better": True, "scaling": "weak", "stand_in": True, "gpu_launches": 0}))
+    if world > 1:
+        dist.destroy_process_group()
 
 
 # ------------------------------------------------------------------------------------------
@@ -190,7 +270,11 @@ def run_ours(args):
         raise RuntimeError("bench.py needs a CUDA device: the library has no CPU fallback")
     torch.cuda.set_device(local)
     if world > 1:
+        os.environ.setdefault("NCCL_DEBUG", "WARN")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if rank == 0:
+            print(f"[bench] {world} ranks, backend nccl {'.'.join(str(v) for v in torch.cuda.nccl.version())}, "
+                  f"one replica of the stage per GPU", file=sys.stderr)
     K, W = args.steps, max(args.warmup, 3)
     sh = inputs.phi3_medium_shape()
     max_ctx = CTX0 + W + 3 * K + 16
@@ -291,6 +375,15 @@ def run_ours(args):
 
     st.close()
     prefill = prefill_config1(torch, hyp, inputs, stream) if world == 1 else None
+    extras = {}
+    if world == 1 and not args.no_extras:
+        # the two other full-model configurations, so that the run's record carries them (one GPU only)
+        from paper_2511_14450_b200 import longgen, serving
+        torch.cuda.empty_cache()
+        extras["longgen"] = longgen.run(steps=args.longgen_steps)
+        torch.cuda.empty_cache()
+        extras["serving"] = serving.run_closed_loop()
+        torch.cuda.empty_cache()
 
     if rank == 0:
         line = {
@@ -306,7 +399,8 @@ def run_ours(args):
                          "frac": (achieved / peak) if achieved else None, "peak_source": f"of {peak_src}",
                          "bytes_per_launch": gu_bytes, "launches_timed": n_k,
                          "avg_launch_us": (k_ms / n_k * 1e3) if n_k else None,
-                         "traffic": 371.2e6,   # dram read + write per launch, profiles/gemm_stream_gateup_M8.md
+                         "traffic": measured_traffic("gemm_stream_gateup_M8.md"),   # ncu dram read + write per launch
+                         "whole_step_frac": step_gbs / peak, "whole_step_frac_of_nominal_8TBs": step_gbs / 8000.0,
                          "timed_in": "second pass of K steps with per-launch events (kernel-by-kernel launches)",
                          "kernel_pass_ms_per_step": kernel_pass_ms},
             "step_roofline": {"bound": "hbm", "bytes_per_step": step_bytes, "achieved": step_gbs, "peak": peak,
@@ -314,9 +408,11 @@ def run_ours(args):
         }
         if prefill is not None:
             line["prefill"] = prefill
+        line.update(extras)
         if not args.no_cpu_baseline and world == 1:
-            tps, dt, cores, desc = oracle_decode_sample(4, 1)
-            line["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+            dt, cores, desc = oracle_decode_sample(4, 1)
+            line["cpu_baseline"] = {"value": oracle_tokens_per_s(dt), "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": desc}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -333,7 +429,7 @@ def prefill_config1(torch, hyp, inputs, stream, iters=10):
     st.load_embed(inputs.embed_weights(sh, device="cuda"))
     ids = inputs.token_ids(inputs.SEED_PROMPTS, 0, M, sh.vocab, device="cuda")
     out = torch.empty(M, sh.hidden, dtype=torch.float32, device="cuda")
-    # a second weight set alternates with the first so that no launch finds its weights in L2
+    # the block's 681 MB of weights exceed L2, so every pass streams them from HBM again
     for _ in range(3):
         st.prefill([0], [M], [0], ids, out)
         st.free_seq(0)
@@ -377,7 +473,7 @@ def prefill_config1(torch, hyp, inputs, stream, iters=10):
                      "peak_source": "of measured (burst)" if peaks else "of fallback",
                      "frac_of_nominal_2250": achieved / 2250.0, "flops": gemm_flops,
                      "dominant_kernel_tflops": gu, "dominant_kernel_frac": gu / peak,
-                     "traffic": 401.7e6},  # gate/up launch, dram read + write, profiles/gemm_tc2_gateup_M512.md
+                     "traffic": measured_traffic("gemm_tc2_gateup_M512.md")},   # gate/up launch, ncu dram read + write
     }
 
 
@@ -388,9 +484,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the configs[3] / configs[4] objects")
+    ap.add_argument("--longgen-steps", type=int, default=2048)
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(relaunch_with_ranks(args.gpus, sys.argv[1:]))
     if args.impl == "reference":
         run_reference(args)
+    elif os.environ.get("HYP_BENCH_STAND_IN") == "1":
+        run_stand_in(args)
     else:
         run_ours(args)
 

@@ -84,10 +84,14 @@ HYP_API int hyp_op_gemm(const void* a, const void* w_packed, int32_t M, int32_t 
  *   HYP_TUNE_PREFILL_ATTN_TC  value != 0 (the default): prefill attention at head_dim 128 runs on the tcgen05 kernel
  *                          (scores, probabilities and output in tensor memory, 128 query rows per CTA); 0: on the
  *                          mma.sync kernel that serves the other head sizes
+ *   HYP_TUNE_FIRST_BLOCK_SPLIT  value != 0 (the default): in stages that hold block 0 the attention scores of that
+ *                          block are formed from two-term fp16 queries and keys (~21 significant bits) and the
+ *                          RMSNorm factor is applied after the q/k/v projection, whose input is then the embedding
+ *                          row itself; 0: block 0 runs like every other block (11-bit operands)
  * Affects launches made after the call; decode graphs already captured keep their setting. */
 enum { HYP_TUNE_PDL = 0, HYP_TUNE_STREAM_SLOTS = 1, HYP_TUNE_ATTN_SPLITS = 2, HYP_TUNE_ATTN_SLOTS = 3,
        HYP_TUNE_STREAM_ROTATION = 4, HYP_TUNE_SWAP_MIN_ROWS = 5, HYP_TUNE_SWAP_MAX_ROWS = 6, HYP_TUNE_SWAP_EPILOGUES = 7,
-       HYP_TUNE_PREFILL_ATTN_TC = 8 };
+       HYP_TUNE_PREFILL_ATTN_TC = 8, HYP_TUNE_FIRST_BLOCK_SPLIT = 9 };
 HYP_API int hyp_tune(int32_t key, int32_t value);
 
 /* Number of context splits hyp_op_attn_decode would pick for this batch, and the scratch bytes

@@ -38,21 +38,27 @@ struct AttnFusedArgs {
   __half* out;               // [n_seqs, Hq * D]
   int slots;                 // ring slots per warp
   int* err;
+  // SPLIT instantiation only (the model's first block): the rows of qkv32 still lack the RMSNorm factor
+  // row_scale[b], and queries / keys are two-term fp16 values, the keys' low terms cached in klo_layer
+  // ([page][Hkv][16][D], the cache's row order), so that the scores carry ~21 significant bits
+  const float* row_scale;
+  __half* klo_layer;
 };
 
 __device__ __forceinline__ __half f16_sat(float x) { return __float2half_rn(fminf(fmaxf(x, -65504.f), 65504.f)); }
-template <int D, int G>
+template <int D, int G, bool SPLIT>
 __global__ void __launch_bounds__(AF_THREADS)
 attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
   constexpr int KS = D / 16, DN = D / 8, CPR = D / 8;
   constexpr int PAGE_BYTES = AF_PT * D * 2;   // 16 keys (or values) of one KV head
-  constexpr int SLOT_BYTES = 2 * PAGE_BYTES;  // keys, then values
+  constexpr int SLOT_BYTES = (SPLIT ? 3 : 2) * PAGE_BYTES;  // keys, then values (then the keys' low terms)
   extern __shared__ __align__(128) uint8_t af_smem[];
   __shared__ uint64_t bars[AF_WARPS * AF_MAX_SLOTS];
   __shared__ float ex_m[8], ex_l[8];              // this CTA's partial: running maximum (log2 units), denominator
   __shared__ __align__(16) float ex_o[G * D];     // and weighted value sum, read by the whole cluster
   __shared__ __align__(16) __half sq[G * D];      // rotated queries
-  __shared__ __align__(16) __half snew[2 * D];    // the new token's rotated key, then its value
+  __shared__ __align__(16) __half snew[3 * D];    // the new token's rotated key, then its value (then the key's low term)
+  __shared__ __align__(16) __half sq_lo[SPLIT ? G * D : 8];  // low terms of the rotated queries
   const int S = a.slots;
   const uint32_t ring0 = (smem_u32(af_smem) + 127u) & ~127u;
   uint8_t* ring_ptr = af_smem + (ring0 - smem_u32(af_smem));
@@ -89,6 +95,7 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
     mbar_expect_tx(bar, SLOT_BYTES);
     bulk_load(dst, src, PAGE_BYTES, bar);
     bulk_load(dst + PAGE_BYTES, src + v_off, PAGE_BYTES, bar);
+    if (SPLIT) bulk_load(dst + 2 * PAGE_BYTES, a.klo_layer + ((size_t)page * d.Hkv + kvh) * AF_PT * D, PAGE_BYTES, bar);
   };
   pdl_trigger();
   if (lane == 0) {
@@ -107,23 +114,32 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
   {
     const float* row = a.qkv32 + (size_t)b * a.stride;
     const float2* cs = a.rope_table + (size_t)pos * (D / 2);
+    const float rs = SPLIT ? a.row_scale[b] : 1.f;
     for (int e = threadIdx.x; e < G * (D / 2); e += AF_THREADS) {
       const int gq = e / (D / 2), i = e % (D / 2);
       const float* hp = row + (size_t)(kvh * G + gq) * D;
-      const float x1 = hp[i], x2 = hp[i + D / 2];
+      const float x1 = hp[i] * rs, x2 = hp[i + D / 2] * rs;
       const float2 c = cs[i];
-      sq[gq * D + i] = f16_sat(x1 * c.x - x2 * c.y);
-      sq[gq * D + i + D / 2] = f16_sat(x2 * c.x + x1 * c.y);
+      const float r1 = x1 * c.x - x2 * c.y, r2 = x2 * c.x + x1 * c.y;
+      const __half h1 = f16_sat(r1), h2 = f16_sat(r2);
+      sq[gq * D + i] = h1;
+      sq[gq * D + i + D / 2] = h2;
+      if (SPLIT) {
+        sq_lo[gq * D + i] = __float2half_rn(r1 - __half2float(h1));
+        sq_lo[gq * D + i + D / 2] = __float2half_rn(r2 - __half2float(h2));
+      }
     }
     if (owner_cta) {
       const float* kp = row + (size_t)(d.Hq + kvh) * D;
       const float* vp = row + (size_t)(d.Hq + d.Hkv + kvh) * D;
       __half* dk = a.kv_layer + (size_t)bt[page_new] * page_elems + ((size_t)kvh * AF_PT + slot_new) * D;
+      __half* dkl = SPLIT ? a.klo_layer + (((size_t)bt[page_new] * d.Hkv + kvh) * AF_PT + slot_new) * D : nullptr;
       for (int i = threadIdx.x; i < D / 2; i += AF_THREADS) {
-        const float x1 = kp[i], x2 = kp[i + D / 2];
+        const float x1 = kp[i] * rs, x2 = kp[i + D / 2] * rs;
         const float2 c = cs[i];
-        const __half k1 = f16_sat(x1 * c.x - x2 * c.y), k2 = f16_sat(x2 * c.x + x1 * c.y);
-        const __half v1 = f16_sat(vp[i]), v2 = f16_sat(vp[i + D / 2]);
+        const float r1 = x1 * c.x - x2 * c.y, r2 = x2 * c.x + x1 * c.y;
+        const __half k1 = f16_sat(r1), k2 = f16_sat(r2);
+        const __half v1 = f16_sat(vp[i] * rs), v2 = f16_sat(vp[i + D / 2] * rs);
         snew[i] = k1; snew[i + D / 2] = k2;
         snew[D + i] = v1; snew[D + i + D / 2] = v2;
         // the cache keeps them for the following steps, in its chunk-permuted row layout
@@ -131,6 +147,11 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
         const int j2 = (kv_chunk_pos((i + D / 2) >> 3, slot_new) << 3) + (i & 7);
         dk[j1] = k1; dk[j2] = k2;
         dk[v_off + j1] = v1; dk[v_off + j2] = v2;
+        if (SPLIT) {
+          const __half l1 = __float2half_rn(r1 - __half2float(k1)), l2 = __float2half_rn(r2 - __half2float(k2));
+          snew[2 * D + i] = l1; snew[2 * D + i + D / 2] = l2;
+          dkl[j1] = l1; dkl[j2] = l2;
+        }
       }
     }
   }
@@ -144,6 +165,15 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
     for (int ks = 0; ks < KS; ++ks) {
       qf[ks][0] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * tq) : 0u;
       qf[ks][1] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * tq) : 0u;
+    }
+  }
+  uint32_t qfl[SPLIT ? KS : 1][2];
+  if (SPLIT) {
+    const __half* qrow = sq_lo + (g < G ? g : 0) * D;
+#pragma unroll
+    for (int ks = 0; ks < (SPLIT ? KS : 1); ++ks) {
+      qfl[ks][0] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * tq) : 0u;
+      qfl[ks][1] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * tq) : 0u;
     }
   }
   const float sl2 = rsqrtf((float)D) * 1.4426950408889634f;
@@ -163,10 +193,10 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
     const bool patched = pi == page_new;
     if (patched) {
       // this page was copied while its last row was being written: put the new key / value over it
-      if (lane < 2 * CPR) {
-        const int which = lane / CPR, c = lane % CPR;
+      for (int e = lane; e < (SPLIT ? 3 : 2) * CPR; e += 32) {
+        const int which = e / CPR, c = e % CPR;   // 0 key, 1 value, 2 key's low term
         const uint4 v = *reinterpret_cast<const uint4*>(snew + which * D + c * 8);
-        const uint32_t dst = (which ? vt : kt) + tile_off<D>(slot_new, c);
+        const uint32_t dst = kt + which * PAGE_BYTES + tile_off<D>(slot_new, c);
         asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
       }
       __syncwarp();
@@ -184,6 +214,14 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
       ldsm_x4(kt + tile_off<D>(r, c), b0, b1, b2, b3);
       mma_f16_16816(s[0], qf[ks][0], 0u, qf[ks][1], 0u, b0, b1);
       mma_f16_16816(s[1], qf[ks][0], 0u, qf[ks][1], 0u, b2, b3);
+      if (SPLIT) {
+        const int kq = SPLIT ? ks : 0;
+        mma_f16_16816(s[0], qfl[kq][0], 0u, qfl[kq][1], 0u, b0, b1);
+        mma_f16_16816(s[1], qfl[kq][0], 0u, qfl[kq][1], 0u, b2, b3);
+        ldsm_x4(kt + 2 * PAGE_BYTES + tile_off<D>(r, c), b0, b1, b2, b3);
+        mma_f16_16816(s[0], qf[ks][0], 0u, qf[ks][1], 0u, b0, b1);
+        mma_f16_16816(s[1], qf[ks][0], 0u, qf[ks][1], 0u, b2, b3);
+      }
     }
     const int key0 = pi * AF_PT + 2 * tq;
     float mx = m_run;
@@ -302,15 +340,15 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
   cluster_barrier();  // nobody leaves while a peer may still read its partial
 }
 
-template <int D, int G>
+template <int D, int G, bool SPLIT>
 int launch_dg(const AttnFusedArgs& a_in, int n_splits, const BatchMeta& bm, const ModelDims& d, cudaStream_t st) {
   static bool configured = false;
-  constexpr int SLOT_BYTES = 2 * AF_PT * D * 2;
+  constexpr int SLOT_BYTES = (SPLIT ? 3 : 2) * AF_PT * D * 2;
   constexpr int COMBINE_BYTES = (2 * AF_WARPS * 8 + AF_WARPS * G * D) * 4;
   constexpr int MAX_DYN = AF_WARPS * AF_MAX_SLOTS * SLOT_BYTES + 128;
   static_assert(AF_WARPS * 2 * SLOT_BYTES >= COMBINE_BYTES, "the combine buffers reuse the ring");
   if (!configured) {
-    HYP_CUDA_TRY(cudaFuncSetAttribute(attn_decode_fused_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN));
+    HYP_CUDA_TRY(cudaFuncSetAttribute(attn_decode_fused_kernel<D, G, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN));
     configured = true;
   }
   AttnFusedArgs a = a_in;
@@ -332,7 +370,7 @@ int launch_dg(const AttnFusedArgs& a_in, int n_splits, const BatchMeta& bm, cons
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl_level() >= 3 ? 2 : 1;  // measured: launching it early at level 2 costs 2 %
-  HYP_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_decode_fused_kernel<D, G>, a, bm, d));
+  HYP_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_decode_fused_kernel<D, G, SPLIT>, a, bm, d));
   return 1;
 }
 
@@ -340,6 +378,10 @@ int launch_dg(const AttnFusedArgs& a_in, int n_splits, const BatchMeta& bm, cons
 
 int& attn_fused_splits_override() {
   static int v = 0;
+  return v;
+}
+int& first_block_split() {
+  static int v = 1;
   return v;
 }
 int& attn_fused_slots_override() {
@@ -360,14 +402,16 @@ int attn_decode_fused_splits(int n_seqs, int Hkv, int max_ctx) {
 }
 
 int launch_attn_decode_fused(const float* qkv32, int stride, __half* kv_layer, const float2* rope_table, __half* attn_out,
-                             int n_splits, int slots, int* err, const BatchMeta& bm, const ModelDims& d, cudaStream_t st) {
-  if (n_splits < 1 || n_splits > 8 || !err) return HYP_EINVAL;
+                             int n_splits, int slots, int* err, const BatchMeta& bm, const ModelDims& d, cudaStream_t st,
+                             const float* row_scale, __half* klo_layer) {
+  if (n_splits < 1 || n_splits > 8 || !err || (row_scale != nullptr) != (klo_layer != nullptr)) return HYP_EINVAL;
   AttnFusedArgs a;
   a.qkv32 = qkv32; a.stride = stride; a.kv_layer = kv_layer; a.rope_table = rope_table; a.out = attn_out;
-  a.slots = slots; a.err = err;
+  a.slots = slots; a.err = err; a.row_scale = row_scale; a.klo_layer = klo_layer;
   const int G = d.Hq / d.Hkv;
-#define HYP_AF_CASE(DD, GG) \
-  if (d.D == DD && G == GG) return launch_dg<DD, GG>(a, n_splits, bm, d, st);
+#define HYP_AF_CASE(DD, GG)                                                \
+  if (d.D == DD && G == GG)                                                \
+    return row_scale ? launch_dg<DD, GG, true>(a, n_splits, bm, d, st) : launch_dg<DD, GG, false>(a, n_splits, bm, d, st);
   HYP_AF_CASE(128, 1) HYP_AF_CASE(128, 2) HYP_AF_CASE(128, 4) HYP_AF_CASE(128, 8)
   HYP_AF_CASE(64, 1) HYP_AF_CASE(64, 2) HYP_AF_CASE(64, 4) HYP_AF_CASE(64, 8)
 #undef HYP_AF_CASE

@@ -18,9 +18,14 @@ namespace {
 
 constexpr int FA_BQ = 64, FA_BKV = 64, FA_THREADS = 128, PT = 16;
 
-template <int D>
-__global__ void __launch_bounds__(FA_THREADS, 3)
+// SPLIT: the scores are formed from two-term operands, q = q_hi + q_lo and k = k_hi + k_lo (each term fp16, the low
+// term the rounding residue of the high one), as q_hi k_hi + q_lo k_hi + q_hi k_lo: ~21 significant bits instead of
+// 11.  `q_lo` has the layout of `qkv`; `klo_layer` is a pool [page][Hkv][16][D] with the cache's row order.  Used for
+// the model's first block, whose attention errors the rest of the network amplifies most (see stage.cu).
+template <int D, bool SPLIT>
+__global__ void __launch_bounds__(FA_THREADS, SPLIT ? 2 : 3)
 attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict__ kv_layer,
+                       const __half* __restrict__ q_lo_buf, const __half* __restrict__ klo_layer,
                        __half* __restrict__ out, BatchMeta bm, ModelDims d, int* __restrict__ err) {
   constexpr int KS = D / 16;       // k-steps of the QK^T contraction
   constexpr int DN = D / 8;        // 8-wide output column tiles of O
@@ -28,9 +33,10 @@ attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict_
   constexpr int TILE_BYTES = FA_BKV * D * 2;
   extern __shared__ __align__(128) uint8_t fa_smem[];
   const uint32_t smem0 = (uint32_t)__cvta_generic_to_shared(fa_smem);
-  // layout: K[2] then V[2]
+  // layout: K[2] then V[2] (then the low terms of K[2])
   auto k_tile = [&](int buf) { return smem0 + buf * TILE_BYTES; };
   auto v_tile = [&](int buf) { return smem0 + (2 + buf) * TILE_BYTES; };
+  auto klo_tile = [&](int buf) { return smem0 + (4 + buf) * TILE_BYTES; };
 
   __shared__ uint64_t kv_bars[2];
   constexpr int PAGE_BYTES = PT * D * 2;  // the 16 keys (or values) of one page and KV head: contiguous in the cache
@@ -74,11 +80,14 @@ attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict_
     const int p0 = j * (FA_BKV / PT);
     const int n_valid = min(FA_BKV / PT, n_pages_seq - p0);
     if (threadIdx.x == 0) {
-      mbar_expect_tx(bar0 + 8u * buf, (uint32_t)(2 * n_valid * PAGE_BYTES));
+      mbar_expect_tx(bar0 + 8u * buf, (uint32_t)((SPLIT ? 3 : 2) * n_valid * PAGE_BYTES));
       for (int pi = 0; pi < n_valid; ++pi) {
         const __half* src = kv_layer + (size_t)bt[p0 + pi] * page_elems + (size_t)kvh * PT * D;
         bulk_load(k_tile(buf) + pi * PAGE_BYTES, src, PAGE_BYTES, bar0 + 8u * buf);
         bulk_load(v_tile(buf) + pi * PAGE_BYTES, src + v_off, PAGE_BYTES, bar0 + 8u * buf);
+        if (SPLIT)
+          bulk_load(klo_tile(buf) + pi * PAGE_BYTES, klo_layer + ((size_t)bt[p0 + pi] * d.Hkv + kvh) * PT * D, PAGE_BYTES,
+                    bar0 + 8u * buf);
       }
     }
     if (n_valid < FA_BKV / PT) {
@@ -86,6 +95,8 @@ attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict_
       for (int o = threadIdx.x * 16; o < bytes; o += FA_THREADS * 16) {
         asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(k_tile(buf) + n_valid * PAGE_BYTES + o), "r"(0u) : "memory");
         asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(v_tile(buf) + n_valid * PAGE_BYTES + o), "r"(0u) : "memory");
+        if (SPLIT)
+          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(klo_tile(buf) + n_valid * PAGE_BYTES + o), "r"(0u) : "memory");
       }
     }
   };
@@ -105,6 +116,20 @@ attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict_
       qf[ks][1] = ok_hi ? *reinterpret_cast<const uint32_t*>(q_hi + 16 * ks + 2 * tq) : 0u;
       qf[ks][2] = ok_lo ? *reinterpret_cast<const uint32_t*>(q_lo + 16 * ks + 8 + 2 * tq) : 0u;
       qf[ks][3] = ok_hi ? *reinterpret_cast<const uint32_t*>(q_hi + 16 * ks + 8 + 2 * tq) : 0u;
+    }
+  }
+  uint32_t qfl[SPLIT ? KS : 1][4];  // low terms of the same fragments
+  if (SPLIT) {
+    const int r_lo = 16 * warp + g, r_hi = r_lo + 8;
+    const __half* q_lo = q_lo_buf + (size_t)(row_base + r_lo) * d.qkv_rows + (size_t)hq * D;
+    const __half* q_hi = q_lo_buf + (size_t)(row_base + r_hi) * d.qkv_rows + (size_t)hq * D;
+    const bool ok_lo = r_lo < rows_here, ok_hi = r_hi < rows_here;
+#pragma unroll
+    for (int ks = 0; ks < (SPLIT ? KS : 1); ++ks) {
+      qfl[ks][0] = ok_lo ? *reinterpret_cast<const uint32_t*>(q_lo + 16 * ks + 2 * tq) : 0u;
+      qfl[ks][1] = ok_hi ? *reinterpret_cast<const uint32_t*>(q_hi + 16 * ks + 2 * tq) : 0u;
+      qfl[ks][2] = ok_lo ? *reinterpret_cast<const uint32_t*>(q_lo + 16 * ks + 8 + 2 * tq) : 0u;
+      qfl[ks][3] = ok_hi ? *reinterpret_cast<const uint32_t*>(q_hi + 16 * ks + 8 + 2 * tq) : 0u;
     }
   }
 
@@ -141,6 +166,14 @@ attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict_
         ldsm_x4(k_tile(buf) + tile_off<D>(r, c), b0, b1, b2, b3);
         mma_f16_16816(s[2 * np], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b0, b1);
         mma_f16_16816(s[2 * np + 1], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b2, b3);
+        if (SPLIT) {
+          const int kq = SPLIT ? ks : 0;
+          mma_f16_16816(s[2 * np], qfl[kq][0], qfl[kq][1], qfl[kq][2], qfl[kq][3], b0, b1);
+          mma_f16_16816(s[2 * np + 1], qfl[kq][0], qfl[kq][1], qfl[kq][2], qfl[kq][3], b2, b3);
+          ldsm_x4(klo_tile(buf) + tile_off<D>(r, c), b0, b1, b2, b3);
+          mma_f16_16816(s[2 * np], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b0, b1);
+          mma_f16_16816(s[2 * np + 1], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b2, b3);
+        }
       }
     }
 
@@ -227,21 +260,21 @@ attn_prefill_fa_kernel(const __half* __restrict__ qkv, const __half* __restrict_
   }
 }
 
-template <int D>
-int launch_fa(const __half* qkv, const __half* kv_layer, __half* attn_out, const BatchMeta& bm,
-              const ModelDims& d, cudaStream_t st) {
+template <int D, bool SPLIT>
+int launch_fa(const __half* qkv, const __half* kv_layer, const __half* q_lo, const __half* klo_layer, __half* attn_out,
+              const BatchMeta& bm, const ModelDims& d, cudaStream_t st) {
   static bool configured = false;
-  constexpr int smem = 4 * FA_BKV * D * 2;
+  constexpr int smem = (SPLIT ? 6 : 4) * FA_BKV * D * 2;
   int rc = tc_prepare();  // the device word that bounded waits report to
   if (rc) return rc;
   if (!configured) {
-    HYP_CUDA_TRY(cudaFuncSetAttribute(attn_prefill_fa_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    HYP_CUDA_TRY(cudaFuncSetAttribute(attn_prefill_fa_kernel<D, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     configured = true;
   }
   // every sequence adds at most one ragged tile on top of floor(rows / 64)
   const int max_tiles = bm.n_tokens / FA_BQ + bm.n_seqs;
-  HYP_CUDA_TRY(launch_pdl<2>(attn_prefill_fa_kernel<D>, dim3(d.Hq, max_tiles), dim3(FA_THREADS), smem, st, qkv, kv_layer,
-                          attn_out, bm, d, tc_err_flag_ptr()));
+  HYP_CUDA_TRY(launch_pdl<2>(attn_prefill_fa_kernel<D, SPLIT>, dim3(d.Hq, max_tiles), dim3(FA_THREADS), smem, st, qkv,
+                             kv_layer, q_lo, klo_layer, attn_out, bm, d, tc_err_flag_ptr()));
   return 1;
 }
 
@@ -252,8 +285,20 @@ int launch_attn_prefill(const __half* q, int q_stride, const __half* kv_layer, _
                         const BatchMeta& bm, const ModelDims& d_in, cudaStream_t st) {
   ModelDims d = d_in;
   d.qkv_rows = q_stride;
-  if (d.D == 128) return launch_fa<128>(q, kv_layer, attn_out, bm, d, st);
-  if (d.D == 64) return launch_fa<64>(q, kv_layer, attn_out, bm, d, st);
+  if (d.D == 128) return launch_fa<128, false>(q, kv_layer, nullptr, nullptr, attn_out, bm, d, st);
+  if (d.D == 64) return launch_fa<64, false>(q, kv_layer, nullptr, nullptr, attn_out, bm, d, st);
+  return HYP_EINVAL;
+}
+
+// The same attention with two-term queries and keys (q_lo: layout of q; klo_layer: [page][Hkv][16][D]).
+int launch_attn_prefill_split(const __half* q, const __half* q_lo, int q_stride, const __half* kv_layer,
+                              const __half* klo_layer, __half* attn_out, const BatchMeta& bm, const ModelDims& d_in,
+                              cudaStream_t st) {
+  ModelDims d = d_in;
+  d.qkv_rows = q_stride;
+  if (!q_lo || !klo_layer) return HYP_EINVAL;
+  if (d.D == 128) return launch_fa<128, true>(q, kv_layer, q_lo, klo_layer, attn_out, bm, d, st);
+  if (d.D == 64) return launch_fa<64, true>(q, kv_layer, q_lo, klo_layer, attn_out, bm, d, st);
   return HYP_EINVAL;
 }
 

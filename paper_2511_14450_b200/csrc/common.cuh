@@ -150,13 +150,21 @@ int launch_copy_f32(const float* src, float* dst, size_t n, cudaStream_t st);
 // h = norm(x) as bf16, or as fp16 when out_f16 (h then points to __half storage)
 int launch_rmsnorm(const float* x, const __nv_bfloat16* g, void* h, bool out_f16, int M, int H, float eps,
                    const int32_t* row_index /* optional gather of rows, may be null */, cudaStream_t st,
-                   bool gains_are_constant = false /* true: g is a loaded weight, never a predecessor's output */);
+                   bool gains_are_constant = false /* true: g is a loaded weight, never a predecessor's output */,
+                   float* defer_scale = nullptr /* non-null: h = x * g * 2^e, defer_scale[r] = rstd / 2^e (fp16 only) */);
 // rotate q, k of every row (fp32 in), write q as fp16 [M, Hq*D] and append k, v as fp16 to the pages
+// row_scale non-null: rows are multiplied by row_scale[t] first, and q, k are stored as two fp16 terms (the low
+// terms to q_lo [M, Hq*D] and klo_layer [page][Hkv][16][D])
 int launch_rope_kv_write(const float* qkv, __half* q16, __half* kv_layer, const float2* rope_table,
-                         const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
+                         const BatchMeta& bm, const ModelDims& d, cudaStream_t st, const float* row_scale = nullptr,
+                         __half* q_lo = nullptr, __half* klo_layer = nullptr);
 // q: fp16 [M, q_stride]
 int launch_attn_prefill(const __half* q, int q_stride, const __half* kv_layer, __half* attn_out,
                         const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
+// the same with two-term queries and keys (see launch_rope_kv_write)
+int launch_attn_prefill_split(const __half* q, const __half* q_lo, int q_stride, const __half* kv_layer,
+                              const __half* klo_layer, __half* attn_out, const BatchMeta& bm, const ModelDims& d,
+                              cudaStream_t st);
 // decode attention: one query row per sequence; `scratch` holds split partials
 size_t attn_decode_scratch_bytes(int max_seqs, int Hq, int D, int max_splits);
 int attn_decode_splits(int n_seqs, int Hkv, int max_ctx);
@@ -167,9 +175,13 @@ int launch_attn_decode(const __half* q, int q_stride, const __half* kv_layer, __
 // projection output, one row per sequence), appends k, v to the pages, attends over n_splits context slices
 // (a thread-block cluster, n_splits <= 8) and merges them.  `err`: device word set if a bounded wait expires.
 int attn_decode_fused_splits(int n_seqs, int Hkv, int max_ctx);
+int& first_block_split();           // 1 (default): the model's first block keeps two-term queries / keys
 int& attn_fused_splits_override();  // 0 = built-in choice
 int& attn_fused_slots_override();   // 0 = built-in choice
+// row_scale / klo_layer (both or neither): the first block's variant - rows of qkv32 are multiplied by row_scale[b]
+// first, and queries / keys are two-term fp16 values (the keys' low terms cached in klo_layer [page][Hkv][16][D]).
 int launch_attn_decode_fused(const float* qkv32, int stride, __half* kv_layer, const float2* rope_table, __half* attn_out,
-                             int n_splits, int slots, int* err, const BatchMeta& bm, const ModelDims& d, cudaStream_t st);
+                             int n_splits, int slots, int* err, const BatchMeta& bm, const ModelDims& d, cudaStream_t st,
+                             const float* row_scale = nullptr, __half* klo_layer = nullptr);
 
 }  // namespace hyp

@@ -47,10 +47,14 @@ int launch_copy_f32(const float* src, float* dst, size_t n, cudaStream_t st) {
 // h[r, :] = x[row, :] * rsqrt(mean(x[row, :]^2) + eps) * g, one CTA per output row.
 // row = row_index ? row_index[r] : r.  fp32 statistics; output bf16, or fp16 for the q/k/v projection
 // (whose inputs need fp16's 11 mantissa bits to keep the softmax weights inside the logit tolerance).
-template <int THREADS, bool F16>
+// DEFER (the model's first block, whose input rows are embedding rows, i.e. bf16 values): the row is written
+// as x * g * 2^e with 2^e the power of two just below the normalisation factor, and the remaining factor
+// rstd / 2^e in [1, 2) goes to row_scale[r] for the consumer of the projection to apply.  x * 2^e is exact, so
+// with unit gains the projection's fp16 input carries no rounding error at all (and never more than before).
+template <int THREADS, bool F16, bool DEFER = false>
 __global__ void __launch_bounds__(THREADS, 1280 / THREADS)  // <= 51 registers: five 256-thread CTAs per SM
 rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ g, void* __restrict__ h,
-                               int H, float eps, const int32_t* __restrict__ row_index) {
+                               int H, float eps, const int32_t* __restrict__ row_index, float* __restrict__ row_scale) {
   constexpr int CACHE = 5;  // float4 per thread kept in registers: rows up to THREADS * 20 wide are read once
   __shared__ float red[THREADS / 32];
   const int r = blockIdx.x;
@@ -85,7 +89,12 @@ rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ g,
   float tot = 0.f;
 #pragma unroll
   for (int w = 0; w < THREADS / 32; ++w) tot += red[w];
-  const float rstd = rsqrtf(tot / (float)H + eps);
+  float rstd = rsqrtf(tot / (float)H + eps);
+  if (DEFER) {
+    const float pow2 = __uint_as_float(__float_as_uint(rstd) & 0x7f800000u);  // 2^floor(log2(rstd))
+    if (threadIdx.x == 0) row_scale[r] = rstd / pow2;
+    rstd = pow2;
+  }
   uint2* hr = reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(h) + (size_t)r * H);
   auto emit = [&](int i, const float4& v, const uint2 gg) {
     const float y0 = v.x * rstd * bf16_lo(gg.x), y1 = v.y * rstd * bf16_hi(gg.x);
@@ -104,19 +113,26 @@ rmsnorm_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ g,
 }
 
 int launch_rmsnorm(const float* x, const __nv_bfloat16* g, void* h, bool out_f16, int M, int H, float eps,
-                   const int32_t* row_index, cudaStream_t st, bool gains_are_constant) {
+                   const int32_t* row_index, cudaStream_t st, bool gains_are_constant, float* defer_scale) {
   // the kernel reads g before it waits for its predecessor: only launched early when g cannot be that
   // predecessor's output
+  if (defer_scale) {
+    if (!out_f16 || !gains_are_constant) return HYP_EINVAL;
+    HYP_CUDA_TRY(launch_pdl<2>(rmsnorm_kernel<256, true, true>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index,
+                               defer_scale));
+    return 1;
+  }
+  float* none = nullptr;
   if (gains_are_constant) {
     if (out_f16)
-      HYP_CUDA_TRY(launch_pdl<2>(rmsnorm_kernel<256, true>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
+      HYP_CUDA_TRY(launch_pdl<2>(rmsnorm_kernel<256, true>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index, none));
     else
-      HYP_CUDA_TRY(launch_pdl<2>(rmsnorm_kernel<256, false>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
+      HYP_CUDA_TRY(launch_pdl<2>(rmsnorm_kernel<256, false>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index, none));
   } else {
     if (out_f16)
-      HYP_CUDA_TRY(launch_pdl<4>(rmsnorm_kernel<256, true>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
+      HYP_CUDA_TRY(launch_pdl<4>(rmsnorm_kernel<256, true>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index, none));
     else
-      HYP_CUDA_TRY(launch_pdl<4>(rmsnorm_kernel<256, false>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index));
+      HYP_CUDA_TRY(launch_pdl<4>(rmsnorm_kernel<256, false>, dim3(M), dim3(256), 0, st, x, g, h, H, eps, row_index, none));
   }
   return 1;
 }
@@ -125,9 +141,20 @@ int launch_rmsnorm(const float* x, const __nv_bfloat16* g, void* h, bool out_f16
 // Input row layout (fp32, straight from the projection's accumulators): [Q heads | K heads | V heads],
 // each head D wide.  Outputs are fp16 (rounded once): q to its own [M, Hq*D] buffer, k and v to the pages.
 // One thread handles 8 rotation pairs (i .. i+7, i+D/2 .. i+D/2+7) of one head of one row.
+// SPLIT (the model's first block): every element of the row is first multiplied by row_scale[t] (the RMSNorm
+// factor that this block applies after the projection instead of before it), and the rotated queries and keys are
+// stored as two fp16 terms, value = hi + lo with lo the rounding residue of hi: the high terms where the plain
+// kernel stores them, the low terms in q_lo (layout of q16) and in klo_layer ([page][Hkv][16][D], the cache's row
+// order).
+__device__ __forceinline__ uint32_t pack_f16_residue(float a, float b, uint32_t hi) {
+  const __half2 h = *reinterpret_cast<const __half2*>(&hi);
+  return pack_f16(a - __low2float(h), b - __high2float(h));
+}
+template <bool SPLIT>
 __global__ void __launch_bounds__(256, 4)
 rope_kv_write_kernel(const float* __restrict__ qkv, __half* __restrict__ q16, __half* __restrict__ kv_layer,
-                     const float2* __restrict__ rope_table, BatchMeta bm, ModelDims d) {
+                     const float2* __restrict__ rope_table, const float* __restrict__ row_scale,
+                     __half* __restrict__ q_lo, __half* __restrict__ klo_layer, BatchMeta bm, ModelDims d) {
   pdl_trigger();
   pdl_wait();
   constexpr int ITEMS = 2;  // work items of a thread whose loads are issued together
@@ -155,6 +182,7 @@ rope_kv_write_kernel(const float* __restrict__ qkv, __half* __restrict__ q16, __
     const int page = bm.block_table[(size_t)sq * bm.max_pages_per_seq + pos / d.page_tokens];
     const int slot = pos % d.page_tokens;
     const size_t page_base = (size_t)page * kv_page_elems(d.Hkv, d.page_tokens, d.D);
+    const float scale = SPLIT ? row_scale[t] : 1.f;
 #pragma unroll
     for (int it = 0; it < ITEMS; ++it) {
       const int w = w0 + it * blockDim.x;
@@ -163,7 +191,12 @@ rope_kv_write_kernel(const float* __restrict__ qkv, __half* __restrict__ q16, __
       const int i0 = (w % vec_per_head) * 8;
       float x1[8] = {a[it][0].x, a[it][0].y, a[it][0].z, a[it][0].w, a[it][1].x, a[it][1].y, a[it][1].z, a[it][1].w};
       float x2[8] = {b[it][0].x, b[it][0].y, b[it][0].z, b[it][0].w, b[it][1].x, b[it][1].y, b[it][1].z, b[it][1].w};
+      if (SPLIT) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { x1[j] *= scale; x2[j] *= scale; }
+      }
       __half* dst;
+      __half* dst_lo = nullptr;
       if (head < d.Hq + d.Hkv) {
         const float4* cs = reinterpret_cast<const float4*>(rope_table + (size_t)pos * (d.D / 2) + i0);  // (cos, sin) pairs
 #pragma unroll
@@ -177,28 +210,48 @@ rope_kv_write_kernel(const float* __restrict__ qkv, __half* __restrict__ q16, __
         }
         dst = head < d.Hq ? q16 + (size_t)t * d.Hq * d.D + (size_t)head * d.D
                           : kv_layer + page_base + ((size_t)(head - d.Hq) * d.page_tokens + slot) * d.D;
+        if (SPLIT)
+          dst_lo = head < d.Hq ? q_lo + (size_t)t * d.Hq * d.D + (size_t)head * d.D
+                               : klo_layer + (((size_t)page * d.Hkv + (head - d.Hq)) * d.page_tokens + slot) * d.D;
       } else {
         dst = kv_layer + page_base + (size_t)d.Hkv * d.page_tokens * d.D +
               ((size_t)(head - d.Hq - d.Hkv) * d.page_tokens + slot) * d.D;
       }
       // cache rows keep their 16-byte chunks XOR-permuted by the token's slot (see kv_chunk_pos); q rows are plain
       const int sw = head < d.Hq ? 0 : (slot & 7);
-      *reinterpret_cast<uint4*>(dst + (((i0 >> 3) ^ sw) << 3)) = make_uint4(
-          pack_f16_sat(x1[0], x1[1]), pack_f16_sat(x1[2], x1[3]), pack_f16_sat(x1[4], x1[5]), pack_f16_sat(x1[6], x1[7]));
-      *reinterpret_cast<uint4*>(dst + ((((d.D / 2 + i0) >> 3) ^ sw) << 3)) = make_uint4(
-          pack_f16_sat(x2[0], x2[1]), pack_f16_sat(x2[2], x2[3]), pack_f16_sat(x2[4], x2[5]), pack_f16_sat(x2[6], x2[7]));
+      const uint4 h1 = make_uint4(pack_f16_sat(x1[0], x1[1]), pack_f16_sat(x1[2], x1[3]), pack_f16_sat(x1[4], x1[5]),
+                                  pack_f16_sat(x1[6], x1[7]));
+      const uint4 h2 = make_uint4(pack_f16_sat(x2[0], x2[1]), pack_f16_sat(x2[2], x2[3]), pack_f16_sat(x2[4], x2[5]),
+                                  pack_f16_sat(x2[6], x2[7]));
+      *reinterpret_cast<uint4*>(dst + (((i0 >> 3) ^ sw) << 3)) = h1;
+      *reinterpret_cast<uint4*>(dst + ((((d.D / 2 + i0) >> 3) ^ sw) << 3)) = h2;
+      if (SPLIT && dst_lo) {
+        *reinterpret_cast<uint4*>(dst_lo + (((i0 >> 3) ^ sw) << 3)) =
+            make_uint4(pack_f16_residue(x1[0], x1[1], h1.x), pack_f16_residue(x1[2], x1[3], h1.y),
+                       pack_f16_residue(x1[4], x1[5], h1.z), pack_f16_residue(x1[6], x1[7], h1.w));
+        *reinterpret_cast<uint4*>(dst_lo + ((((d.D / 2 + i0) >> 3) ^ sw) << 3)) =
+            make_uint4(pack_f16_residue(x2[0], x2[1], h2.x), pack_f16_residue(x2[2], x2[3], h2.y),
+                       pack_f16_residue(x2[4], x2[5], h2.z), pack_f16_residue(x2[6], x2[7], h2.w));
+      }
     }
   }
 }
 
 int launch_rope_kv_write(const float* qkv, __half* q16, __half* kv_layer, const float2* rope_table,
-                         const BatchMeta& bm, const ModelDims& d, cudaStream_t st) {
+                         const BatchMeta& bm, const ModelDims& d, cudaStream_t st, const float* row_scale,
+                         __half* q_lo, __half* klo_layer) {
   const int work = (d.Hq + 2 * d.Hkv) * (d.D / 16);
   int threads = ((work / 2 + 31) / 32) * 32;  // two work items per thread
   if (threads > 256) threads = 256;
   if (threads < 32) threads = 32;
-  HYP_CUDA_TRY(launch_pdl<2>(rope_kv_write_kernel, dim3(bm.n_tokens), dim3(threads), 0, st, qkv, q16, kv_layer, rope_table,
-                          bm, d));
+  if (row_scale) {
+    if (!q_lo || !klo_layer) return HYP_EINVAL;
+    HYP_CUDA_TRY(launch_pdl<2>(rope_kv_write_kernel<true>, dim3(bm.n_tokens), dim3(threads), 0, st, qkv, q16, kv_layer,
+                               rope_table, row_scale, q_lo, klo_layer, bm, d));
+  } else {
+    HYP_CUDA_TRY(launch_pdl<2>(rope_kv_write_kernel<false>, dim3(bm.n_tokens), dim3(threads), 0, st, qkv, q16, kv_layer,
+                               rope_table, row_scale, q_lo, klo_layer, bm, d));
+  }
   return 1;
 }
 

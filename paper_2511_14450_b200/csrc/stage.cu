@@ -55,6 +55,16 @@ struct hyp_stage {
   float* x = nullptr;
   float* qkv32 = nullptr;             // q | k | v straight from the projection's accumulators
   __half* q16 = nullptr;              // rotated queries
+  // The model's first block (stages with layer_lo == 0) runs its attention scores at higher precision: the
+  // projection's input is the embedding row times the gain times a power of two (exact in fp16 for unit gains),
+  // the rest of the RMSNorm factor (row_scale) is applied to q, k, v afterwards, and q, k are kept as two fp16
+  // terms (q16_lo; klo_pool [page][Hkv][16][D]).  Reason: the residual stream entering block 0 is tiny, so the
+  // block's FFN sees its attention output almost alone and amplifies that branch's rounding errors ~10x more than
+  // any later block does; measured on the 40-block Phi-3-medium shape, block 0's fp16 score errors alone made up
+  // two thirds of the final logit error.
+  float* row_scale = nullptr;
+  __half* q16_lo = nullptr;
+  __half* klo_pool = nullptr;
   __half *h = nullptr, *attn = nullptr, *u = nullptr;  // projection inputs (fp16)
   TcAct tc_h, tc_attn, tc_u, tc_q16;
   int* err_host = nullptr;  // pinned: the device error word, copied behind a host-buffer call's last kernel
@@ -306,13 +316,21 @@ int run_blocks(hyp_stage* s, const BatchMeta& bm, bool decode, int n_splits, cud
     __half* kv_layer = s->kv_pool + (size_t)li * s->kv_layer_elems;
     // every projection runs fp16 x fp16 -> fp32: with bf16 inputs the rounding of the activations alone
     // (8 mantissa bits, amplified from block to block) puts the 40-block logits outside the tolerance
-    HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g1, s->h, true, M, d.H, d.eps, nullptr, st, true));
+    const bool split = li == 0 && s->klo_pool != nullptr && first_block_split();
+    HYP_LAUNCH_T(HYP_K_NORM, launch_rmsnorm(s->x, lw.g1, s->h, true, M, d.H, d.eps, nullptr, st, true,
+                                            split ? s->row_scale : nullptr));
     HYP_LAUNCH_T(HYP_K_GEMM_QKV, project(s, s->tc_h, nullptr, d.H, lw.tc_qkv, nullptr, d.qkv_rows, d.H, M,
                                          EPI_STORE_F32, s->qkv32, d.qkv_rows, st));
     if (decode) {
       // rotation, cache append, attention and the merge of its splits in one launch
       HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_decode_fused(s->qkv32, d.qkv_rows, kv_layer, s->rope_table, s->attn, n_splits,
-                                                        2, tc_err_flag_ptr(), bm, d, st));
+                                                        2, tc_err_flag_ptr(), bm, d, st, split ? s->row_scale : nullptr,
+                                                        split ? s->klo_pool : nullptr));
+    } else if (split) {
+      HYP_LAUNCH_T(HYP_K_ROPE, launch_rope_kv_write(s->qkv32, s->q16, kv_layer, s->rope_table, bm, d, st, s->row_scale,
+                                                    s->q16_lo, s->klo_pool));
+      HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_prefill_split(s->q16, s->q16_lo, d.Hq * d.D, kv_layer, s->klo_pool, s->attn, bm,
+                                                         d, st));
     } else {
       HYP_LAUNCH_T(HYP_K_ROPE, launch_rope_kv_write(s->qkv32, s->q16, kv_layer, s->rope_table, bm, d, st));
       if (attn_prefill_tc_enabled() && !s->kv_maps.empty())
@@ -521,6 +539,7 @@ extern "C" void hyp_stage_destroy(hyp_stage* s) {
   }
   cudaFree(s->embed); cudaFree(s->gf); cudaFree(s->wlm); cudaFree(s->kv_pool);
   cudaFree(s->x); cudaFree(s->h); cudaFree(s->qkv32); cudaFree(s->q16);
+  cudaFree(s->row_scale); cudaFree(s->q16_lo); cudaFree(s->klo_pool);
   cudaFree(s->attn); cudaFree(s->u);
   cudaFree(s->rope_table); cudaFree(s->meta_dev);
   cudaFree(s->io_in); cudaFree(s->io_out);
@@ -599,6 +618,13 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
   TRY(dev_alloc(&s->h, rows_pad * d.H));
   TRY(dev_alloc(&s->qkv32, rows_pad * d.qkv_rows));
   TRY(dev_alloc(&s->q16, rows_pad * d.Hq * d.D));
+  if (s->first) {
+    const size_t klo_elems = (size_t)s->n_pages * d.Hkv * d.page_tokens * d.D;
+    TRY(dev_alloc(&s->row_scale, rows_pad));
+    TRY(dev_alloc(&s->q16_lo, rows_pad * d.Hq * d.D));
+    TRY(dev_alloc(&s->klo_pool, klo_elems));
+    TRY_CUDA(cudaMemset(s->klo_pool, 0, klo_elems * sizeof(__half)));
+  }
   TRY(dev_alloc(&s->attn, rows_pad * d.Hq * d.D));
   TRY(dev_alloc(&s->u, rows_pad * d.F));
   TRY_CUDA(cudaMemset(s->h, 0, rows_pad * d.H * sizeof(__half)));
@@ -828,6 +854,7 @@ extern "C" int hyp_stage_profile(hyp_stage* s, int32_t mode, int32_t batch, int3
       const ModelDims& d = s->dims;
       const size_t wbytes = ((size_t)d.qkv_rows * d.H + (size_t)d.H * d.Hq * d.D + (size_t)3 * d.F * d.H + 2 * d.H) * 2;
       layer_bytes[li] = wbytes + s->kv_layer_elems * sizeof(__half) + s->workspace_bytes / s->L;
+      if (li == 0 && s->klo_pool) layer_bytes[li] += s->kv_layer_elems / 2 * sizeof(__half);  // the keys' low terms
     }
   }
   for (auto& e : ev) cudaEventDestroy(e);

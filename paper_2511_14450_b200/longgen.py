@@ -20,15 +20,11 @@ from paper_2511_14450_b200 import hyperion as hyp  # noqa: E402
 from paper_2511_14450_b200 import inputs  # noqa: E402
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--steps", type=int, default=2048)
-    ap.add_argument("--prompt", type=int, default=2048)
-    ap.add_argument("--batch", type=int, default=4)
-    ap.add_argument("--layers", type=int, default=40)
-    a = ap.parse_args()
-    sh = inputs.phi3_medium_shape(a.layers)
-    B, P, S, L = a.batch, a.prompt, a.steps, a.layers
+def run(steps: int = 2048, prompt: int = 2048, batch: int = 4, layers: int = 40) -> dict:
+    """Prefill of batch x prompt rows in one call, then `steps` teacher-forced decode steps; returns the figures
+    main() prints (times from CUDA events on the current stream)."""
+    sh = inputs.phi3_medium_shape(layers)
+    B, P, S, L = batch, prompt, steps, layers
     st = hyp.Stage(sh, 0, L, max_seqs=B, max_ctx=P + S + 16, max_tokens=B * P)
     for layer in range(L):
         st.load_layer(layer, inputs.layer_weights(sh, layer, device="cuda"))
@@ -78,14 +74,24 @@ def main():
     hbm = float(peaks.get("hbm_gbs", 6650.0))
     tf = float(peaks.get("bf16_tflops_sustained", 1400.0))
     gbs = (w_bytes + kv_bytes) / 1e9 / (decode_ms / 1e3)
-    print(json.dumps({
+    return {
         "workload": f"configs[4]: {L} Phi-3-medium-shaped blocks + LM head, batch {B}, prompt {P}, {S} decode steps",
         "prefill_ms": prefill_ms, "prefill_tokens_per_s": B * P / (prefill_ms / 1e3),
         "prefill_tflops": (lin_flops + attn_flops) / prefill_ms / 1e9,
         "prefill_frac_of_measured_sustained": (lin_flops + attn_flops) / prefill_ms / 1e9 / tf,
         "decode_steps_timed": n, "decode_ms_per_step": decode_ms, "decode_tokens_per_s": B / (decode_ms / 1e3),
         "decode_bytes_per_step": w_bytes + kv_bytes, "decode_gbs": gbs, "decode_frac_of_measured_hbm": gbs / hbm,
-        "decode_frac_of_nominal_8TBs": gbs / 8000.0, "mean_ctx": ctx_sum / n}))
+        "decode_frac_of_nominal_8TBs": gbs / 8000.0, "mean_ctx": ctx_sum / n}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--steps", type=int, default=2048)
+    ap.add_argument("--prompt", type=int, default=2048)
+    ap.add_argument("--batch", type=int, default=4)
+    ap.add_argument("--layers", type=int, default=40)
+    a = ap.parse_args()
+    print(json.dumps(run(a.steps, a.prompt, a.batch, a.layers)))
 
 
 if __name__ == "__main__":

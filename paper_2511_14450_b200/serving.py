@@ -282,17 +282,29 @@ def main():
         print(json.dumps({"shape": a.shape, "blocks": shape.n_layers_total, "block_ms_min_max": [min(ms), max(ms)],
                           "splits": [compare_splits(ms, nbytes, t) for t in (2, 3, 4)]}))
         return
-    shape = inputs.phi3_medium_shape(a.layers)
-    bounds, tau, ms, nbytes = plan_stages(shape, a.tiers)
-    eng = PipelineEngine(shape, bounds, max_seqs=a.requests, max_ctx=a.len_hi + a.n_out + 16, max_tokens=2048)
-    reqs = synthetic_requests(shape, a.requests, a.rate, a.len_lo, a.len_hi, a.n_out)
-    stats = eng.run(reqs, realtime=(a.mode == "replay"))
+    print(json.dumps(run_workload(a.mode == "replay", a.requests, a.rate, a.len_lo, a.len_hi, a.n_out, a.tiers, a.layers)))
+
+
+def run_workload(realtime: bool, requests: int = 32, rate: float = 4.0, len_lo: int = 128, len_hi: int = 1024,
+                 n_out: int = 256, tiers: int = 3, layers: int = 40) -> dict:
+    """The serving configuration end to end: profile the blocks, split them with HypSplit-DP, build one stage per
+    tier and serve the seeded request set (in real time, or closed-loop with everything admitted at once)."""
+    shape = inputs.phi3_medium_shape(layers)
+    bounds, tau, ms, nbytes = plan_stages(shape, tiers)
+    eng = PipelineEngine(shape, bounds, max_seqs=requests, max_ctx=len_hi + n_out + 16, max_tokens=2048)
+    reqs = synthetic_requests(shape, requests, rate, len_lo, len_hi, n_out)
+    stats = eng.run(reqs, realtime=realtime)
     eng.close()
-    stats.update({"mode": a.mode, "stage_boundaries": bounds, "split_bottleneck_ms": tau,
-                  "block_ms_min_max": [min(ms), max(ms)], "offered_tokens_per_s": a.rate * a.n_out,
-                  "workload": f"configs[3]: {a.layers} Phi-3-medium-shaped blocks as {a.tiers} stages, {a.requests} requests, "
-                              f"Poisson {a.rate}/s, prompts U[{a.len_lo},{a.len_hi}], {a.n_out} forced output tokens"})
-    print(json.dumps(stats))
+    stats.update({"mode": "replay" if realtime else "closed", "stage_boundaries": bounds, "split_bottleneck_ms": tau,
+                  "block_ms_min_max": [min(ms), max(ms)], "offered_tokens_per_s": rate * n_out,
+                  "workload": f"configs[3]: {layers} Phi-3-medium-shaped blocks as {tiers} stages, {requests} requests, "
+                              f"Poisson {rate}/s, prompts U[{len_lo},{len_hi}], {n_out} forced output tokens"})
+    return stats
+
+
+def run_closed_loop() -> dict:
+    """configs[3] with all 32 requests admitted at t = 0: output tokens per second of the three-stage engine."""
+    return run_workload(False)
 
 
 if __name__ == "__main__":
