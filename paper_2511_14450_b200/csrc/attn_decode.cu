@@ -26,7 +26,7 @@ size_t attn_decode_scratch_bytes(int max_seqs, int Hq, int D, int max_splits) {
 }
 
 int attn_decode_splits(int n_seqs, int Hkv, int max_ctx) {
-  int want = (3 * 148 + n_seqs * Hkv - 1) / (n_seqs * Hkv);
+  int want = (3 * sm_count() + n_seqs * Hkv - 1) / (n_seqs * Hkv);
   int cap = (max_ctx + 2 * AD_TILE - 1) / (2 * AD_TILE);  // at least two tiles per split
   if (want > cap) want = cap;
   if (want > 32) want = 32;

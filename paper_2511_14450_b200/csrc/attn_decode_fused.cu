@@ -3,7 +3,7 @@
 // split-context attention, and the merge of the splits.
 //
 //   grid (n_splits, Hkv, n_seqs), 4 warps, the n_splits CTAs of one (sequence, KV head) form a thread-block
-//   cluster.  A CTA owns a run of the sequence's pages; warp w takes pages w, w + 4, ... of that run and streams
+//   cluster.  Page p of a sequence belongs to split p % n_splits; warp w takes every fourth page of its split and streams
 //   them through its own ring: one bulk copy brings the 16 keys of a page for this KV head (contiguous in the
 //   cache, already chunk-permuted for ldmatrix), another the 16 values; the warp waits on the slot's mbarrier,
 //   forms the scores of its 16 keys for the G = Hq/Hkv query heads (rows of one mma.sync.m16n8k16 operand, rows
@@ -68,26 +68,28 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, tq = lane & 3;
 
-  // metadata and cache pages written by earlier steps do not depend on the predecessor kernel
+  // Which pages are mine does not depend on the sequence's length: page p belongs to split p % n_splits, and inside
+  // the CTA the pages of a split go round-robin over the warps, so this warp's i-th page is
+  // split + n_splits * (warp + AF_WARPS * i).  The block-table entries (one per lane, two rounds) are therefore
+  // fetched together with the length instead of behind it; only "how many of them exist" waits for the length.
+  // Metadata and cache pages written by earlier steps do not depend on the predecessor kernel.
+  const int32_t* bt = bm.block_table + (size_t)b * bm.max_pages_per_seq;
+  auto page_index = [&](int i) { return split + n_splits * (warp + AF_WARPS * i); };
+  const int pi_lo = page_index(lane), pi_hi = page_index(lane + 32);
+  const int32_t bt_lo = pi_lo < bm.max_pages_per_seq ? bt[pi_lo] : 0;
+  const int32_t bt_hi = pi_hi < bm.max_pages_per_seq ? bt[pi_hi] : 0;
   const int pos = bm.ctx_lens[b];  // the new token's position
   const int ctx_total = pos + 1;
   const int n_pages = (ctx_total + AF_PT - 1) / AF_PT;
-  const int pps = (n_pages + n_splits - 1) / n_splits;
-  const int p_begin = split * pps;
-  const int p_end = min(n_pages, p_begin + pps);
-  const int32_t* bt = bm.block_table + (size_t)b * bm.max_pages_per_seq;
   const size_t page_elems = kv_page_elems(d.Hkv, AF_PT, D);
   const size_t v_off = (size_t)d.Hkv * AF_PT * D;
   const uint32_t my_bars = smem_u32(bars) + 8u * (warp * AF_MAX_SLOTS);
   const uint32_t my_ring = ring0 + (uint32_t)(warp * S) * SLOT_BYTES;
-  const int my_n = p_begin + warp < p_end ? (p_end - p_begin - warp + AF_WARPS - 1) / AF_WARPS : 0;
-  // the block-table entries of this warp's pages, one per lane (two rounds): a refill then needs no dependent
-  // global load in front of its copy
-  const int32_t bt_lo = lane < my_n ? bt[p_begin + warp + AF_WARPS * lane] : 0;
-  const int32_t bt_hi = lane + 32 < my_n ? bt[p_begin + warp + AF_WARPS * (lane + 32)] : 0;
+  const int first = page_index(0), stride_p = n_splits * AF_WARPS;
+  const int my_n = first < n_pages ? (n_pages - first + stride_p - 1) / stride_p : 0;
   auto page_of = [&](int i) {  // all lanes call; page id of this warp's i-th page
     const int32_t lo = __shfl_sync(0xffffffffu, bt_lo, i & 31), hi = __shfl_sync(0xffffffffu, bt_hi, i & 31);
-    return i < 32 ? lo : i < 64 ? hi : bt[p_begin + warp + AF_WARPS * i];
+    return i < 32 ? lo : i < 64 ? hi : bt[page_index(i)];
   };
   auto issue = [&](int page, int slot) {  // lane 0: copy one page's keys and values of this head into a slot
     const __half* src = a.kv_layer + (size_t)page * page_elems + (size_t)kvh * AF_PT * D;
@@ -110,7 +112,7 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
 
   // rotate: this CTA's G query heads; and, in the CTA whose run holds the new token's page, its key (+ value)
   const int page_new = pos / AF_PT, slot_new = pos % AF_PT;
-  const bool owner_cta = page_new >= p_begin && page_new < p_end;
+  const bool owner_cta = page_new % n_splits == split;
   {
     const float* row = a.qkv32 + (size_t)b * a.stride;
     const float2* cs = a.rope_table + (size_t)pos * (D / 2);
@@ -187,7 +189,7 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
   int slot = 0;
   uint32_t phase = 0;
   for (int i = 0; i < my_n; ++i) {
-    const int pi = p_begin + warp + AF_WARPS * i;
+    const int pi = page_index(i);
     if (!mbar_wait(my_bars + 8u * slot, phase, nullptr)) { ok = false; break; }
     const uint32_t kt = my_ring + slot * SLOT_BYTES, vt = kt + PAGE_BYTES;
     const bool patched = pi == page_new;
@@ -392,7 +394,7 @@ int& attn_fused_slots_override() {
 int attn_decode_fused_splits(int n_seqs, int Hkv, int max_ctx) {
   if (attn_fused_splits_override() > 0) return attn_fused_splits_override();
   // one resident wave: about three CTAs per SM; at least 8 pages (two per warp) per split; clusters of up to 8
-  int want = (3 * 148) / (n_seqs * Hkv);
+  int want = (3 * sm_count()) / (n_seqs * Hkv);
   const int pages = (max_ctx + AF_PT - 1) / AF_PT;
   const int cap = (pages + 7) / 8;
   if (want > cap) want = cap;

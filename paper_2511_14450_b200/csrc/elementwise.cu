@@ -37,7 +37,7 @@ __global__ void copy_f32_kernel(const float4* __restrict__ src, float4* __restri
 int launch_copy_f32(const float* src, float* dst, size_t n, cudaStream_t st) {
   const size_t n4 = n / 4;  // H is a multiple of 8, so n is a multiple of 4
   int blocks = (int)((n4 + 255) / 256);
-  if (blocks > 148 * 8) blocks = 148 * 8;
+  if (blocks > sm_count() * 8) blocks = sm_count() * 8;
   if (blocks < 1) blocks = 1;
   HYP_CUDA_TRY(launch_pdl(copy_f32_kernel, dim3(blocks), dim3(256), 0, st, reinterpret_cast<const float4*>(src),
                           reinterpret_cast<float4*>(dst), n4));

@@ -30,7 +30,7 @@ namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment*/ + 1024 /*barriers*/ + 4 * 2 * 32 * 128 /*epilogue boxes*/;
 constexpr int TC_THREADS = 192;
 
 // Instruction descriptor: (bf16 x bf16 | fp16 x fp16) -> fp32, both operands K-major, M = 128, N = 256.
@@ -87,72 +87,106 @@ struct Segments {
   }
 };
 
-__device__ __forceinline__ void red_add_f32x4(float* p, float a, float b, float c, float d) {
-  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+// ---------------------------------------------------------------------------------------------------------
+// Epilogue through shared memory and TMA.  An accumulator row lives in one thread (tcgen05.ld, lane = row), so
+// direct global stores touch 32 rows per warp instruction, 16 bytes each.  Instead every epilogue warp turns its
+// 32 rows x 128 bytes of results through a 4 KB staging box (128-byte swizzle: chunk c of row r at c ^ (r & 7),
+// conflict-free for 16-byte stores by rows) and one lane hands the box to the copy engine: a tensor store, or - for
+// the residual epilogue, whole tiles and split-K partial tiles alike - a tensor reduction that adds the box to
+// the residual stream in L2.  The tensor map clips rows >= M and columns >= N, so ragged tiles need no predicates.
+// Two boxes per warp: the next one is filled while the copy engine reads the previous one.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int EPI_BOX_BYTES = 32 * 128;                 // 32 rows x 128 bytes
+constexpr int EPI_STAGING_BYTES = 4 * 2 * EPI_BOX_BYTES;  // 4 epilogue warps x 2 boxes
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
-template <int EPI>
-__device__ __forceinline__ void epilogue_chunk(const uint32_t (&v)[16], const uint32_t (&v2)[16], void* out, int ldo,
-                                               int row, int col, int N, bool partial, bool f16) {
-  const size_t o = (size_t)row * ldo + col;
-  const bool full = col + 16 <= N;
-  if (EPI == EPI_STORE_BF16 || EPI == EPI_SWIGLU_BF16) {
-    float f[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const float a = __uint_as_float(v[i]);
-      f[i] = (EPI == EPI_SWIGLU_BF16) ? a / (1.f + __expf(-a)) * __uint_as_float(v2[i]) : a;
+// One warp's share (32 rows) of one accumulator tile.  t0: tensor-memory address of the warp's lane quarter at
+// the accumulator's first column; up_cols: column distance from a gate column to its up column (SwiGLU);
+// boxes: shared address of the warp's two staging boxes; n_box: running count of boxes this warp has issued.
+template <int EPI, int BN_ACC>
+__device__ __forceinline__ void epilogue_warp(uint32_t t0, const CUtensorMap* tm_out, uint32_t boxes, int lane, int row0,
+                                              int n0, int N, bool f16, uint32_t& n_box) {
+  constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
+  constexpr bool OUT16 = EPI == EPI_STORE_BF16 || EPI == EPI_SWIGLU_BF16;
+  constexpr int BN_OUT = SWIGLU ? BN_ACC / 2 : BN_ACC;
+  constexpr int BOX_COLS = OUT16 ? 64 : 32;  // 128 bytes of output per row
+  const uint32_t sw = (uint32_t)(lane & 7);
+#pragma unroll 1
+  for (int c = 0; c < BN_OUT; c += BOX_COLS) {
+    if (n0 + c >= N) break;  // uniform across the warp
+    const uint32_t box = boxes + (n_box & 1u) * EPI_BOX_BYTES;
+    const uint32_t rowp = box + (uint32_t)lane * 128u;
+    // the copy that last read this box (two boxes ago) must have finished reading it
+    if (n_box >= 2) {
+      if (lane == 0) bulk_wait_read<1>();
+      __syncwarp();
     }
-    // 16-bit results take the operands' type (bf16 or fp16, both 2 bytes)
-    uint16_t* p = reinterpret_cast<uint16_t*>(out) + o;
-    uint32_t pk[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) pk[i] = f16 ? pack_f16_sat(f[2 * i], f[2 * i + 1]) : pack_bf16(f[2 * i], f[2 * i + 1]);
-    if (full) {
-      reinterpret_cast<uint4*>(p)[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-      reinterpret_cast<uint4*>(p)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-    } else {
+    for (int hh = 0; hh < (OUT16 ? 2 : 1); ++hh) {  // 32 accumulator columns at a time
+      uint32_t v[32], u[SWIGLU ? 32 : 1];
+      tmem_ld16(t0 + c + 32 * hh, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+      tmem_ld16(t0 + c + 32 * hh + 16, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
+      if (SWIGLU) {
+        tmem_ld16(t0 + BN_ACC / 2 + c + 32 * hh, *reinterpret_cast<uint32_t(*)[16]>(&u[0]));
+        tmem_ld16(t0 + BN_ACC / 2 + c + 32 * hh + 16, *reinterpret_cast<uint32_t(*)[16]>(&u[SWIGLU ? 16 : 0]));
+      }
+      tmem_ld_wait();
+      if (OUT16) {
+        uint32_t pk[16];
 #pragma unroll
-      for (int i = 0; i < 16; ++i)
-        if (col + i < N) p[i] = (uint16_t)((i & 1) ? (pk[i >> 1] >> 16) : (pk[i >> 1] & 0xffffu));
-    }
-  } else {
-    float* p = reinterpret_cast<float*>(out) + o;
-    if (EPI == EPI_RESID_F32 && partial) {
-      // this CTA holds only part of the tile's k range: add, never overwrite
-      if (full) {
+        for (int i = 0; i < 16; ++i) {
+          float y0 = __uint_as_float(v[2 * i]), y1 = __uint_as_float(v[2 * i + 1]);
+          if (SWIGLU) {
+            y0 = y0 / (1.f + __expf(-y0)) * __uint_as_float(u[SWIGLU ? 2 * i : 0]);
+            y1 = y1 / (1.f + __expf(-y1)) * __uint_as_float(u[SWIGLU ? 2 * i + 1 : 0]);
+          }
+          pk[i] = f16 ? pack_f16_sat(y0, y1) : pack_bf16(y0, y1);  // 16-bit results take the operands' type
+        }
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-          red_add_f32x4(p + 4 * i, __uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                        __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+        for (int j = 0; j < 4; ++j)
+          st_shared_v4(rowp + ((((uint32_t)(4 * hh + j)) ^ sw) << 4), pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
       } else {
 #pragma unroll
-        for (int i = 0; i < 16; ++i)
-          if (col + i < N) atomicAdd(p + i, __uint_as_float(v[i]));
+        for (int j = 0; j < 8; ++j)
+          st_shared_v4(rowp + (((uint32_t)j ^ sw) << 4), v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
       }
-    } else if (full) {
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        float4 a = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
-                               __uint_as_float(v[4 * i + 3]));
-        if (EPI == EPI_RESID_F32) {
-          const float4 b = reinterpret_cast<const float4*>(p)[i];
-          a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
-        }
-        reinterpret_cast<float4*>(p)[i] = a;
-      }
-    } else {
-#pragma unroll
-      for (int i = 0; i < 16; ++i)
-        if (col + i < N) p[i] = (EPI == EPI_RESID_F32 ? p[i] : 0.f) + __uint_as_float(v[i]);
     }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the copy engine must see these stores
+    __syncwarp();
+    if (lane == 0) {
+      if (EPI == EPI_RESID_F32)
+        tma_reduce_add_2d(tm_out, box, n0 + c, row0);
+      else
+        tma_store_2d(tm_out, box, n0 + c, row0);
+      bulk_commit();
+    }
+    ++n_box;
   }
 }
 
 template <int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int M, int N, int K,
-               int up_tile0, void* __restrict__ out, int ldo, int team, uint32_t idesc, int* __restrict__ err) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+               const __grid_constant__ CUtensorMap tm_out, int M, int N, int K, int up_tile0, int team, uint32_t idesc,
+               int* __restrict__ err) {
   constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
   const bool STREAMK = EPI == EPI_RESID_F32 && team > 0;
   constexpr int BN_OUT = SWIGLU ? BN / 2 : BN;  // output columns per tile
@@ -168,12 +202,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t staging = base + STAGES * STAGE_BYTES + 1024;  // 1024-aligned: the boxes are 128-byte swizzled
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN_OUT - 1) / BN_OUT;
   const int KB = (K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
+    prefetch_tensormap(&tm_a);
+    prefetch_tensormap(&tm_b);
+    prefetch_tensormap(&tm_out);
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
@@ -263,32 +301,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
     pdl_wait();              // the output buffer may still be in use by the predecessor
     int acc = 0;
-    uint32_t acc_phase = 0;
+    uint32_t acc_phase = 0, n_box = 0;
     bool ok = true;
+    const uint32_t boxes = staging + (uint32_t)q * (2 * EPI_BOX_BYTES);
     Segments seg(STREAMK, tiles_m, tiles_n, KB, team, (int)blockIdx.x, (int)gridDim.x);
     int tile, kb0, kb1;
     while (ok && seg.next(tile, kb0, kb1)) {
       const int m0 = (tile % tiles_m) * BM;
       const int n0 = (tile / tiles_m) * BN_OUT;
-      const bool partial = kb0 != 0 || kb1 != KB;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const int row = m0 + 32 * q + lane;
       const uint32_t t0 = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * BN);
-#pragma unroll 2
-      for (int c = 0; c < BN_OUT; c += 16) {
-        if (n0 + c >= N) break;  // uniform across the warp
-        uint32_t v[16], v2[16];
-        tmem_ld16(t0 + c, v);
-        if (SWIGLU) tmem_ld16(t0 + BN / 2 + c, v2);
-        tmem_ld_wait();
-        if (row < M) epilogue_chunk<EPI>(v, v2, out, ldo, row, n0 + c, N, partial, idesc == IDESC_F16);
-      }
+      epilogue_warp<EPI, BN>(t0, &tm_out, boxes, lane, m0 + 32 * q, n0, N, idesc == IDESC_F16, n_box);
       tc_fence_before();
       mbar_arrive(tempty_bar(acc));
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1;
     }
+    if (lane == 0) bulk_wait_all();  // the boxes must outlive the copies that read them; results complete before exit
     if (!ok && lane == 0) {
       *abort_flag = 1;
       atomicCAS(err, 0, 3);
@@ -316,7 +346,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 // ---------------------------------------------------------------------------------------------------------
 constexpr int STAGES2 = 6;
 constexpr int STAGE2_BYTES = A_BYTES + B_BYTES / 2;  // per CTA: 16 KB of A + 16 KB of its half of B
-constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 + 256;
+constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 /*alignment*/ + 1024 /*barriers*/ + EPI_STAGING_BYTES;
 constexpr uint32_t IDESC2_BF16 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 constexpr uint32_t IDESC2_F16 = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 
@@ -367,8 +397,9 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uin
 
 template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
-gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, int M, int N, int K,
-                int up_tile0, void* __restrict__ out, int ldo, int team, uint32_t idesc, int* __restrict__ err) {
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                const __grid_constant__ CUtensorMap tm_out, int M, int N, int K, int up_tile0, int team, uint32_t idesc,
+                int* __restrict__ err) {
   constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
   const bool STREAMK = EPI == EPI_RESID_F32 && team > 0;
   constexpr int BN_OUT = SWIGLU ? BN / 2 : BN;
@@ -384,6 +415,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES2 + 2 + a); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES2 + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t staging = base + STAGES2 * STAGE2_BYTES + 1024;  // 1024-aligned: the boxes are 128-byte swizzled
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();      // 0 = leader
@@ -393,6 +425,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   const int KB = (K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
+    prefetch_tensormap(&tm_a);
+    prefetch_tensormap(&tm_b);
+    prefetch_tensormap(&tm_out);
     for (int s = 0; s < STAGES2; ++s) {
       mbar_init(full_bar(s), 1);    // the leader's arrive.expect_tx; bytes come from both CTAs' copies
       mbar_init(empty_bar(s), 1);   // the leader's MMA commit (multicast)
@@ -483,32 +518,24 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     const int q = warp & 3;
     pdl_wait();
     int acc = 0;
-    uint32_t acc_phase = 0;
+    uint32_t acc_phase = 0, n_box = 0;
     bool ok = true;
+    const uint32_t boxes = staging + (uint32_t)q * (2 * EPI_BOX_BYTES);
     Segments seg(STREAMK, pairs_m, tiles_n, KB, team, pair, n_pairs);
     int tile, kb0, kb1;
     while (ok && seg.next(tile, kb0, kb1)) {
       const int m0 = (tile % pairs_m) * (2 * BM) + (int)rank * BM;
       const int n0 = (tile / pairs_m) * BN_OUT;
-      const bool partial = kb0 != 0 || kb1 != KB;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const int row = m0 + 32 * q + lane;
       const uint32_t t0 = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * BN);
-#pragma unroll 2
-      for (int c = 0; c < BN_OUT; c += 16) {
-        if (n0 + c >= N) break;
-        uint32_t v[16], v2[16];
-        tmem_ld16(t0 + c, v);
-        if (SWIGLU) tmem_ld16(t0 + BN / 2 + c, v2);
-        tmem_ld_wait();
-        if (row < M) epilogue_chunk<EPI>(v, v2, out, ldo, row, n0 + c, N, partial, idesc == IDESC2_F16);
-      }
+      epilogue_warp<EPI, BN>(t0, &tm_out, boxes, lane, m0 + 32 * q, n0, N, idesc == IDESC2_F16, n_box);
       tc_fence_before();
       mbar_arrive_cluster(mapa_rank(tempty_bar(acc), 0));
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1;
     }
+    if (lane == 0) bulk_wait_all();  // the boxes must outlive the copies that read them; results complete before exit
     if (!ok && lane == 0) {
       *abort_flag = 1;
       atomicCAS(err, 0, 8);
@@ -558,6 +585,28 @@ int encode_map(CUtensorMap* map, const void* ptr, int rows, int K, int box_rows,
   return HYP_OK;
 }
 
+// Output matrix [M, N] (row stride ldo elements) as the epilogue's boxes see it: 32 rows x 128 bytes, 128-byte
+// swizzle, extents M and N so that the copy engine clips ragged tiles.
+int encode_out_map(CUtensorMap* map, void* out, int ldo, int M, int N, int epi, bool f16) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return HYP_ECUDA;
+  const bool out16 = epi == EPI_STORE_BF16 || epi == EPI_SWIGLU_BF16;
+  const size_t es = out16 ? 2 : 4;
+  const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)ldo * es};
+  const cuuint32_t box[2] = {(cuuint32_t)(128 / es), 32u};
+  const cuuint32_t estr[2] = {1u, 1u};
+  const CUtensorMapDataType dt = !out16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                 : f16  ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  CUresult r = enc(map, dt, 2, out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error((int)r);
+    return HYP_ECUDA;
+  }
+  return HYP_OK;
+}
+
 int* g_err_flag = nullptr;  // one device word per process: first non-zero code wins
 
 template <int EPI>
@@ -591,12 +640,15 @@ int launch_pair(const TcAct& act, const TcWeight& w, int M, int N, int K, void* 
   } else if (tiles < pairs) {
     pairs = tiles;
   }
+  CUtensorMap tm_out;
+  const int mrc = encode_out_map(&tm_out, out, ldo, M, N, EPI, act.f16);
+  if (mrc) return mrc;
   if (early)
     HYP_CUDA_TRY(launch_pdl<1>(gemm_tc2_kernel<EPI>, dim3((unsigned)(2 * pairs)), dim3(TC_THREADS), (size_t)SMEM2_BYTES, st,
-                               act.map, w.map, M, N, K, w.N16p, out, ldo, team, act.f16 ? IDESC2_F16 : IDESC2_BF16, g_err_flag));
+                               act.map, w.map, tm_out, M, N, K, w.N16p, team, act.f16 ? IDESC2_F16 : IDESC2_BF16, g_err_flag));
   else
     HYP_CUDA_TRY(launch_pdl(gemm_tc2_kernel<EPI>, dim3((unsigned)(2 * pairs)), dim3(TC_THREADS), (size_t)SMEM2_BYTES, st,
-                            act.map, w.map, M, N, K, w.N16p, out, ldo, team, act.f16 ? IDESC2_F16 : IDESC2_BF16, g_err_flag));
+                            act.map, w.map, tm_out, M, N, K, w.N16p, team, act.f16 ? IDESC2_F16 : IDESC2_BF16, g_err_flag));
   return 1;
 }
 
@@ -637,12 +689,15 @@ int launch_epi(const TcAct& act, const TcWeight& w, int M, int N, int K, void* o
     grid = (int)(tiles < num_sms ? tiles : num_sms);
   }
   // launched early (set-up under the predecessor's tail; every load waits for it) where the caller allows
+  CUtensorMap tm_out;
+  const int mrc = encode_out_map(&tm_out, out, ldo, M, N, EPI, act.f16);
+  if (mrc) return mrc;
   if (early)
-    HYP_CUDA_TRY(launch_pdl<1>(gemm_tc_kernel<EPI>, dim3(grid), dim3(TC_THREADS), (size_t)SMEM_BYTES, st, act.map, w.map, M,
-                               N, K, w.N16p, out, ldo, team, act.f16 ? IDESC_F16 : IDESC_BF16, g_err_flag));
+    HYP_CUDA_TRY(launch_pdl<1>(gemm_tc_kernel<EPI>, dim3(grid), dim3(TC_THREADS), (size_t)SMEM_BYTES, st, act.map, w.map,
+                               tm_out, M, N, K, w.N16p, team, act.f16 ? IDESC_F16 : IDESC_BF16, g_err_flag));
   else
-    HYP_CUDA_TRY(launch_pdl(gemm_tc_kernel<EPI>, dim3(grid), dim3(TC_THREADS), (size_t)SMEM_BYTES, st, act.map, w.map, M, N,
-                            K, w.N16p, out, ldo, team, act.f16 ? IDESC_F16 : IDESC_BF16, g_err_flag));
+    HYP_CUDA_TRY(launch_pdl(gemm_tc_kernel<EPI>, dim3(grid), dim3(TC_THREADS), (size_t)SMEM_BYTES, st, act.map, w.map,
+                            tm_out, M, N, K, w.N16p, team, act.f16 ? IDESC_F16 : IDESC_BF16, g_err_flag));
   return 1;
 }
 
@@ -701,7 +756,7 @@ int tc_pack_weight(const void* src, void* dst, int rows, int halves, int K, bool
   if (!src || !dst || rows < 1 || (halves != 1 && halves != 2) || K < 8 || (K % 8) != 0) return HYP_EINVAL;
   if (((uintptr_t)src & 15) != 0 || ((uintptr_t)dst & 15) != 0) return HYP_EINVAL;
   const size_t chunks = tc_packed_bytes(rows, halves, K) / 16;
-  const int blocks = (int)std::min<size_t>((chunks + 255) / 256, (size_t)148 * 16);
+  const int blocks = (int)std::min<size_t>((chunks + 255) / 256, (size_t)sm_count() * 16);
   pack_weight_kernel<<<blocks, 256, 0, st>>>((const uint4*)src, (uint4*)dst, rows, halves, K, pk_n16p(rows), pk_kbp(K), to_f16);
   return 1;
 }

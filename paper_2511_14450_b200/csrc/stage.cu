@@ -322,8 +322,11 @@ int run_blocks(hyp_stage* s, const BatchMeta& bm, bool decode, int n_splits, cud
     HYP_LAUNCH_T(HYP_K_GEMM_QKV, project(s, s->tc_h, nullptr, d.H, lw.tc_qkv, nullptr, d.qkv_rows, d.H, M,
                                          EPI_STORE_F32, s->qkv32, d.qkv_rows, st));
     if (decode) {
-      // rotation, cache append, attention and the merge of its splits in one launch
-      HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_decode_fused(s->qkv32, d.qkv_rows, kv_layer, s->rope_table, s->attn, n_splits,
+      // rotation, cache append, attention and the merge of its splits in one launch; the two-term variant holds
+      // half as much again in shared memory (two CTAs per SM, not three), so it takes fewer context splits to
+      // stay within one resident wave
+      const int ns = split ? std::max(1, std::min(n_splits, 2 * sm_count() / std::max(1, M * d.Hkv))) : n_splits;
+      HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_decode_fused(s->qkv32, d.qkv_rows, kv_layer, s->rope_table, s->attn, ns,
                                                         2, tc_err_flag_ptr(), bm, d, st, split ? s->row_scale : nullptr,
                                                         split ? s->klo_pool : nullptr));
     } else if (split) {
@@ -834,7 +837,7 @@ extern "C" int hyp_stage_profile(hyp_stage* s, int32_t mode, int32_t batch, int3
   for (auto& e : ev) HYP_CUDA_TRY(cudaEventCreate(&e));
   rc = HYP_OK;
   for (int it = -1; it < iters && rc == HYP_OK; ++it) {
-    fill_pattern_kernel<<<148 * 4, 256, 0, st>>>(s->x, (size_t)M * s->dims.H);
+    fill_pattern_kernel<<<sm_count() * 4, 256, 0, st>>>(s->x, (size_t)M * s->dims.H);
     s->launches += 1;
     rc = run_blocks(s, bm, decode, n_splits, st, it < 0 ? nullptr : &ev[(size_t)it * (s->L + 1)]);
   }
