@@ -88,10 +88,13 @@ HYP_API int hyp_op_gemm(const void* a, const void* w_packed, int32_t M, int32_t 
  *                          block are formed from two-term fp16 queries and keys (~21 significant bits) and the
  *                          RMSNorm factor is applied after the q/k/v projection, whose input is then the embedding
  *                          row itself; 0: block 0 runs like every other block (11-bit operands)
+ *   HYP_TUNE_TILE_224      value != 0 (the default): projections of more than 128 rows with whole-tile epilogues may
+ *                          use 256 x 224 tiles per CTA pair where that fills the last wave of the GPU better than
+ *                          256 x 256 (e.g. 7680 columns at 512 rows: 70 tiles on 74 pairs); 0: always 256 x 256
  * Affects launches made after the call; decode graphs already captured keep their setting. */
 enum { HYP_TUNE_PDL = 0, HYP_TUNE_STREAM_SLOTS = 1, HYP_TUNE_ATTN_SPLITS = 2, HYP_TUNE_ATTN_SLOTS = 3,
        HYP_TUNE_STREAM_ROTATION = 4, HYP_TUNE_SWAP_MIN_ROWS = 5, HYP_TUNE_SWAP_MAX_ROWS = 6, HYP_TUNE_SWAP_EPILOGUES = 7,
-       HYP_TUNE_PREFILL_ATTN_TC = 8, HYP_TUNE_FIRST_BLOCK_SPLIT = 9 };
+       HYP_TUNE_PREFILL_ATTN_TC = 8, HYP_TUNE_FIRST_BLOCK_SPLIT = 9, HYP_TUNE_TILE_224 = 10 };
 HYP_API int hyp_tune(int32_t key, int32_t value);
 
 /* Number of context splits hyp_op_attn_decode would pick for this batch, and the scratch bytes

@@ -347,8 +347,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 constexpr int STAGES2 = 6;
 constexpr int STAGE2_BYTES = A_BYTES + B_BYTES / 2;  // per CTA: 16 KB of A + 16 KB of its half of B
 constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 /*alignment*/ + 1024 /*barriers*/ + EPI_STAGING_BYTES;
-constexpr uint32_t IDESC2_BF16 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-constexpr uint32_t IDESC2_F16 = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+constexpr uint32_t idesc2(bool f16, int bn) {  // M = 256 (the pair), N = bn, fp32 accumulate, both operands K-major
+  return (1u << 4) | (f16 ? 0u : ((1u << 7) | (1u << 10))) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -395,14 +396,17 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uin
       : "memory");
 }
 
-template <int EPI>
+// BNT: accumulator columns of the pair's tile, 256 or 224 (each CTA supplies BNT / 2 weight rows = 8 or 7 packed
+// tiles per k-block; the launcher picks the width that leaves the fewest idle pairs in the last wave).
+template <int EPI, int BNT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                 const __grid_constant__ CUtensorMap tm_out, int M, int N, int K, int up_tile0, int team, uint32_t idesc,
                 int* __restrict__ err) {
   constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
   const bool STREAMK = EPI == EPI_RESID_F32 && team > 0;
-  constexpr int BN_OUT = SWIGLU ? BN / 2 : BN;
+  constexpr int BN_OUT = SWIGLU ? BNT / 2 : BNT;
+  constexpr int B_HALF_BYTES = (BNT / 2) * BK * 2;  // this CTA's half of the weight tile
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* aligned = smem_raw + (base - smem_u32(smem_raw));
@@ -463,12 +467,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         const int m0 = (tile % pairs_m) * (2 * BM) + (int)rank * BM;
         const int n0 = (tile / pairs_m) * BN_OUT;
         // this CTA's half of the weight tile, as an index of 16-row packed tiles
-        const int tb = SWIGLU ? (int)rank * up_tile0 + (n0 >> 4) : (n0 >> 4) + (int)rank * 8;
+        const int tb = SWIGLU ? (int)rank * up_tile0 + (n0 >> 4) : (n0 >> 4) + (int)rank * (BNT / 32);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) { ok = false; break; }
           const uint32_t sa = base + stage * STAGE2_BYTES, sb = sa + A_BYTES;
           const uint32_t lead_full = mapa_rank(full_bar(stage), 0);
-          if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * STAGE2_BYTES);
+          if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * (A_BYTES + B_HALF_BYTES));
           tma_load_2d_pair(sa, &tm_a, kb * BK, m0, lead_full);
           tma_load_4d_pair(sb, &tm_b, 0, 0, kb, tb, lead_full);
           if (++stage == STAGES2) { stage = 0; phase ^= 1; }
@@ -529,7 +533,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t t0 = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * BN);
-      epilogue_warp<EPI, BN>(t0, &tm_out, boxes, lane, m0 + 32 * q, n0, N, idesc == IDESC2_F16, n_box);
+      epilogue_warp<EPI, BNT>(t0, &tm_out, boxes, lane, m0 + 32 * q, n0, N, (idesc & (1u << 7)) == 0, n_box);
       tc_fence_before();
       mbar_arrive_cluster(mapa_rank(tempty_bar(acc), 0));
       acc ^= 1;
@@ -609,22 +613,38 @@ int encode_out_map(CUtensorMap* map, void* out, int ldo, int M, int N, int epi, 
 
 int* g_err_flag = nullptr;  // one device word per process: first non-zero code wins
 
+template <int EPI, int BNT>
+int launch_pair_bn(const TcAct& act, const TcWeight& w, int M, int N, int K, void* out, int ldo, cudaStream_t st,
+                   long pairs, int team, bool early) {
+  static bool configured = false;
+  if (!configured) {
+    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_tc2_kernel<EPI, BNT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
+    configured = true;
+  }
+  CUtensorMap tm_out;
+  const int mrc = encode_out_map(&tm_out, out, ldo, M, N, EPI, act.f16);
+  if (mrc) return mrc;
+  const CUtensorMap& tm_b = BNT == 256 ? w.map : w.map7;
+  if (early)
+    HYP_CUDA_TRY(launch_pdl<1>(gemm_tc2_kernel<EPI, BNT>, dim3((unsigned)(2 * pairs)), dim3(TC_THREADS), (size_t)SMEM2_BYTES, st,
+                               act.map, tm_b, tm_out, M, N, K, w.N16p, team, idesc2(act.f16, BNT), g_err_flag));
+  else
+    HYP_CUDA_TRY(launch_pdl(gemm_tc2_kernel<EPI, BNT>, dim3((unsigned)(2 * pairs)), dim3(TC_THREADS), (size_t)SMEM2_BYTES, st,
+                            act.map, tm_b, tm_out, M, N, K, w.N16p, team, idesc2(act.f16, BNT), g_err_flag));
+  return 1;
+}
+
 template <int EPI>
 int launch_pair(const TcAct& act, const TcWeight& w, int M, int N, int K, void* out, int ldo, cudaStream_t st,
                 int num_sms, bool early) {
-  static bool configured = false;
-  if (!configured) {
-    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_tc2_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
-    configured = true;
-  }
-  constexpr int BN_OUT = EPI == EPI_SWIGLU_BF16 ? BN / 2 : BN;
-  const int pairs_m = (M + 2 * BM - 1) / (2 * BM), tiles_n = (N + BN_OUT - 1) / BN_OUT;
-  const long tiles = (long)pairs_m * tiles_n;
+  constexpr int OUT_PER_ACC = EPI == EPI_SWIGLU_BF16 ? 2 : 1;  // SwiGLU: a gate and an up column per output column
+  const int pairs_m = (M + 2 * BM - 1) / (2 * BM);
   long pairs = num_sms / 2;
   int team = 0;  // 0 = whole tiles per CTA pair
   if (EPI == EPI_RESID_F32) {
     // stream-K over CTA pairs: teams of `team` pairs (a divisor of the 256-row M-tiles) share the weight k-blocks
     // they walk; every team gets the same number of k-blocks
+    const int tiles_n = (N + BN - 1) / BN;
     double best = -1.0;
     team = 1;
     for (int ts = 1; ts <= pairs_m && ts <= pairs; ++ts) {
@@ -637,19 +657,21 @@ int launch_pair(const TcAct& act, const TcWeight& w, int M, int N, int K, void* 
     const long cols = (long)(pairs_m / team) * tiles_n * ((K + BK - 1) / BK);
     if (teams > cols) teams = cols;
     pairs = teams * team;
-  } else if (tiles < pairs) {
-    pairs = tiles;
+    return launch_pair_bn<EPI, 256>(act, w, M, N, K, out, ldo, st, pairs, team, early);
   }
-  CUtensorMap tm_out;
-  const int mrc = encode_out_map(&tm_out, out, ldo, M, N, EPI, act.f16);
-  if (mrc) return mrc;
-  if (early)
-    HYP_CUDA_TRY(launch_pdl<1>(gemm_tc2_kernel<EPI>, dim3((unsigned)(2 * pairs)), dim3(TC_THREADS), (size_t)SMEM2_BYTES, st,
-                               act.map, w.map, tm_out, M, N, K, w.N16p, team, act.f16 ? IDESC2_F16 : IDESC2_BF16, g_err_flag));
-  else
-    HYP_CUDA_TRY(launch_pdl(gemm_tc2_kernel<EPI>, dim3((unsigned)(2 * pairs)), dim3(TC_THREADS), (size_t)SMEM2_BYTES, st,
-                            act.map, w.map, tm_out, M, N, K, w.N16p, team, act.f16 ? IDESC2_F16 : IDESC2_BF16, g_err_flag));
-  return 1;
+  // whole tiles per pair: a 224-column tile is taken when it needs less tensor time over all waves than a 256-column
+  // one (7680 columns at 512 rows: 70 tiles of 224 fill 74 pairs once, 60 tiles of 256 leave 14 idle for longer)
+  auto waves_cost = [&](int bn, long* tiles_out) {
+    const long tiles = (long)pairs_m * ((N + bn / OUT_PER_ACC - 1) / (bn / OUT_PER_ACC));
+    *tiles_out = tiles;
+    return ((tiles + pairs - 1) / pairs) * bn;
+  };
+  long tiles256, tiles224;
+  const long c256 = waves_cost(256, &tiles256), c224 = waves_cost(224, &tiles224);
+  // (fp32 stores only: their 32-column output boxes divide 224, the 64-column boxes of the 16-bit epilogues do not)
+  if (EPI == EPI_STORE_F32 && c224 < c256 && tile_width_224_enabled())
+    return launch_pair_bn<EPI, 224>(act, w, M, N, K, out, ldo, st, tiles224 < pairs ? tiles224 : pairs, 0, early);
+  return launch_pair_bn<EPI, 256>(act, w, M, N, K, out, ldo, st, tiles256 < pairs ? tiles256 : pairs, 0, early);
 }
 
 template <int EPI>
@@ -719,11 +741,21 @@ int tc_make_weight(TcWeight* w, const void* packed, int rows, int halves, int K,
   CUresult r = enc(&w->map, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void*)packed, dims,
                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  const cuuint32_t box7[4] = {64, 16, 1, 7};  // 112 rows: a CTA's half of a 224-column pair tile
+  if (r == CUDA_SUCCESS)
+    r = enc(&w->map7, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void*)packed, dims, strides,
+            box7, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     set_last_cuda_error((int)r);
     return HYP_ECUDA;
   }
   return HYP_OK;
+}
+
+int& tile_width_224_enabled() {
+  static int v = 1;
+  return v;
 }
 
 namespace {

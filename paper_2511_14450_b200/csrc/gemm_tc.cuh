@@ -21,6 +21,7 @@ struct TcWeight {
   int K = 0, KBp = 0, N16p = 0;
   bool f16 = false;
   CUtensorMap map;  // 4-D view {64 k, 16 rows, KBp, halves * N16p}, box = 8 tiles x 1 k-block (128 rows), no swizzle
+  CUtensorMap map7;  // the same view with boxes of 7 tiles (112 rows)
 };
 inline int pk_kbp(int K) { return ((K + 63) / 64 + 1) & ~1; }
 inline int pk_n16p(int rows) { return ((rows + 15) / 16 + 1) & ~1; }
@@ -49,6 +50,9 @@ int tc_make_kv_map(CUtensorMap* map, const void* kv_layer, size_t n_pages, int H
 int& attn_prefill_tc_enabled();
 int launch_attn_prefill_tc(const CUtensorMap& q_map, const CUtensorMap& kv_map, __half* attn_out, const BatchMeta& bm,
                            const ModelDims& d, cudaStream_t st);
+
+// 1 (default): the two-CTA tile kernel may take 224-column tiles where they fill the last wave better.
+int& tile_width_224_enabled();
 
 // One-time set-up of the device-side error word (allocates; call from stage creation, not from the hot path).
 int tc_prepare();

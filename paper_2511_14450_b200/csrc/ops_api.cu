@@ -85,6 +85,9 @@ extern "C" int hyp_tune(int32_t key, int32_t value) {
       if (value < 0 || value > 8) return HYP_EINVAL;
       attn_fused_splits_override() = value;
       return HYP_OK;
+    case HYP_TUNE_TILE_224:
+      tile_width_224_enabled() = value != 0;
+      return HYP_OK;
     case HYP_TUNE_FIRST_BLOCK_SPLIT:
       first_block_split() = value != 0;
       return HYP_OK;
