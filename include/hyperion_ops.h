@@ -67,6 +67,22 @@ HYP_API int hyp_op_pack_weight(const void* w, int32_t N, int32_t K, int32_t swig
 HYP_API int hyp_op_gemm(const void* a, const void* w_packed, int32_t M, int32_t N, int32_t K, int32_t epilogue,
                         void* out, int32_t ldo, void* stream);
 
+/* The same two calls for the fp16 instantiation, the one hyp_stage_* runs (reading 11 of the block's arithmetic:
+ * fp16 operands, fp32 accumulation): hyp_op_pack_weight_f16 converts the bf16 matrix to fp16 while tiling it
+ * (exact for |w| >= 2^-17, saturating at +-65504); hyp_op_gemm_f16 takes `a` as fp16 [M, K] and such a packed
+ * copy, and its 16-bit epilogues write fp16.  Everything else as above. */
+HYP_API int hyp_op_pack_weight_f16(const void* w, int32_t N, int32_t K, int32_t swiglu, void* packed, size_t packed_bytes,
+                                   void* stream);
+HYP_API int hyp_op_gemm_f16(const void* a, const void* w_packed, int32_t M, int32_t N, int32_t K, int32_t epilogue,
+                            void* out, int32_t ldo, void* stream);
+
+/* Device-side wait status.  Every wait inside the library's kernels (on a copy's completion, on tensor memory, on a
+ * peer CTA) is bounded; a kernel whose wait runs out records a small non-zero code in one device word, unwinds and
+ * returns by itself (its results are invalid).  The calls that synchronise report that word as HYP_ETIMEOUT; this
+ * call reads it for the others: it synchronises the device, writes the code to *code_out (HOST; 0 = no wait ever
+ * expired) and, if clear != 0, resets the word.  Errors: HYP_EINVAL, HYP_ECUDA. */
+HYP_API int hyp_device_wait_status(int32_t* code_out, int32_t clear);
+
 /* Process-wide tuning switches (measurement aids; the defaults are the measured best).
  *   HYP_TUNE_PDL           which kernels are launched with programmatic dependent launch, so that their
  *                          prologue and weight prefetch may overlap the predecessor's tail: 0 none, 1 the
@@ -91,10 +107,17 @@ HYP_API int hyp_op_gemm(const void* a, const void* w_packed, int32_t M, int32_t 
  *   HYP_TUNE_TILE_224      value != 0 (the default): projections of more than 128 rows with whole-tile epilogues may
  *                          use 256 x 224 tiles per CTA pair where that fills the last wave of the GPU better than
  *                          256 x 256 (e.g. 7680 columns at 512 rows: 70 tiles on 74 pairs); 0: always 256 x 256
+ *   HYP_TUNE_WAIT_LIMIT_US  limit of the weight-streaming kernel's bounded waits in microseconds (0 = the built-in
+ *                          4 s; the other kernels always use 4 s)
+ *   HYP_TUNE_STREAM_WITHHOLD_COPY  value != 0: the NEXT launch of the weight-streaming kernel leaves one weight copy
+ *                          unissued, so that one warp's wait runs into the limit and the kernel takes its
+ *                          give-up path (records code 4, lets its other copies land, returns).  One-shot; exists
+ *                          so that the HYP_ETIMEOUT path can be exercised without faulting or hanging anything.
  * Affects launches made after the call; decode graphs already captured keep their setting. */
 enum { HYP_TUNE_PDL = 0, HYP_TUNE_STREAM_SLOTS = 1, HYP_TUNE_ATTN_SPLITS = 2, HYP_TUNE_ATTN_SLOTS = 3,
        HYP_TUNE_STREAM_ROTATION = 4, HYP_TUNE_SWAP_MIN_ROWS = 5, HYP_TUNE_SWAP_MAX_ROWS = 6, HYP_TUNE_SWAP_EPILOGUES = 7,
-       HYP_TUNE_PREFILL_ATTN_TC = 8, HYP_TUNE_FIRST_BLOCK_SPLIT = 9, HYP_TUNE_TILE_224 = 10 };
+       HYP_TUNE_PREFILL_ATTN_TC = 8, HYP_TUNE_FIRST_BLOCK_SPLIT = 9, HYP_TUNE_TILE_224 = 10,
+       HYP_TUNE_WAIT_LIMIT_US = 11, HYP_TUNE_STREAM_WITHHOLD_COPY = 12 };
 HYP_API int hyp_tune(int32_t key, int32_t value);
 
 /* Number of context splits hyp_op_attn_decode would pick for this batch, and the scratch bytes

@@ -30,6 +30,14 @@ int& gemm_stream_rotation() {
   static int v = 13;
   return v;
 }
+int& gemm_stream_wait_limit_us() {
+  static int v = 0;
+  return v;
+}
+int& gemm_stream_withhold_next() {
+  static int v = 0;
+  return v;
+}
 
 namespace {
 
@@ -59,7 +67,8 @@ __device__ __forceinline__ uint4 ldg_act(const void* p) {
 template <int NB, int EPI, int TILES, bool F16>
 __global__ void __launch_bounds__(GS_THREADS, 3)
 gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ act, int lda, int K, int N, int KBp,
-                   int tile1_off, int M, void* __restrict__ out, int ldo, int S, int rot_mul, int* __restrict__ err) {
+                   int tile1_off, int M, void* __restrict__ out, int ldo, int S, int rot_mul, int* __restrict__ err,
+                   uint64_t wait_ns, int withhold) {
   constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
   static_assert(!SWIGLU || TILES == 2, "SwiGLU pairs a gate strip with an up strip");
   constexpr int OUT_COLS = (TILES == 2 && !SWIGLU) ? 32 : 16;
@@ -89,10 +98,12 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
     const int ch = ch_logical + rot;
     return ch >= NCH ? ch - NCH : ch;
   };
+  uint32_t inflight = 0;  // lane 0: slots whose copy has been asked for and not yet been waited for
   // weights: never written by any kernel, may be fetched before the predecessor has finished
   auto issue_w = [&](int ch_logical, int slot) {
     const int ch = actual(ch_logical);
     const uint32_t dst = my_ring + slot * STAGE_BYTES, bar = my_bars + 8u * slot;
+    inflight |= 1u << slot;
     mbar_expect_tx(bar, STAGE_BYTES);
     bulk_load(dst, w0 + (size_t)ch * W_CHUNK_BYTES, W_CHUNK_BYTES, bar);
     if (TILES == 2) bulk_load(dst + W_CHUNK_BYTES, w1 + (size_t)ch * W_CHUNK_BYTES, W_CHUNK_BYTES, bar);
@@ -104,8 +115,10 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
   if (lane == 0) {
     for (int sl = 0; sl < S; ++sl) mbar_init(my_bars + 8u * sl, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // `withhold` (a test hook, see launch_cfg): warp 0 of CTA 0 never asks for its first copy, so its first
+    // wait below runs into the limit and the kernel leaves through the path that a lost copy would take
     for (int sl = 0; sl < S; ++sl)
-      if (warp + GS_WARPS * sl < NCH) issue_w(warp + GS_WARPS * sl, sl);
+      if (warp + GS_WARPS * sl < NCH && !(withhold && blockIdx.x == 0 && warp == 0 && sl == 0)) issue_w(warp + GS_WARPS * sl, sl);
   }
   __syncwarp();
 
@@ -142,7 +155,9 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
   // shared-memory offset of this lane's 16 bytes in tile row g, first 32-k group (the tile is stored swizzled:
   // 16-byte chunk c of row r sits at chunk position c ^ (r & 7); rows g and g + 8 share g & 7)
   for (int ch = warp; ch < NCH; ch += GS_WARPS) {
-    if (!mbar_wait(my_bars + 8u * slot, phase, nullptr)) { ok = false; break; }
+    // one decision for the whole warp (a bounded wait could run out for some lanes only)
+    if (!__all_sync(0xffffffffu, mbar_wait(my_bars + 8u * slot, phase, nullptr, wait_ns))) { ok = false; break; }
+    inflight &= ~(1u << slot);
     const uint32_t sbase = my_ring + slot * STAGE_BYTES;
     const bool more = ch + GS_WARPS < NCH;
 #pragma unroll
@@ -175,9 +190,15 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
     if (++slot == S) { slot = 0; phase ^= 1u; }
   }
   if (!ok) {
-    // a copy never landed: record it and let whatever is still in flight arrive (bounded) before leaving
-    if (lane == 0) atomicCAS(err, 0, 4);
-    for (int sl = 0; sl < S; ++sl) mbar_wait(my_bars + 8u * sl, 0, nullptr), mbar_wait(my_bars + 8u * sl, 1, nullptr);
+    // a copy never landed: record it and let whatever is still in flight arrive (bounded) before leaving, so that
+    // no copy writes into shared memory that already belongs to another CTA.  Slots from the failing one on still
+    // owe the current phase, the slots before it were refilled for the next one.
+    if (lane == 0) {
+      atomicCAS(err, 0, 4);
+      for (int sl = 0; sl < S; ++sl)
+        if ((inflight >> sl) & 1u) mbar_wait(my_bars + 8u * sl, sl >= slot ? phase : phase ^ 1u, nullptr, wait_ns);
+    }
+    __syncwarp();
   }
   // partial sums of this warp go to the start of its own ring space (nothing is in flight into it any more)
   float* red = reinterpret_cast<float*>(base_ptr);
@@ -259,16 +280,21 @@ int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, void* out, int
   if (slots > GS_MAX_SLOTS) slots = GS_MAX_SLOTS;
   while (slots > 2 && GS_WARPS * slots * STAGE_BYTES + 128 > MAX_DYN) --slots;
   const int smem = GS_WARPS * slots * STAGE_BYTES + 128;
+  // bounded waits: 4 s unless a shorter limit was set (hyp_tune); `withhold` is a one-shot test hook that makes
+  // one wait of the next launch run into that limit (nothing faults: the kernel records the code and returns)
+  const uint64_t wait_ns = gemm_stream_wait_limit_us() > 0 ? (uint64_t)gemm_stream_wait_limit_us() * 1000ull : WAIT_LIMIT_NS;
+  const int withhold = gemm_stream_withhold_next();
+  gemm_stream_withhold_next() = 0;
   // the kernel fetches weights before it waits for its predecessor: launched early only when the weights cannot
   // be that predecessor's output
   if (early)
     HYP_CUDA_TRY(launch_pdl<1>(gemm_stream_kernel<NB, EPI, TILES, F16>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
                                (const uint8_t*)w.packed, (const uint16_t*)act.ptr, act.K, act.K, N, w.KBp, w.N16p, M, out,
-                               ldo, slots, gemm_stream_rotation(), tc_err_flag_ptr()));
+                               ldo, slots, gemm_stream_rotation(), tc_err_flag_ptr(), wait_ns, withhold));
   else
     HYP_CUDA_TRY(launch_pdl<4>(gemm_stream_kernel<NB, EPI, TILES, F16>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
                                (const uint8_t*)w.packed, (const uint16_t*)act.ptr, act.K, act.K, N, w.KBp, w.N16p, M, out,
-                               ldo, slots, gemm_stream_rotation(), tc_err_flag_ptr()));
+                               ldo, slots, gemm_stream_rotation(), tc_err_flag_ptr(), wait_ns, withhold));
   return 1;
 }
 

@@ -839,6 +839,12 @@ int tc_error_flag(int* value_out) {
   return HYP_OK;
 }
 
+int tc_error_flag_take(int* value_out, bool clear) {
+  const int rc = tc_error_flag(value_out);
+  if (rc == HYP_OK && clear && g_err_flag && *value_out) HYP_CUDA_TRY(cudaMemset(g_err_flag, 0, sizeof(int)));
+  return rc;
+}
+
 int launch_gemm_tc(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,
                    cudaStream_t st, bool early) {
   if (M < 1 || N < 1 || K < 8 || act.K != K || w.K != K || M > act.rows || !g_err_flag) return HYP_EINVAL;

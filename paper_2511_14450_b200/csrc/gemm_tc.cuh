@@ -67,6 +67,14 @@ int& gemm_stream_slots_override();
 // Per-CTA stagger of the K walk of the weight-streaming kernel: CTA b starts at copy (b * rotation) mod copies.
 int& gemm_stream_rotation();
 
+// Limit of the weight-streaming kernel's bounded waits in microseconds (0 = the built-in 4 s), and a one-shot hook
+// that makes the next launch of that kernel withhold one copy so that a wait runs into the limit (for the test of
+// the HYP_ETIMEOUT path: no fault, the kernel records the code and returns).
+int& gemm_stream_wait_limit_us();
+int& gemm_stream_withhold_next();
+// Reads the device word like tc_error_flag and, if `clear`, zeroes it afterwards.
+int tc_error_flag_take(int* value_out, bool clear);
+
 // Weight-streaming projection for M <= 8 rows (decode); same contract as launch_gemm_tc.  `early`: the packed
 // weights are long-lived (not written by the kernel launched just before), so the launch may overlap that kernel.
 int launch_gemm_stream(const TcAct& act, const TcWeight& w, int M, int N, int K, int epi, void* out, int ldo,

@@ -44,12 +44,31 @@ extern "C" size_t hyp_op_weight_packed_bytes(int32_t N, int32_t K, int32_t swigl
   return tc_packed_bytes(N, swiglu ? 2 : 1, K);
 }
 
-extern "C" int hyp_op_pack_weight(const void* w, int32_t N, int32_t K, int32_t swiglu, void* packed, size_t packed_bytes,
-                                  void* stream) {
+namespace {
+int pack_weight(const void* w, int32_t N, int32_t K, int32_t swiglu, void* packed, size_t packed_bytes, void* stream,
+                bool to_f16) {
   if (!w || !packed || N < 1 || K < 8 || K % 8) return HYP_EINVAL;
   if (((uintptr_t)w & 15) != 0 || ((uintptr_t)packed & 127) != 0) return HYP_EINVAL;
   if (packed_bytes < tc_packed_bytes(N, swiglu ? 2 : 1, K)) return HYP_ECAPACITY;
-  return finish(tc_pack_weight(w, packed, N, swiglu ? 2 : 1, K, false, (cudaStream_t)stream));
+  return finish(tc_pack_weight(w, packed, N, swiglu ? 2 : 1, K, to_f16, (cudaStream_t)stream));
+}
+}  // namespace
+
+extern "C" int hyp_op_pack_weight(const void* w, int32_t N, int32_t K, int32_t swiglu, void* packed, size_t packed_bytes,
+                                  void* stream) {
+  return pack_weight(w, N, K, swiglu, packed, packed_bytes, stream, false);
+}
+extern "C" int hyp_op_pack_weight_f16(const void* w, int32_t N, int32_t K, int32_t swiglu, void* packed,
+                                      size_t packed_bytes, void* stream) {
+  return pack_weight(w, N, K, swiglu, packed, packed_bytes, stream, true);
+}
+
+extern "C" int hyp_device_wait_status(int32_t* code_out, int32_t clear) {
+  if (!code_out) return HYP_EINVAL;
+  int v = 0;
+  const int rc = tc_error_flag_take(&v, clear != 0);
+  *code_out = v;
+  return rc;
 }
 
 extern "C" int hyp_tune(int32_t key, int32_t value) {
@@ -85,6 +104,13 @@ extern "C" int hyp_tune(int32_t key, int32_t value) {
       if (value < 0 || value > 8) return HYP_EINVAL;
       attn_fused_splits_override() = value;
       return HYP_OK;
+    case HYP_TUNE_WAIT_LIMIT_US:
+      if (value < 0) return HYP_EINVAL;
+      gemm_stream_wait_limit_us() = value;
+      return HYP_OK;
+    case HYP_TUNE_STREAM_WITHHOLD_COPY:
+      gemm_stream_withhold_next() = value != 0;
+      return HYP_OK;
     case HYP_TUNE_TILE_224:
       tile_width_224_enabled() = value != 0;
       return HYP_OK;
@@ -99,8 +125,9 @@ extern "C" int hyp_tune(int32_t key, int32_t value) {
   }
 }
 
-extern "C" int hyp_op_gemm(const void* a, const void* w, int32_t M, int32_t N, int32_t K, int32_t epilogue, void* out,
-                           int32_t ldo, void* stream) {
+namespace {
+int op_gemm(const void* a, const void* w, int32_t M, int32_t N, int32_t K, int32_t epilogue, void* out, int32_t ldo,
+            void* stream, bool f16) {
   if (!a || !w || !out || M < 1 || N < 1 || K < 8 || K % 8 || ldo < N || ((uintptr_t)w & 127) != 0) return HYP_EINVAL;
   if (epilogue < HYP_EPI_STORE_BF16 || epilogue > HYP_EPI_STORE_F32) return HYP_EINVAL;
   cudaStream_t st = (cudaStream_t)stream;
@@ -109,11 +136,21 @@ extern "C" int hyp_op_gemm(const void* a, const void* w, int32_t M, int32_t N, i
   if (rc) return rc;
   TcAct ta;
   TcWeight tw;
-  rc = tc_make_act(&ta, (const __nv_bfloat16*)a, M, K);
+  rc = tc_make_act(&ta, a, M, K, f16);
   if (rc) return rc;
-  rc = tc_make_weight(&tw, w, N, epilogue == HYP_EPI_SWIGLU_BF16 ? 2 : 1, K, false);
+  rc = tc_make_weight(&tw, w, N, epilogue == HYP_EPI_SWIGLU_BF16 ? 2 : 1, K, f16);
   if (rc) return rc;
   return finish(launch_projection(ta, tw, M, N, K, epilogue, out, ldo, st));
+}
+}  // namespace
+
+extern "C" int hyp_op_gemm(const void* a, const void* w, int32_t M, int32_t N, int32_t K, int32_t epilogue, void* out,
+                           int32_t ldo, void* stream) {
+  return op_gemm(a, w, M, N, K, epilogue, out, ldo, stream, false);
+}
+extern "C" int hyp_op_gemm_f16(const void* a, const void* w, int32_t M, int32_t N, int32_t K, int32_t epilogue, void* out,
+                               int32_t ldo, void* stream) {
+  return op_gemm(a, w, M, N, K, epilogue, out, ldo, stream, true);
 }
 
 extern "C" int hyp_op_attn_decode_splits(int32_t n_seqs, int32_t n_kv_heads, int32_t max_ctx) {

@@ -37,7 +37,8 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // Bounded wait.  Returns false after WAIT_LIMIT_NS or once another role has raised `abort_flag`
 // (null: time limit only).  An mbarrier distinguishes only the current phase from the one before it,
 // so a given barrier must be waited on by one thread sequence that never skips a phase.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          uint64_t limit_ns = WAIT_LIMIT_NS) {
   for (int i = 0; i < 64; ++i)
     if (mbar_try(bar, parity)) return true;
   const uint64_t t0 = globaltimer();
@@ -45,7 +46,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     for (int i = 0; i < 256; ++i)
       if (mbar_try(bar, parity)) return true;
     if (abort_flag && *abort_flag) return false;
-    if (globaltimer() - t0 > WAIT_LIMIT_NS) return false;
+    if (globaltimer() - t0 > limit_ns) return false;
   }
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {

@@ -86,6 +86,10 @@ SIGNATURES = {
     "hyp_tune": (C.c_int, [C.c_int32, C.c_int32]),
     "hyp_op_gemm": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
                               C.c_int32, C.c_void_p]),
+    "hyp_op_pack_weight_f16": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "hyp_op_gemm_f16": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                  C.c_int32, C.c_void_p]),
+    "hyp_device_wait_status": (C.c_int, [C.POINTER(C.c_int32), C.c_int32]),
     "hyp_op_attn_decode_splits": (C.c_int, [C.c_int32, C.c_int32, C.c_int32]),
     "hyp_op_attn_decode_scratch_bytes": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
     "hyp_op_attn_decode": (C.c_int, [C.POINTER(hyp_attn_shape), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
@@ -300,23 +304,24 @@ def hyp_op_rmsnorm(x, g, out, eps: float, stream=None):
 
 (HYP_TUNE_PDL, HYP_TUNE_STREAM_SLOTS, HYP_TUNE_ATTN_SPLITS, HYP_TUNE_ATTN_SLOTS, HYP_TUNE_STREAM_ROTATION,
  HYP_TUNE_SWAP_MIN_ROWS, HYP_TUNE_SWAP_MAX_ROWS, HYP_TUNE_SWAP_EPILOGUES, HYP_TUNE_PREFILL_ATTN_TC,
- HYP_TUNE_FIRST_BLOCK_SPLIT, HYP_TUNE_TILE_224) = range(11)
+ HYP_TUNE_FIRST_BLOCK_SPLIT, HYP_TUNE_TILE_224, HYP_TUNE_WAIT_LIMIT_US, HYP_TUNE_STREAM_WITHHOLD_COPY) = range(13)
 
 
 def hyp_tune(key: int, value: int):
     _check(lib().hyp_tune(key, value), "hyp_tune")
 
 
-def hyp_op_pack_weight(w, N: int, swiglu: bool, stream=None):
-    """Packed copy of a bf16 [N (2N for SwiGLU), K] weight matrix, as hyp_op_gemm reads it (a uint8 tensor)."""
+def hyp_op_pack_weight(w, N: int, swiglu: bool, stream=None, f16: bool = False):
+    """Packed copy of a bf16 [N (2N for SwiGLU), K] weight matrix, as hyp_op_gemm reads it (a uint8 tensor);
+    f16: the values converted to fp16 on the way (hyp_op_pack_weight_f16, for hyp_op_gemm_f16)."""
     import torch
     K = w.shape[1]
     nbytes = lib().hyp_op_weight_packed_bytes(N, K, int(swiglu))
     if nbytes == 0:
         raise HyperionError(HYP_EINVAL, "hyp_op_weight_packed_bytes")
     packed = torch.empty(nbytes, dtype=torch.uint8, device=w.device)
-    _check(lib().hyp_op_pack_weight(_ptr(w), N, K, int(swiglu), _ptr(packed), nbytes, _stream_handle(stream)),
-           "hyp_op_pack_weight")
+    name = "hyp_op_pack_weight_f16" if f16 else "hyp_op_pack_weight"
+    _check(getattr(lib(), name)(_ptr(w), N, K, int(swiglu), _ptr(packed), nbytes, _stream_handle(stream)), name)
     return packed
 
 
@@ -324,6 +329,19 @@ def hyp_op_gemm(a, w_packed, N: int, epilogue: int, out, stream=None):
     M, K = a.shape
     _check(lib().hyp_op_gemm(_ptr(a), _ptr(w_packed), M, N, K, epilogue, _ptr(out), out.stride(0),
                              _stream_handle(stream)), "hyp_op_gemm")
+
+
+def hyp_op_gemm_f16(a, w_packed, N: int, epilogue: int, out, stream=None):
+    M, K = a.shape
+    _check(lib().hyp_op_gemm_f16(_ptr(a), _ptr(w_packed), M, N, K, epilogue, _ptr(out), out.stride(0),
+                                 _stream_handle(stream)), "hyp_op_gemm_f16")
+
+
+def hyp_device_wait_status(clear: bool = False) -> int:
+    """Code recorded by a kernel whose bounded wait ran out (0 = none); synchronises the device."""
+    code = C.c_int32(0)
+    _check(lib().hyp_device_wait_status(C.byref(code), int(clear)), "hyp_device_wait_status")
+    return code.value
 
 
 def hyp_op_attn_decode_splits(n_seqs: int, n_kv_heads: int, max_ctx: int) -> int:

@@ -39,15 +39,20 @@ GEMM_SHAPES = [  # (M, N, K)
 @pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
 @pytest.mark.parametrize("epi", [hyp.HYP_EPI_STORE_BF16, hyp.HYP_EPI_RESID_F32, hyp.HYP_EPI_SWIGLU_BF16,
                                  hyp.HYP_EPI_STORE_F32])
-def test_gemm_all_epilogues(M, N, K, epi):
+@pytest.mark.parametrize("f16", [False, True])
+def test_gemm_all_epilogues(M, N, K, epi, f16):
+    """Both instantiations of the projection kernels: bf16 operands (hyp_op_gemm) and fp16 operands
+    (hyp_op_gemm_f16, the one the stage path runs)."""
     if M == 512 and epi not in (hyp.HYP_EPI_STORE_BF16, hyp.HYP_EPI_SWIGLU_BF16):
-        pytest.skip("full-size case runs the two bf16 epilogues only")
+        pytest.skip("full-size case runs the two 16-bit epilogues only")
     swiglu = epi == hyp.HYP_EPI_SWIGLU_BF16
     a = bf16_normal(3, (M, K))
     w = bf16_normal(4, ((2 * N if swiglu else N), K), std=1.0 / np.sqrt(K))
-    acc = f64(a) @ f64(w).T
+    if f16:
+        a = a.half()                       # bf16 values of this size are exact in fp16
+    acc = f64(a) @ f64(w.half() if f16 else w).T
     if epi in (hyp.HYP_EPI_STORE_BF16, hyp.HYP_EPI_SWIGLU_BF16):
-        out = torch.full((M, N), 7.0, dtype=torch.bfloat16, device="cuda")
+        out = torch.full((M, N), 7.0, dtype=torch.float16 if f16 else torch.bfloat16, device="cuda")
         want = od.silu(acc[:, :N]) * acc[:, N:] if swiglu else acc
         tol = 6e-3
     else:
@@ -55,7 +60,8 @@ def test_gemm_all_epilogues(M, N, K, epi):
         out = res.clone()
         want = acc + (f64(res) if epi == hyp.HYP_EPI_RESID_F32 else 0.0)
         tol = 2e-5 * np.sqrt(K)
-    hyp.hyp_op_gemm(a, hyp.hyp_op_pack_weight(w, N, swiglu), N, epi, out)
+    packed = hyp.hyp_op_pack_weight(w, N, swiglu, f16=f16)
+    (hyp.hyp_op_gemm_f16 if f16 else hyp.hyp_op_gemm)(a, packed, N, epi, out)
     torch.cuda.synchronize()
     err = np.abs(f64(out) - want) / (np.abs(want) + 1.0)
     assert np.max(err) < tol, (np.max(err), np.unravel_index(np.argmax(err), err.shape))
@@ -65,13 +71,14 @@ def test_gemm_all_epilogues(M, N, K, epi):
                                    (100, 1024, 688), (16, 17920, 512)])
 @pytest.mark.parametrize("epi", [hyp.HYP_EPI_STORE_BF16, hyp.HYP_EPI_RESID_F32, hyp.HYP_EPI_SWIGLU_BF16,
                                  hyp.HYP_EPI_STORE_F32])
-def test_gemm_swapped_operand_kernel_all_epilogues(M, N, K, epi):
+@pytest.mark.parametrize("f16", [False, True])
+def test_gemm_swapped_operand_kernel_all_epilogues(M, N, K, epi, f16):
     """Every epilogue and 1-128 rows forced through the swapped-operand kernel (by default it only takes the plain
     stores of 9-128 rows): ragged N (not a multiple of 128), K tails, clusters of 1-8 K shares, all four token tiles."""
     hyp.hyp_tune(hyp.HYP_TUNE_SWAP_MIN_ROWS, 1)
     hyp.hyp_tune(hyp.HYP_TUNE_SWAP_EPILOGUES, 15)
     try:
-        test_gemm_all_epilogues(M, N, K, epi)
+        test_gemm_all_epilogues(M, N, K, epi, f16)
     finally:
         hyp.hyp_tune(hyp.HYP_TUNE_SWAP_MIN_ROWS, 9)
         hyp.hyp_tune(hyp.HYP_TUNE_SWAP_EPILOGUES, (1 << hyp.HYP_EPI_STORE_BF16) | (1 << hyp.HYP_EPI_STORE_F32))
@@ -220,3 +227,31 @@ def test_attn_prefill(Hq, Hkv, D, lens, new):
         want = od.attention(qi, f64(ks[i]), f64(vs[i]), q_pos0=lens[i] - c).reshape(c, -1)
         assert np.max(np.abs(f64(out[row:row + c]) - want)) < 2e-2, i
         row += c
+
+
+def test_expired_wait_is_reported_and_the_next_call_is_clean():
+    """The give-up path of a bounded wait, driven once without faulting anything: with the wait limit at 1 ms, one
+    launch of the weight-streaming kernel is told to leave one weight copy unissued; the warp that waits for it runs
+    into the limit, the kernel records its code, lets its other copies land and returns by itself.  The status
+    call reports the code; after clearing it, the same projection is correct again and the status stays clean."""
+    M, N, K = 4, 512, 1024
+    a = bf16_normal(3, (M, K)).half()
+    w = bf16_normal(4, (N, K), std=1.0 / np.sqrt(K))
+    packed = hyp.hyp_op_pack_weight(w, N, False, f16=True)
+    want = f64(a) @ f64(w.half()).T
+    out = torch.zeros(M, N, dtype=torch.float32, device="cuda")
+    assert hyp.hyp_device_wait_status() == 0
+    hyp.hyp_tune(hyp.HYP_TUNE_WAIT_LIMIT_US, 1000)
+    try:
+        hyp.hyp_tune(hyp.HYP_TUNE_STREAM_WITHHOLD_COPY, 1)
+        hyp.hyp_op_gemm_f16(a, packed, N, hyp.HYP_EPI_STORE_F32, out)      # returns: the kernel gives up by itself
+        assert hyp.hyp_device_wait_status(clear=True) == 4                  # the streaming kernel's code
+        assert hyp.hyp_device_wait_status() == 0
+        out.zero_()
+        hyp.hyp_op_gemm_f16(a, packed, N, hyp.HYP_EPI_STORE_F32, out)      # the hook was one-shot
+        torch.cuda.synchronize()
+        assert np.max(np.abs(f64(out) - want)) < 2e-5 * np.sqrt(K) * (np.max(np.abs(want)) + 1.0)
+        assert hyp.hyp_device_wait_status() == 0
+    finally:
+        hyp.hyp_tune(hyp.HYP_TUNE_WAIT_LIMIT_US, 0)
+        hyp.hyp_tune(hyp.HYP_TUNE_STREAM_WITHHOLD_COPY, 0)
