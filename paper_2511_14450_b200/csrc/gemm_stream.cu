@@ -30,6 +30,10 @@ int& gemm_stream_rotation() {
   static int v = 13;
   return v;
 }
+int& gemm_stream_act_depth() {  // copies ahead that a warp's activation fragments are fetched; 0 = built-in choice
+  static int v = 0;
+  return v;
+}
 int& gemm_stream_wait_limit_us() {
   static int v = 0;
   return v;
@@ -64,7 +68,11 @@ __device__ __forceinline__ uint4 ldg_act(const void* p) {
 
 // TILES = 1: 16 output columns per CTA (one strip).  TILES = 2: 32 adjacent columns (strips 2b, 2b + 1), or (SwiGLU)
 // gate strip b and the matching up strip tile1_off + b.  S = ring slots per warp; a slot holds TILES copies.
-template <int NB, int EPI, int TILES, bool F16>
+// AD = how many of a warp's copies ahead its activation fragments are fetched.  A warp handles one copy per
+// iteration; with the fragments of only the next copy in flight an iteration cannot be shorter than one L2 round
+// trip.  Measured on the 14-block decode stage (batch 8, us per step): AD 1: 1837, AD 2: 1818, AD 3: 1830 (the
+// registers of the third copy cost more than its latency cover gives).
+template <int NB, int EPI, int TILES, bool F16, int AD>
 __global__ void __launch_bounds__(GS_THREADS, 3)
 gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ act, int lda, int K, int N, int KBp,
                    int tile1_off, int M, void* __restrict__ out, int ldo, int S, int rot_mul, int* __restrict__ err,
@@ -130,7 +138,7 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
     avalid[j] = 8 * j + g < M;
     arow[j] = act + (size_t)(avalid[j] ? 8 * j + g : 0) * lda + 8 * t;
   }
-  uint4 bq[GS_GROUPS][NB];  // fragment entries of the copy being worked on, refilled group by group for the next one
+  uint4 bq[AD][GS_GROUPS][NB];  // fragment entries of this warp's next AD copies, refilled group by group as they are used
   auto load_act = [&](int ch_logical, int q, uint4 (&dst)[NB]) {
     const int k = actual(ch_logical) * GS_CHUNK_K + q * 32;
 #pragma unroll
@@ -138,9 +146,12 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
       dst[j] = (avalid[j] && k + 8 * t < K) ? ldg_act(arow[j] + k) : make_uint4(0u, 0u, 0u, 0u);
   };
   pdl_wait();  // activations (and, for the residual epilogue, the output) belong to the predecessor until here
-  if (warp < NCH) {
 #pragma unroll
-    for (int q = 0; q < GS_GROUPS; ++q) load_act(warp, q, bq[q]);
+  for (int a = 0; a < AD; ++a) {
+    if (warp + GS_WARPS * a < NCH) {
+#pragma unroll
+      for (int q = 0; q < GS_GROUPS; ++q) load_act(warp + GS_WARPS * a, q, bq[a][q]);
+    }
   }
 
   float acc[TILES][NB][4];
@@ -154,40 +165,45 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
   uint32_t phase = 0;
   // shared-memory offset of this lane's 16 bytes in tile row g, first 32-k group (the tile is stored swizzled:
   // 16-byte chunk c of row r sits at chunk position c ^ (r & 7); rows g and g + 8 share g & 7)
-  for (int ch = warp; ch < NCH; ch += GS_WARPS) {
-    // one decision for the whole warp (a bounded wait could run out for some lanes only)
-    if (!__all_sync(0xffffffffu, mbar_wait(my_bars + 8u * slot, phase, nullptr, wait_ns))) { ok = false; break; }
-    inflight &= ~(1u << slot);
-    const uint32_t sbase = my_ring + slot * STAGE_BYTES;
-    const bool more = ch + GS_WARPS < NCH;
+  for (int ch0 = warp; ch0 < NCH && ok; ch0 += GS_WARPS * AD) {
 #pragma unroll
-    for (int q = 0; q < GS_GROUPS; ++q) {
-      const uint32_t off = (uint32_t)((q >> 1) * W_TILE_BYTES + g * 128 + (((4 * (q & 1) + t) ^ g) << 4));
+    for (int a = 0; a < AD; ++a) {
+      const int ch = ch0 + GS_WARPS * a;
+      if (ch >= NCH) break;
+      // one decision for the whole warp (a bounded wait could run out for some lanes only)
+      if (!__all_sync(0xffffffffu, mbar_wait(my_bars + 8u * slot, phase, nullptr, wait_ns))) { ok = false; break; }
+      inflight &= ~(1u << slot);
+      const uint32_t sbase = my_ring + slot * STAGE_BYTES;
+      const bool more = ch + GS_WARPS * AD < NCH;
 #pragma unroll
-      for (int i = 0; i < TILES; ++i) {
-        const uint4 lo = lds128(sbase + i * W_CHUNK_BYTES + off);          // row g:     k 8t .. 8t+7 of the group
-        const uint4 hi = lds128(sbase + i * W_CHUNK_BYTES + off + 1024u);  // row g + 8
+      for (int q = 0; q < GS_GROUPS; ++q) {
+        const uint32_t off = (uint32_t)((q >> 1) * W_TILE_BYTES + g * 128 + (((4 * (q & 1) + t) ^ g) << 4));
 #pragma unroll
-        for (int j = 0; j < NB; ++j) {
-          if (F16) {
-            mma_f16_16816(acc[i][j], lo.x, hi.x, lo.y, hi.y, bq[q][j].x, bq[q][j].y);
-            mma_f16_16816(acc[i][j], lo.z, hi.z, lo.w, hi.w, bq[q][j].z, bq[q][j].w);
-          } else {
-            mma_bf16_16816(acc[i][j], lo.x, hi.x, lo.y, hi.y, bq[q][j].x, bq[q][j].y);
-            mma_bf16_16816(acc[i][j], lo.z, hi.z, lo.w, hi.w, bq[q][j].z, bq[q][j].w);
+        for (int i = 0; i < TILES; ++i) {
+          const uint4 lo = lds128(sbase + i * W_CHUNK_BYTES + off);          // row g:     k 8t .. 8t+7 of the group
+          const uint4 hi = lds128(sbase + i * W_CHUNK_BYTES + off + 1024u);  // row g + 8
+#pragma unroll
+          for (int j = 0; j < NB; ++j) {
+            if (F16) {
+              mma_f16_16816(acc[i][j], lo.x, hi.x, lo.y, hi.y, bq[a][q][j].x, bq[a][q][j].y);
+              mma_f16_16816(acc[i][j], lo.z, hi.z, lo.w, hi.w, bq[a][q][j].z, bq[a][q][j].w);
+            } else {
+              mma_bf16_16816(acc[i][j], lo.x, hi.x, lo.y, hi.y, bq[a][q][j].x, bq[a][q][j].y);
+              mma_bf16_16816(acc[i][j], lo.z, hi.z, lo.w, hi.w, bq[a][q][j].z, bq[a][q][j].w);
+            }
           }
         }
+        if (more) load_act(ch + GS_WARPS * AD, q, bq[a][q]);  // the same group, AD copies further on
       }
-      if (more) load_act(ch + GS_WARPS, q, bq[q]);  // the same group of this warp's next copy
+      // Every shared-memory read above has been consumed by an MMA that is already issued, so after this
+      // warp barrier no lane still reads the slot and lane 0 may hand it back to the copy engine.
+      __syncwarp();
+      if (lane == 0) {
+        const int next = ch + GS_WARPS * S;
+        if (next < NCH) issue_w(next, slot);
+      }
+      if (++slot == S) { slot = 0; phase ^= 1u; }
     }
-    // Every shared-memory read above has been consumed by an MMA that is already issued, so after this
-    // warp barrier no lane still reads the slot and lane 0 may hand it back to the copy engine.
-    __syncwarp();
-    if (lane == 0) {
-      const int next = ch + GS_WARPS * S;
-      if (next < NCH) issue_w(next, slot);
-    }
-    if (++slot == S) { slot = 0; phase ^= 1u; }
   }
   if (!ok) {
     // a copy never landed: record it and let whatever is still in flight arrive (bounded) before leaving, so that
@@ -243,17 +259,17 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
   }
 }
 
-template <int NB, int EPI, int TILES, bool F16>
-int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, void* out, int ldo, cudaStream_t st, bool early) {
+template <int NB, int EPI, int TILES, bool F16, int AD>
+int launch_cfg_ad(const TcAct& act, const TcWeight& w, int M, int N, void* out, int ldo, cudaStream_t st, bool early) {
   static bool configured = false;
   static int num_sms = 0, smem_per_sm = 0;
   constexpr int STAGE_BYTES = TILES * W_CHUNK_BYTES;
   constexpr int MAX_DYN = GS_WARPS * GS_MAX_SLOTS * STAGE_BYTES + 128 > 200 * 1024 ? 200 * 1024
                                                                                      : GS_WARPS * GS_MAX_SLOTS * STAGE_BYTES + 128;
   if (!configured) {
-    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_stream_kernel<NB, EPI, TILES, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN));
+    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_stream_kernel<NB, EPI, TILES, F16, AD>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN));
     // several CTAs per SM share the ring space: ask for the largest shared-memory carve-out
-    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_stream_kernel<NB, EPI, TILES, F16>, cudaFuncAttributePreferredSharedMemoryCarveout,
+    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_stream_kernel<NB, EPI, TILES, F16, AD>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                       cudaSharedmemCarveoutMaxShared));
     int dev = 0;
     HYP_CUDA_TRY(cudaGetDevice(&dev));
@@ -288,14 +304,23 @@ int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, void* out, int
   // the kernel fetches weights before it waits for its predecessor: launched early only when the weights cannot
   // be that predecessor's output
   if (early)
-    HYP_CUDA_TRY(launch_pdl<1>(gemm_stream_kernel<NB, EPI, TILES, F16>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
+    HYP_CUDA_TRY(launch_pdl<1>(gemm_stream_kernel<NB, EPI, TILES, F16, AD>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
                                (const uint8_t*)w.packed, (const uint16_t*)act.ptr, act.K, act.K, N, w.KBp, w.N16p, M, out,
                                ldo, slots, gemm_stream_rotation(), tc_err_flag_ptr(), wait_ns, withhold));
   else
-    HYP_CUDA_TRY(launch_pdl<4>(gemm_stream_kernel<NB, EPI, TILES, F16>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
+    HYP_CUDA_TRY(launch_pdl<4>(gemm_stream_kernel<NB, EPI, TILES, F16, AD>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
                                (const uint8_t*)w.packed, (const uint16_t*)act.ptr, act.K, act.K, N, w.KBp, w.N16p, M, out,
                                ldo, slots, gemm_stream_rotation(), tc_err_flag_ptr(), wait_ns, withhold));
   return 1;
+}
+
+template <int NB, int EPI, int TILES, bool F16>
+int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, void* out, int ldo, cudaStream_t st, bool early) {
+  int ad = 2;  // measured best, see the kernel
+  if (gemm_stream_act_depth() > 0) ad = gemm_stream_act_depth();
+  if (ad >= 3) return launch_cfg_ad<NB, EPI, TILES, F16, 3>(act, w, M, N, out, ldo, st, early);
+  if (ad == 2) return launch_cfg_ad<NB, EPI, TILES, F16, 2>(act, w, M, N, out, ldo, st, early);
+  return launch_cfg_ad<NB, EPI, TILES, F16, 1>(act, w, M, N, out, ldo, st, early);
 }
 
 template <int NB, bool F16>

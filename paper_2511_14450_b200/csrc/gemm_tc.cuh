@@ -70,6 +70,7 @@ int& gemm_stream_rotation();
 // Limit of the weight-streaming kernel's bounded waits in microseconds (0 = the built-in 4 s), and a one-shot hook
 // that makes the next launch of that kernel withhold one copy so that a wait runs into the limit (for the test of
 // the HYP_ETIMEOUT path: no fault, the kernel records the code and returns).
+int& gemm_stream_act_depth();
 int& gemm_stream_wait_limit_us();
 int& gemm_stream_withhold_next();
 // Reads the device word like tc_error_flag and, if `clear`, zeroes it afterwards.
