@@ -340,7 +340,7 @@ int launch_projection(const TcAct& act, const TcWeight& w, int M, int N, int K, 
   const bool store = epi >= 0 && epi < 4 && ((gemm_swap_epilogues() >> epi) & 1);
   if (store && M >= gemm_swap_min_rows() && M <= gemm_swap_max_rows() && (N + 255) / 256 < 100)
     return launch_gemm_swap(act, w, M, N, K, epi, out, ldo, st, early);
-  return launch_gemm_tc(act, w, M, N, K, epi, out, ldo, st, early && M <= 128);
+  return launch_gemm_tc(act, w, M, N, K, epi, out, ldo, st, early);
 }
 
 }  // namespace hyp

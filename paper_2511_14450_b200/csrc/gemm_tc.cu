@@ -236,24 +236,43 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
   if (warp == 0) {
     if (lane == 0) {
       // ---------------- TMA producer ----------------
-      int stage = 0;
+      int stage = 0, issued = 0;
       uint32_t phase = 0;
       bool ok = true;
+      int tile, kb0, kb1;
+      // The weight boxes of the first ring-full of k-blocks go out before the wait for the predecessor (weights are
+      // never written by a kernel); the activation boxes of the same stages follow it.  When this kernel was
+      // launched early, its weights are then on their way while the predecessor drains.
+      {
+        Segments pre(STREAMK, tiles_m, tiles_n, KB, team, (int)blockIdx.x, (int)gridDim.x);
+        int n = 0;
+        while (n < STAGES && pre.next(tile, kb0, kb1)) {
+          const int n0 = (tile / tiles_m) * BN_OUT;
+          const int tb0 = n0 >> 4, tb1 = SWIGLU ? up_tile0 + (n0 >> 4) : (n0 >> 4) + 8;
+          for (int kb = kb0; kb < kb1 && n < STAGES; ++kb, ++n) {
+            const uint32_t sb = base + n * STAGE_BYTES + A_BYTES;
+            mbar_expect_tx(full_bar(n), STAGE_BYTES);
+            tma_load_4d(sb, &tm_b, 0, 0, kb, tb0, full_bar(n));
+            tma_load_4d(sb + B_BYTES / 2, &tm_b, 0, 0, kb, tb1, full_bar(n));
+          }
+        }
+      }
       pdl_wait();  // the activation operand is the predecessor's output
       Segments seg(STREAMK, tiles_m, tiles_n, KB, team, (int)blockIdx.x, (int)gridDim.x);
-      int tile, kb0, kb1;
       while (ok && seg.next(tile, kb0, kb1)) {
         const int m0 = (tile % tiles_m) * BM;
         const int n0 = (tile / tiles_m) * BN_OUT;
         // weight tiles (16 rows each) of the two 128-row boxes: SwiGLU pairs gate rows with the matching up rows
         const int tb0 = n0 >> 4, tb1 = SWIGLU ? up_tile0 + (n0 >> 4) : (n0 >> 4) + 8;
-        for (int kb = kb0; kb < kb1; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) { ok = false; break; }
+        for (int kb = kb0; kb < kb1; ++kb, ++issued) {
           const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
-          mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+          if (issued >= STAGES) {
+            if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) { ok = false; break; }
+            mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+            tma_load_4d(sb, &tm_b, 0, 0, kb, tb0, full_bar(stage));
+            tma_load_4d(sb + B_BYTES / 2, &tm_b, 0, 0, kb, tb1, full_bar(stage));
+          }
           tma_load_2d(sa, &tm_a, kb * BK, m0, full_bar(stage));
-          tma_load_4d(sb, &tm_b, 0, 0, kb, tb0, full_bar(stage));
-          tma_load_4d(sb + B_BYTES / 2, &tm_b, 0, 0, kb, tb1, full_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
       }
@@ -457,24 +476,39 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   if (warp == 0) {
     if (lane == 0) {
       // ---------------- TMA producer (both CTAs) ----------------
-      pdl_wait();
-      int stage = 0;
+      int stage = 0, issued = 0;
       uint32_t phase = 0;
       bool ok = true;
-      Segments seg(STREAMK, pairs_m, tiles_n, KB, team, pair, n_pairs);
       int tile, kb0, kb1;
+      // weight boxes of the first ring-full of k-blocks before the wait for the predecessor, see gemm_tc_kernel
+      {
+        Segments pre(STREAMK, pairs_m, tiles_n, KB, team, pair, n_pairs);
+        int n = 0;
+        while (n < STAGES2 && pre.next(tile, kb0, kb1)) {
+          const int n0 = (tile / pairs_m) * BN_OUT;
+          const int tb = SWIGLU ? (int)rank * up_tile0 + (n0 >> 4) : (n0 >> 4) + (int)rank * (BNT / 32);
+          for (int kb = kb0; kb < kb1 && n < STAGES2; ++kb, ++n) {
+            if (rank == 0) mbar_expect_tx(full_bar(n), 2 * (A_BYTES + B_HALF_BYTES));
+            tma_load_4d_pair(base + n * STAGE2_BYTES + A_BYTES, &tm_b, 0, 0, kb, tb, mapa_rank(full_bar(n), 0));
+          }
+        }
+      }
+      pdl_wait();
+      Segments seg(STREAMK, pairs_m, tiles_n, KB, team, pair, n_pairs);
       while (ok && seg.next(tile, kb0, kb1)) {
         const int m0 = (tile % pairs_m) * (2 * BM) + (int)rank * BM;
         const int n0 = (tile / pairs_m) * BN_OUT;
         // this CTA's half of the weight tile, as an index of 16-row packed tiles
         const int tb = SWIGLU ? (int)rank * up_tile0 + (n0 >> 4) : (n0 >> 4) + (int)rank * (BNT / 32);
-        for (int kb = kb0; kb < kb1; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) { ok = false; break; }
+        for (int kb = kb0; kb < kb1; ++kb, ++issued) {
           const uint32_t sa = base + stage * STAGE2_BYTES, sb = sa + A_BYTES;
           const uint32_t lead_full = mapa_rank(full_bar(stage), 0);
-          if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * (A_BYTES + B_HALF_BYTES));
+          if (issued >= STAGES2) {
+            if (!mbar_wait(empty_bar(stage), phase ^ 1, abort_flag)) { ok = false; break; }
+            if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * (A_BYTES + B_HALF_BYTES));
+            tma_load_4d_pair(sb, &tm_b, 0, 0, kb, tb, lead_full);
+          }
           tma_load_2d_pair(sa, &tm_a, kb * BK, m0, lead_full);
-          tma_load_4d_pair(sb, &tm_b, 0, 0, kb, tb, lead_full);
           if (++stage == STAGES2) { stage = 0; phase ^= 1; }
         }
       }
