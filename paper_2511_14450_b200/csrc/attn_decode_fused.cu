@@ -317,23 +317,42 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
     }
   }
 
-  // merge over the splits: every CTA of the cluster takes a slice of the G x D outputs
+  // merge over the splits: every CTA of the cluster takes a slice of the G x D outputs.  Loads from a peer's shared
+  // memory have a long latency, so none of them may wait for another: first one thread per (head, split) fetches
+  // that split's maximum and denominator into this CTA's own shared memory, then every thread fetches the n_splits
+  // partial outputs of its element in one batch and only then combines them.
   __syncthreads();
   cluster_barrier();
   {
+    __shared__ float all_m[8 * 8], all_l[8 * 8];  // [head][split]
     const uint32_t rank = cluster_rank_x();  // == split
+    const uint32_t a_m = smem_u32(ex_m), a_l = smem_u32(ex_l), a_o = smem_u32(ex_o);
+    if ((int)threadIdx.x < G * n_splits) {
+      const int gq = threadIdx.x / n_splits, sp = threadIdx.x % n_splits;
+      const float mv = ld_cluster_f32(a_m + 4u * gq, sp), lv = ld_cluster_f32(a_l + 4u * gq, sp);
+      all_m[gq * 8 + sp] = mv;
+      all_l[gq * 8 + sp] = lv;
+    }
+    __syncthreads();
     const int per = (G * D + n_splits - 1) / n_splits;
     const int e0 = (int)rank * per, e1 = min(G * D, e0 + per);
-    const uint32_t a_m = smem_u32(ex_m), a_l = smem_u32(ex_l), a_o = smem_u32(ex_o);
     for (int e = e0 + threadIdx.x; e < e1; e += AF_THREADS) {
       const int gq = e / D, dd = e % D;
+      float ov[8];
+#pragma unroll
+      for (int sp = 0; sp < 8; ++sp) ov[sp] = sp < n_splits ? ld_cluster_f32(a_o + 4u * e, sp) : 0.f;
       float mx = AF_NEG;
-      for (int sp = 0; sp < n_splits; ++sp) mx = fmaxf(mx, ld_cluster_f32(a_m + 4u * gq, sp));
+#pragma unroll
+      for (int sp = 0; sp < 8; ++sp)
+        if (sp < n_splits) mx = fmaxf(mx, all_m[gq * 8 + sp]);
       float l = 0.f, acc = 0.f;
-      for (int sp = 0; sp < n_splits; ++sp) {
-        const float wgt = exp2f(ld_cluster_f32(a_m + 4u * gq, sp) - mx);
-        l += wgt * ld_cluster_f32(a_l + 4u * gq, sp);
-        acc += wgt * ld_cluster_f32(a_o + 4u * e, sp);
+#pragma unroll
+      for (int sp = 0; sp < 8; ++sp) {
+        if (sp < n_splits) {
+          const float wgt = exp2f(all_m[gq * 8 + sp] - mx);
+          l += wgt * all_l[gq * 8 + sp];
+          acc += wgt * ov[sp];
+        }
       }
       a.out[((size_t)b * d.Hq + kvh * G + gq) * D + dd] = f16_sat(acc / l);
     }
