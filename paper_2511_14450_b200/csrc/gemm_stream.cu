@@ -34,6 +34,10 @@ int& gemm_stream_act_depth() {  // copies ahead that a warp's activation fragmen
   static int v = 0;
   return v;
 }
+int& gemm_stream_act_tma() {  // 1 (default): activations ride into the ring by TMA where the operand allows it
+  static int v = 1;
+  return v;
+}
 int& gemm_stream_wait_limit_us() {
   static int v = 0;
   return v;
@@ -72,20 +76,27 @@ __device__ __forceinline__ uint4 ldg_act(const void* p) {
 // iteration; with the fragments of only the next copy in flight an iteration cannot be shorter than one L2 round
 // trip.  Measured on the 14-block decode stage (batch 8, us per step): AD 1: 1837, AD 2: 1818, AD 3: 1830 (the
 // registers of the third copy cost more than its latency cover gives).
-template <int NB, int EPI, int TILES, bool F16, int AD>
+// ATMA: the activations of a copy's k range (8 token rows x 128 k, 2 KB) ride into the same ring slot by one TMA box
+// load (tensor map {64 k, rows, K / 64}, box {64, 8, 2}, 128-byte swizzle) instead of per-lane global loads.  Measured
+// with the loads taken out, the one-strip projections spend 19-29 % of their loop time on those loads (they
+// queue in the load/store unit, 12 warps x 4 x 512 bytes per copy round; a deeper register prefetch does not help),
+// and only without them does a warp wait for HBM rather than for its own instructions.  Needs K % 64 == 0.
+template <int NB, int EPI, int TILES, bool F16, int AD, bool ATMA>
 __global__ void __launch_bounds__(GS_THREADS, 3)
 gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ act, int lda, int K, int N, int KBp,
                    int tile1_off, int M, void* __restrict__ out, int ldo, int S, int rot_mul, int* __restrict__ err,
-                   uint64_t wait_ns, int withhold) {
+                   uint64_t wait_ns, int withhold, const __grid_constant__ CUtensorMap tm_act) {
   constexpr bool SWIGLU = EPI == EPI_SWIGLU_BF16;
   static_assert(!SWIGLU || TILES == 2, "SwiGLU pairs a gate strip with an up strip");
   constexpr int OUT_COLS = (TILES == 2 && !SWIGLU) ? 32 : 16;
-  constexpr int STAGE_BYTES = TILES * W_CHUNK_BYTES;
+  constexpr int ACT_BYTES = ATMA ? GS_CHUNK_K * 8 * 2 : 0;  // 8 token rows of the copy's k range
+  constexpr int STAGE_BYTES = TILES * W_CHUNK_BYTES + ACT_BYTES;
   constexpr int RED_LD = NB * 8 + 1;
   static_assert(16 * TILES * RED_LD * 4 <= 2 * STAGE_BYTES, "a warp's partial sums reuse its own ring space");
+  static_assert(!ATMA || NB == 1, "the activation box holds one group of 8 tokens");
   extern __shared__ uint8_t gs_smem_raw[];
   __shared__ uint64_t bars[GS_WARPS * GS_MAX_SLOTS];
-  const uint32_t base = (smem_u32(gs_smem_raw) + 127u) & ~127u;
+  const uint32_t base = (smem_u32(gs_smem_raw) + 1023u) & ~1023u;  // the activation boxes are 128-byte swizzled
   uint8_t* base_ptr = gs_smem_raw + (base - smem_u32(gs_smem_raw));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -117,10 +128,22 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
     if (TILES == 2) bulk_load(dst + W_CHUNK_BYTES, w1 + (size_t)ch * W_CHUNK_BYTES, W_CHUNK_BYTES, bar);
   };
 
+  // activations of the same copy (the predecessor's output: only after the wait for it)
+  auto issue_a = [&](int ch_logical, int slot) {
+    if (ATMA) {
+      const uint32_t dst = my_ring + slot * STAGE_BYTES + TILES * W_CHUNK_BYTES, bar = my_bars + 8u * slot;
+      asm volatile(
+          "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+          ::"r"(dst), "l"(&tm_act), "r"(bar), "r"(0), "r"(0), "r"(actual(ch_logical) * GS_CH)
+          : "memory");
+    }
+  };
+
   // Every CTA of this grid is resident by the time the last one gets here, so the successor may be scheduled
   // into whatever room is left: it only sets up and prefetches until this grid has completed.
   pdl_trigger();
   if (lane == 0) {
+    if (ATMA) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_act) : "memory");
     for (int sl = 0; sl < S; ++sl) mbar_init(my_bars + 8u * sl, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     // `withhold` (a test hook, see launch_cfg): warp 0 of CTA 0 never asks for its first copy, so its first
@@ -146,19 +169,31 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
       dst[j] = (avalid[j] && k + 8 * t < K) ? ldg_act(arow[j] + k) : make_uint4(0u, 0u, 0u, 0u);
   };
   pdl_wait();  // activations (and, for the residual epilogue, the output) belong to the predecessor until here
+  if (ATMA) {
+    if (lane == 0)
+      for (int sl = 0; sl < S; ++sl)
+        if (warp + GS_WARPS * sl < NCH && !(withhold && blockIdx.x == 0 && warp == 0 && sl == 0)) issue_a(warp + GS_WARPS * sl, sl);
+  } else {
 #pragma unroll
-  for (int a = 0; a < AD; ++a) {
-    if (warp + GS_WARPS * a < NCH) {
+    for (int a = 0; a < AD; ++a) {
+      if (warp + GS_WARPS * a < NCH) {
 #pragma unroll
-      for (int q = 0; q < GS_GROUPS; ++q) load_act(warp + GS_WARPS * a, q, bq[a][q]);
+        for (int q = 0; q < GS_GROUPS; ++q) load_act(warp + GS_WARPS * a, q, bq[a][q]);
+      }
     }
   }
 
-  float acc[TILES][NB][4];
+  // CH independent accumulator chains per output fragment: the MMAs of one copy would otherwise form one chain of
+  // eight dependent instructions, and the one-strip kernels then spend their time in that chain's latency instead
+  // of waiting for HBM (measured: 8 % of a warp's loop time waiting for copies against 42 % in the two-strip grid)
+  constexpr int CH = TILES == 1 ? GS_GROUPS : 2;
+  float acc[CH][TILES][NB][4];
 #pragma unroll
-  for (int i = 0; i < TILES; ++i)
+  for (int c = 0; c < CH; ++c)
 #pragma unroll
-    for (int j = 0; j < NB; ++j) acc[i][j][0] = acc[i][j][1] = acc[i][j][2] = acc[i][j][3] = 0.f;
+    for (int i = 0; i < TILES; ++i)
+#pragma unroll
+      for (int j = 0; j < NB; ++j) acc[c][i][j][0] = acc[c][i][j][1] = acc[c][i][j][2] = acc[c][i][j][3] = 0.f;
 
   bool ok = true;
   int slot = 0;
@@ -178,6 +213,8 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
 #pragma unroll
       for (int q = 0; q < GS_GROUPS; ++q) {
         const uint32_t off = (uint32_t)((q >> 1) * W_TILE_BYTES + g * 128 + (((4 * (q & 1) + t) ^ g) << 4));
+        if (ATMA)  // token g, k 8t .. 8t+7 of the group: the box keeps the weight tiles' chunk permutation
+          bq[a][q][0] = lds128(sbase + TILES * W_CHUNK_BYTES + (uint32_t)((q >> 1) * 1024 + g * 128 + (((4 * (q & 1) + t) ^ g) << 4)));
 #pragma unroll
         for (int i = 0; i < TILES; ++i) {
           const uint4 lo = lds128(sbase + i * W_CHUNK_BYTES + off);          // row g:     k 8t .. 8t+7 of the group
@@ -185,22 +222,25 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
 #pragma unroll
           for (int j = 0; j < NB; ++j) {
             if (F16) {
-              mma_f16_16816(acc[i][j], lo.x, hi.x, lo.y, hi.y, bq[a][q][j].x, bq[a][q][j].y);
-              mma_f16_16816(acc[i][j], lo.z, hi.z, lo.w, hi.w, bq[a][q][j].z, bq[a][q][j].w);
+              mma_f16_16816(acc[q % CH][i][j], lo.x, hi.x, lo.y, hi.y, bq[a][q][j].x, bq[a][q][j].y);
+              mma_f16_16816(acc[q % CH][i][j], lo.z, hi.z, lo.w, hi.w, bq[a][q][j].z, bq[a][q][j].w);
             } else {
-              mma_bf16_16816(acc[i][j], lo.x, hi.x, lo.y, hi.y, bq[a][q][j].x, bq[a][q][j].y);
-              mma_bf16_16816(acc[i][j], lo.z, hi.z, lo.w, hi.w, bq[a][q][j].z, bq[a][q][j].w);
+              mma_bf16_16816(acc[q % CH][i][j], lo.x, hi.x, lo.y, hi.y, bq[a][q][j].x, bq[a][q][j].y);
+              mma_bf16_16816(acc[q % CH][i][j], lo.z, hi.z, lo.w, hi.w, bq[a][q][j].z, bq[a][q][j].w);
             }
           }
         }
-        if (more) load_act(ch + GS_WARPS * AD, q, bq[a][q]);  // the same group, AD copies further on
+        if (!ATMA && more) load_act(ch + GS_WARPS * AD, q, bq[a][q]);  // the same group, AD copies further on
       }
       // Every shared-memory read above has been consumed by an MMA that is already issued, so after this
       // warp barrier no lane still reads the slot and lane 0 may hand it back to the copy engine.
       __syncwarp();
       if (lane == 0) {
         const int next = ch + GS_WARPS * S;
-        if (next < NCH) issue_w(next, slot);
+        if (next < NCH) {
+          issue_w(next, slot);
+          issue_a(next, slot);
+        }
       }
       if (++slot == S) { slot = 0; phase ^= 1u; }
     }
@@ -225,10 +265,15 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
     for (int i = 0; i < TILES; ++i)
 #pragma unroll
       for (int j = 0; j < NB; ++j) {
-        mine[(16 * i + g) * RED_LD + 8 * j + 2 * t] = acc[i][j][0];
-        mine[(16 * i + g) * RED_LD + 8 * j + 2 * t + 1] = acc[i][j][1];
-        mine[(16 * i + g + 8) * RED_LD + 8 * j + 2 * t] = acc[i][j][2];
-        mine[(16 * i + g + 8) * RED_LD + 8 * j + 2 * t + 1] = acc[i][j][3];
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {  // the chains in a fixed order
+          v[0] += acc[c][i][j][0]; v[1] += acc[c][i][j][1]; v[2] += acc[c][i][j][2]; v[3] += acc[c][i][j][3];
+        }
+        mine[(16 * i + g) * RED_LD + 8 * j + 2 * t] = v[0];
+        mine[(16 * i + g) * RED_LD + 8 * j + 2 * t + 1] = v[1];
+        mine[(16 * i + g + 8) * RED_LD + 8 * j + 2 * t] = v[2];
+        mine[(16 * i + g + 8) * RED_LD + 8 * j + 2 * t + 1] = v[3];
       }
   }
   __syncthreads();
@@ -259,17 +304,17 @@ gemm_stream_kernel(const uint8_t* __restrict__ wp, const uint16_t* __restrict__ 
   }
 }
 
-template <int NB, int EPI, int TILES, bool F16, int AD>
+template <int NB, int EPI, int TILES, bool F16, int AD, bool ATMA>
 int launch_cfg_ad(const TcAct& act, const TcWeight& w, int M, int N, void* out, int ldo, cudaStream_t st, bool early) {
   static bool configured = false;
   static int num_sms = 0, smem_per_sm = 0;
-  constexpr int STAGE_BYTES = TILES * W_CHUNK_BYTES;
-  constexpr int MAX_DYN = GS_WARPS * GS_MAX_SLOTS * STAGE_BYTES + 128 > 200 * 1024 ? 200 * 1024
-                                                                                     : GS_WARPS * GS_MAX_SLOTS * STAGE_BYTES + 128;
+  constexpr int STAGE_BYTES = TILES * W_CHUNK_BYTES + (ATMA ? GS_CHUNK_K * 8 * 2 : 0);
+  constexpr int MAX_DYN = GS_WARPS * GS_MAX_SLOTS * STAGE_BYTES + 1024 > 200 * 1024 ? 200 * 1024
+                                                                                      : GS_WARPS * GS_MAX_SLOTS * STAGE_BYTES + 1024;
   if (!configured) {
-    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_stream_kernel<NB, EPI, TILES, F16, AD>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN));
+    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_stream_kernel<NB, EPI, TILES, F16, AD, ATMA>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN));
     // several CTAs per SM share the ring space: ask for the largest shared-memory carve-out
-    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_stream_kernel<NB, EPI, TILES, F16, AD>, cudaFuncAttributePreferredSharedMemoryCarveout,
+    HYP_CUDA_TRY(cudaFuncSetAttribute(gemm_stream_kernel<NB, EPI, TILES, F16, AD, ATMA>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                       cudaSharedmemCarveoutMaxShared));
     int dev = 0;
     HYP_CUDA_TRY(cudaGetDevice(&dev));
@@ -289,13 +334,13 @@ int launch_cfg_ad(const TcAct& act, const TcWeight& w, int M, int N, void* out, 
   // CTAs per SM hide each other's start and end).  1 KB per CTA is reserved by the driver; 512 B cover barriers
   // and alignment.
   const int per_sm = (n_ctas + num_sms - 1) / num_sms;
-  int slots = (smem_per_sm / per_sm - 1024 - 512) / (GS_WARPS * STAGE_BYTES);
+  int slots = (smem_per_sm / per_sm - 1024 - 1024 - 384) / (GS_WARPS * STAGE_BYTES);
   if (slots > GS_MAX_SLOTS) slots = GS_MAX_SLOTS;
   if (slots < 2) slots = 2;
   if (gemm_stream_slots_override() > 0) slots = gemm_stream_slots_override();
   if (slots > GS_MAX_SLOTS) slots = GS_MAX_SLOTS;
-  while (slots > 2 && GS_WARPS * slots * STAGE_BYTES + 128 > MAX_DYN) --slots;
-  const int smem = GS_WARPS * slots * STAGE_BYTES + 128;
+  while (slots > 2 && GS_WARPS * slots * STAGE_BYTES + 1024 > MAX_DYN) --slots;
+  const int smem = GS_WARPS * slots * STAGE_BYTES + 1024;
   // bounded waits: 4 s unless a shorter limit was set (hyp_tune); `withhold` is a one-shot test hook that makes
   // one wait of the next launch run into that limit (nothing faults: the kernel records the code and returns)
   const uint64_t wait_ns = gemm_stream_wait_limit_us() > 0 ? (uint64_t)gemm_stream_wait_limit_us() * 1000ull : WAIT_LIMIT_NS;
@@ -304,23 +349,25 @@ int launch_cfg_ad(const TcAct& act, const TcWeight& w, int M, int N, void* out, 
   // the kernel fetches weights before it waits for its predecessor: launched early only when the weights cannot
   // be that predecessor's output
   if (early)
-    HYP_CUDA_TRY(launch_pdl<1>(gemm_stream_kernel<NB, EPI, TILES, F16, AD>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
+    HYP_CUDA_TRY(launch_pdl<1>(gemm_stream_kernel<NB, EPI, TILES, F16, AD, ATMA>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
                                (const uint8_t*)w.packed, (const uint16_t*)act.ptr, act.K, act.K, N, w.KBp, w.N16p, M, out,
-                               ldo, slots, gemm_stream_rotation(), tc_err_flag_ptr(), wait_ns, withhold));
+                               ldo, slots, gemm_stream_rotation(), tc_err_flag_ptr(), wait_ns, withhold, act.map_a8));
   else
-    HYP_CUDA_TRY(launch_pdl<4>(gemm_stream_kernel<NB, EPI, TILES, F16, AD>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
+    HYP_CUDA_TRY(launch_pdl<4>(gemm_stream_kernel<NB, EPI, TILES, F16, AD, ATMA>, dim3(n_ctas), dim3(GS_THREADS), (size_t)smem, st,
                                (const uint8_t*)w.packed, (const uint16_t*)act.ptr, act.K, act.K, N, w.KBp, w.N16p, M, out,
-                               ldo, slots, gemm_stream_rotation(), tc_err_flag_ptr(), wait_ns, withhold));
+                               ldo, slots, gemm_stream_rotation(), tc_err_flag_ptr(), wait_ns, withhold, act.map_a8));
   return 1;
 }
 
 template <int NB, int EPI, int TILES, bool F16>
 int launch_cfg(const TcAct& act, const TcWeight& w, int M, int N, void* out, int ldo, cudaStream_t st, bool early) {
+  // activations by TMA into the ring whenever the operand has the tensor map for it (K a multiple of 64)
+  if (act.has_a8 && gemm_stream_act_tma()) return launch_cfg_ad<NB, EPI, TILES, F16, 1, true>(act, w, M, N, out, ldo, st, early);
   int ad = 2;  // measured best, see the kernel
   if (gemm_stream_act_depth() > 0) ad = gemm_stream_act_depth();
-  if (ad >= 3) return launch_cfg_ad<NB, EPI, TILES, F16, 3>(act, w, M, N, out, ldo, st, early);
-  if (ad == 2) return launch_cfg_ad<NB, EPI, TILES, F16, 2>(act, w, M, N, out, ldo, st, early);
-  return launch_cfg_ad<NB, EPI, TILES, F16, 1>(act, w, M, N, out, ldo, st, early);
+  if (ad >= 3) return launch_cfg_ad<NB, EPI, TILES, F16, 3, false>(act, w, M, N, out, ldo, st, early);
+  if (ad == 2) return launch_cfg_ad<NB, EPI, TILES, F16, 2, false>(act, w, M, N, out, ldo, st, early);
+  return launch_cfg_ad<NB, EPI, TILES, F16, 1, false>(act, w, M, N, out, ldo, st, early);
 }
 
 template <int NB, bool F16>

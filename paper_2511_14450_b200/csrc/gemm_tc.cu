@@ -853,6 +853,18 @@ int tc_make_act(TcAct* a, const void* ptr, int rows, int K, bool f16) {
   a->ptr = ptr; a->rows = rows; a->K = K; a->f16 = f16;
   int rc = encode_map(&a->map, ptr, rows, K, 128, f16);
   for (int i = 0; i < 3 && !rc; ++i) rc = encode_map(&a->map_small[i], ptr, rows, K, 16 << i, f16);
+  a->has_a8 = false;
+  if (!rc && K % 64 == 0) {
+    EncodeTiledFn enc = encode_fn();
+    const cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(K / 64)};
+    const cuuint64_t strides[2] = {(cuuint64_t)K * 2, 128};
+    const cuuint32_t box[3] = {64, 8, 2};
+    const cuuint32_t estr[3] = {1u, 1u, 1u};
+    CUresult r = enc(&a->map_a8, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)ptr, dims,
+                     strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    a->has_a8 = r == CUDA_SUCCESS;  // without it the streaming kernel reads its fragments from global memory
+  }
   return rc;
 }
 

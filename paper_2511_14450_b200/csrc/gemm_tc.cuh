@@ -41,6 +41,10 @@ struct TcAct {
   int rows = 0, K = 0;
   bool f16 = false;
   CUtensorMap map_small[3];  // boxes of 16, 32, 64 rows (swapped-operand kernel: the tokens are the N operand)
+  // {64 k, rows, K / 64} view with boxes of 64 k x 8 rows x 2 k-blocks (weight-streaming kernel: the activations of
+  // one 128-k copy, 2 KB); only when K is a multiple of 64
+  CUtensorMap map_a8;
+  bool has_a8 = false;
 };
 int tc_make_act(TcAct* a, const void* ptr, int rows, int K, bool f16 = false);
 
@@ -71,6 +75,7 @@ int& gemm_stream_rotation();
 // that makes the next launch of that kernel withhold one copy so that a wait runs into the limit (for the test of
 // the HYP_ETIMEOUT path: no fault, the kernel records the code and returns).
 int& gemm_stream_act_depth();
+int& gemm_stream_act_tma();
 int& gemm_stream_wait_limit_us();
 int& gemm_stream_withhold_next();
 // Reads the device word like tc_error_flag and, if `clear`, zeroes it afterwards.

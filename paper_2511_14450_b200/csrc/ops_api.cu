@@ -104,6 +104,9 @@ extern "C" int hyp_tune(int32_t key, int32_t value) {
       if (value < 0 || value > 8) return HYP_EINVAL;
       attn_fused_splits_override() = value;
       return HYP_OK;
+    case HYP_TUNE_STREAM_ACT_TMA:
+      gemm_stream_act_tma() = value != 0;
+      return HYP_OK;
     case HYP_TUNE_STREAM_ACT_DEPTH:
       if (value < 0 || value > 3) return HYP_EINVAL;
       gemm_stream_act_depth() = value;
