@@ -110,6 +110,10 @@ HYP_API int hyp_device_wait_status(int32_t* code_out, int32_t clear);
  *   HYP_TUNE_STREAM_ACT_TMA  value != 0 (the default): the weight-streaming kernel brings the activations of every weight
  *                          copy's k range into its ring by a TMA box load (when K is a multiple of 64); 0: each
  *                          lane reads its fragment entries from global memory
+ *   HYP_TUNE_ATTN_GLOBAL_MERGE  value != 0 (the default): the stage's decode attention merges its context splits through
+ *                          a scratch row per split in global memory (the CTA that finishes last merges) and is
+ *                          launched early; 0: the splits form a thread-block cluster and merge through distributed
+ *                          shared memory (what hyp_op_attn_decode_fused always does)
  *   HYP_TUNE_STREAM_ACT_DEPTH  how many of its weight copies ahead a warp of the weight-streaming kernel fetches its
  *                          activation fragments, 1..3 (0 = built-in: 2)
  *   HYP_TUNE_WAIT_LIMIT_US  limit of the weight-streaming kernel's bounded waits in microseconds (0 = the built-in
@@ -122,7 +126,8 @@ HYP_API int hyp_device_wait_status(int32_t* code_out, int32_t clear);
 enum { HYP_TUNE_PDL = 0, HYP_TUNE_STREAM_SLOTS = 1, HYP_TUNE_ATTN_SPLITS = 2, HYP_TUNE_ATTN_SLOTS = 3,
        HYP_TUNE_STREAM_ROTATION = 4, HYP_TUNE_SWAP_MIN_ROWS = 5, HYP_TUNE_SWAP_MAX_ROWS = 6, HYP_TUNE_SWAP_EPILOGUES = 7,
        HYP_TUNE_PREFILL_ATTN_TC = 8, HYP_TUNE_FIRST_BLOCK_SPLIT = 9, HYP_TUNE_TILE_224 = 10,
-       HYP_TUNE_WAIT_LIMIT_US = 11, HYP_TUNE_STREAM_WITHHOLD_COPY = 12, HYP_TUNE_STREAM_ACT_DEPTH = 13, HYP_TUNE_STREAM_ACT_TMA = 14 };
+       HYP_TUNE_WAIT_LIMIT_US = 11, HYP_TUNE_STREAM_WITHHOLD_COPY = 12, HYP_TUNE_STREAM_ACT_DEPTH = 13, HYP_TUNE_STREAM_ACT_TMA = 14,
+       HYP_TUNE_ATTN_GLOBAL_MERGE = 15 };
 HYP_API int hyp_tune(int32_t key, int32_t value);
 
 /* Number of context splits hyp_op_attn_decode would pick for this batch, and the scratch bytes

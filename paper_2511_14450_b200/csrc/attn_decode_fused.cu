@@ -2,9 +2,8 @@
 // rotary encoding of the new token's query and key, append of its key / value to the paged cache,
 // split-context attention, and the merge of the splits.
 //
-//   grid (n_splits, Hkv, n_seqs), 4 warps, the n_splits CTAs of one (sequence, KV head) form a thread-block
-//   cluster.  Page p of a sequence belongs to split p % n_splits; warp w takes every fourth page of its split and streams
-//   them through its own ring: one bulk copy brings the 16 keys of a page for this KV head (contiguous in the
+//   grid (n_splits, Hkv, n_seqs), 4 warps.  Page p of a sequence belongs to split p % n_splits; warp w takes every
+//   fourth page of its split and streams them through its own ring: one bulk copy brings the 16 keys of a page for this KV head (contiguous in the
 //   cache, already chunk-permuted for ldmatrix), another the 16 values; the warp waits on the slot's mbarrier,
 //   forms the scores of its 16 keys for the G = Hq/Hkv query heads (rows of one mma.sync.m16n8k16 operand, rows
 //   >= G are padding), keeps its own online-softmax state and O += P V partial, and lane 0 refills the slot.
@@ -13,9 +12,15 @@
 //   CTA rotates its G query heads from the projection's fp32 output into shared memory, and the CTA whose run
 //   ends with the new token rotates that token's key, rounds key and value to fp16, writes them to the page
 //   (for the following steps) and, once that page has landed in its ring, over the stale row in shared memory.
-//   Epilogue: the four warps are combined in shared memory; after a cluster barrier every CTA merges a slice of
-//   the G x D outputs over all splits, reading the other CTAs' partials through distributed shared memory.
-//   No global scratch, no atomics.  Every mbarrier wait is bounded; the cluster barriers are reached by every CTA.
+//   Epilogue: the four warps are combined in shared memory; then the splits are merged, in one of two ways.
+//   Cluster variant (the op-level entry point: no scratch memory, no atomics): the n_splits CTAs form a thread-block
+//   cluster; after a cluster barrier every CTA merges a slice of the G x D outputs over all splits, reading the
+//   other CTAs' partials through distributed shared memory.  Global variant (the stage path): every CTA writes its
+//   partial to a scratch row and takes a ticket; the CTA with the last ticket merges.  A cluster's CTAs must be
+//   co-scheduled, which made an early (programmatic) launch of the cluster variant slower than a plain one; the
+//   global variant is launched early, so its CTAs move in as the q/k/v projection's CTAs leave and have their first
+//   pages on the way before the projection has finished (14-block decode step, batch 8: 1784 -> 1768 us).
+//   Every mbarrier wait is bounded; the cluster barriers are reached by every CTA; nothing waits for another CTA.
 #include "attn_common.cuh"
 #include "hyperion.h"
 #include "sm100_common.cuh"
@@ -43,10 +48,18 @@ struct AttnFusedArgs {
   // ([page][Hkv][16][D], the cache's row order), so that the scores carry ~21 significant bits
   const float* row_scale;
   __half* klo_layer;
+  // GLOBAL instantiation only: the splits meet in global memory instead of a cluster's shared memory
+  float* scratch;            // [n_seqs * Hkv][n_splits][G * D + 16] partial outputs, then maxima and denominators
+  int* tickets;              // [n_seqs * Hkv], zero between launches
 };
 
 __device__ __forceinline__ __half f16_sat(float x) { return __float2half_rn(fminf(fmaxf(x, -65504.f), 65504.f)); }
-template <int D, int G, bool SPLIT>
+// GLOBAL: no cluster.  Every CTA writes its partial (G x D sums, G maxima, G denominators) to a scratch row, fences,
+// and takes a ticket on the (sequence, KV head)'s counter; the CTA that takes the last ticket reads the n_splits
+// rows back (L2) and merges them.  Nothing waits for another CTA, and without the co-scheduling that a cluster
+// needs the grid can be launched early (programmatic dependent launch): its CTAs take the SMs' slots as the
+// projection's CTAs leave them and have their first pages on the way before the projection has finished.
+template <int D, int G, bool SPLIT, bool GLOBAL>
 __global__ void __launch_bounds__(AF_THREADS)
 attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
   constexpr int KS = D / 16, DN = D / 8, CPR = D / 8;
@@ -317,6 +330,66 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
     }
   }
 
+  if (GLOBAL) {
+    __shared__ int last_flag;
+    __shared__ float all_m[8 * 8], all_l[8 * 8];  // [head][split]
+    constexpr int ROW = G * D + 16;
+    const int group = b * d.Hkv + kvh;
+    float* grp = a.scratch + (size_t)group * n_splits * ROW;
+    __syncthreads();  // ex_o, ex_m, ex_l are complete
+    float* mine = grp + (size_t)split * ROW;
+    for (int e = threadIdx.x * 4; e < G * D; e += AF_THREADS * 4)
+      __stcg(reinterpret_cast<float4*>(mine + e), *reinterpret_cast<const float4*>(ex_o + e));
+    if ((int)threadIdx.x < G) {
+      __stcg(mine + G * D + threadIdx.x, ex_m[threadIdx.x]);
+      __stcg(mine + G * D + 8 + threadIdx.x, ex_l[threadIdx.x]);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      const int t = atomicAdd(a.tickets + group, 1);
+      last_flag = t == n_splits - 1;
+      if (last_flag) a.tickets[group] = 0;  // for the next launch (it starts after this grid has completed)
+    }
+    __syncthreads();
+    if (!last_flag) return;
+    __threadfence();
+    if ((int)threadIdx.x < G * n_splits) {
+      const int gq = threadIdx.x / n_splits, sp = threadIdx.x % n_splits;
+      all_m[gq * 8 + sp] = sp == split ? ex_m[gq] : __ldcg(grp + (size_t)sp * ROW + G * D + gq);
+      all_l[gq * 8 + sp] = sp == split ? ex_l[gq] : __ldcg(grp + (size_t)sp * ROW + G * D + 8 + gq);
+    }
+    __syncthreads();
+    // every thread fetches the n_splits partial sums of its four outputs in one batch, then combines them
+    for (int e = threadIdx.x * 4; e < G * D; e += AF_THREADS * 4) {
+      const int gq = e / D, dd = e % D;
+      float4 ov[8];
+#pragma unroll
+      for (int sp = 0; sp < 8; ++sp)
+        ov[sp] = sp < n_splits ? __ldcg(reinterpret_cast<const float4*>(grp + (size_t)sp * ROW + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      float mx = AF_NEG;
+#pragma unroll
+      for (int sp = 0; sp < 8; ++sp)
+        if (sp < n_splits) mx = fmaxf(mx, all_m[gq * 8 + sp]);
+      float l = 0.f;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int sp = 0; sp < 8; ++sp) {
+        if (sp < n_splits) {
+          const float wgt = exp2f(all_m[gq * 8 + sp] - mx);
+          l += wgt * all_l[gq * 8 + sp];
+          acc.x += wgt * ov[sp].x; acc.y += wgt * ov[sp].y; acc.z += wgt * ov[sp].z; acc.w += wgt * ov[sp].w;
+        }
+      }
+      __half* op = a.out + ((size_t)b * d.Hq + kvh * G + gq) * D + dd;
+      uint2 pk;  // the same quotient as the cluster variant forms: both variants give the same bits
+      pk.x = pack_f16_sat(acc.x / l, acc.y / l);
+      pk.y = pack_f16_sat(acc.z / l, acc.w / l);
+      *reinterpret_cast<uint2*>(op) = pk;
+    }
+    return;
+  }
+
   // merge over the splits: every CTA of the cluster takes a slice of the G x D outputs.  Loads from a peer's shared
   // memory have a long latency, so none of them may wait for another: first one thread per (head, split) fetches
   // that split's maximum and denominator into this CTA's own shared memory, then every thread fetches the n_splits
@@ -361,7 +434,7 @@ attn_decode_fused_kernel(AttnFusedArgs a, BatchMeta bm, ModelDims d) {
   cluster_barrier();  // nobody leaves while a peer may still read its partial
 }
 
-template <int D, int G, bool SPLIT>
+template <int D, int G, bool SPLIT, bool GLOBAL>
 int launch_dg(const AttnFusedArgs& a_in, int n_splits, const BatchMeta& bm, const ModelDims& d, cudaStream_t st) {
   static bool configured = false;
   constexpr int SLOT_BYTES = (SPLIT ? 3 : 2) * AF_PT * D * 2;
@@ -369,7 +442,7 @@ int launch_dg(const AttnFusedArgs& a_in, int n_splits, const BatchMeta& bm, cons
   constexpr int MAX_DYN = AF_WARPS * AF_MAX_SLOTS * SLOT_BYTES + 128;
   static_assert(AF_WARPS * 2 * SLOT_BYTES >= COMBINE_BYTES, "the combine buffers reuse the ring");
   if (!configured) {
-    HYP_CUDA_TRY(cudaFuncSetAttribute(attn_decode_fused_kernel<D, G, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN));
+    HYP_CUDA_TRY(cudaFuncSetAttribute(attn_decode_fused_kernel<D, G, SPLIT, GLOBAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_DYN));
     configured = true;
   }
   AttnFusedArgs a = a_in;
@@ -383,15 +456,22 @@ int launch_dg(const AttnFusedArgs& a_in, int n_splits, const BatchMeta& bm, cons
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = n_splits;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[1].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = pdl_level() >= 3 ? 2 : 1;  // measured: launching it early at level 2 costs 2 %
-  HYP_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_decode_fused_kernel<D, G, SPLIT>, a, bm, d));
+  if (GLOBAL) {
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_level() >= 2 ? 1 : 0;
+  } else {
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = n_splits;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_level() >= 3 ? 2 : 1;  // measured: launching the cluster variant early costs 2 %
+  }
+  HYP_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_decode_fused_kernel<D, G, SPLIT, GLOBAL>, a, bm, d));
   return 1;
 }
 
@@ -402,6 +482,10 @@ int& attn_fused_splits_override() {
   return v;
 }
 int& first_block_split() {
+  static int v = 1;
+  return v;
+}
+int& attn_global_merge() {
   static int v = 1;
   return v;
 }
@@ -424,15 +508,20 @@ int attn_decode_fused_splits(int n_seqs, int Hkv, int max_ctx) {
 
 int launch_attn_decode_fused(const float* qkv32, int stride, __half* kv_layer, const float2* rope_table, __half* attn_out,
                              int n_splits, int slots, int* err, const BatchMeta& bm, const ModelDims& d, cudaStream_t st,
-                             const float* row_scale, __half* klo_layer) {
+                             const float* row_scale, __half* klo_layer, float* scratch, int* tickets) {
   if (n_splits < 1 || n_splits > 8 || !err || (row_scale != nullptr) != (klo_layer != nullptr)) return HYP_EINVAL;
+  if ((scratch != nullptr) != (tickets != nullptr)) return HYP_EINVAL;
   AttnFusedArgs a;
   a.qkv32 = qkv32; a.stride = stride; a.kv_layer = kv_layer; a.rope_table = rope_table; a.out = attn_out;
   a.slots = slots; a.err = err; a.row_scale = row_scale; a.klo_layer = klo_layer;
+  a.scratch = scratch; a.tickets = tickets;
   const int G = d.Hq / d.Hkv;
 #define HYP_AF_CASE(DD, GG)                                                \
   if (d.D == DD && G == GG)                                                \
-    return row_scale ? launch_dg<DD, GG, true>(a, n_splits, bm, d, st) : launch_dg<DD, GG, false>(a, n_splits, bm, d, st);
+    return scratch ? (row_scale ? launch_dg<DD, GG, true, true>(a, n_splits, bm, d, st)                            \
+                                : launch_dg<DD, GG, false, true>(a, n_splits, bm, d, st))                          \
+                   : (row_scale ? launch_dg<DD, GG, true, false>(a, n_splits, bm, d, st)                           \
+                                : launch_dg<DD, GG, false, false>(a, n_splits, bm, d, st));
   HYP_AF_CASE(128, 1) HYP_AF_CASE(128, 2) HYP_AF_CASE(128, 4) HYP_AF_CASE(128, 8)
   HYP_AF_CASE(64, 1) HYP_AF_CASE(64, 2) HYP_AF_CASE(64, 4) HYP_AF_CASE(64, 8)
 #undef HYP_AF_CASE

@@ -187,6 +187,7 @@ int launch_attn_decode(const __half* q, int q_stride, const __half* kv_layer, __
 // projection output, one row per sequence), appends k, v to the pages, attends over n_splits context slices
 // (a thread-block cluster, n_splits <= 8) and merges them.  `err`: device word set if a bounded wait expires.
 int attn_decode_fused_splits(int n_seqs, int Hkv, int max_ctx);
+int& attn_global_merge();           // 1 (default): the stage's decode attention merges its splits through global memory
 int& first_block_split();           // 1 (default): the model's first block keeps two-term queries / keys
 int& attn_fused_splits_override();  // 0 = built-in choice
 int& attn_fused_slots_override();   // 0 = built-in choice
@@ -194,6 +195,10 @@ int& attn_fused_slots_override();   // 0 = built-in choice
 // first, and queries / keys are two-term fp16 values (the keys' low terms cached in klo_layer [page][Hkv][16][D]).
 int launch_attn_decode_fused(const float* qkv32, int stride, __half* kv_layer, const float2* rope_table, __half* attn_out,
                              int n_splits, int slots, int* err, const BatchMeta& bm, const ModelDims& d, cudaStream_t st,
-                             const float* row_scale = nullptr, __half* klo_layer = nullptr);
+                             const float* row_scale = nullptr, __half* klo_layer = nullptr,
+                             float* scratch = nullptr, int* tickets = nullptr);
+// scratch / tickets (both or neither): the splits meet in global memory instead of a cluster (see the kernel);
+// scratch holds n_seqs * Hkv * n_splits rows of attn_fused_scratch_row(G, D) floats, tickets n_seqs * Hkv zeroed ints
+inline size_t attn_fused_scratch_row(int G, int D) { return (size_t)G * D + 16; }
 
 }  // namespace hyp

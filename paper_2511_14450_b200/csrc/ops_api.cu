@@ -107,6 +107,9 @@ extern "C" int hyp_tune(int32_t key, int32_t value) {
     case HYP_TUNE_STREAM_ACT_TMA:
       gemm_stream_act_tma() = value != 0;
       return HYP_OK;
+    case HYP_TUNE_ATTN_GLOBAL_MERGE:
+      attn_global_merge() = value != 0;
+      return HYP_OK;
     case HYP_TUNE_STREAM_ACT_DEPTH:
       if (value < 0 || value > 3) return HYP_EINVAL;
       gemm_stream_act_depth() = value;

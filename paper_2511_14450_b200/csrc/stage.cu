@@ -65,6 +65,8 @@ struct hyp_stage {
   float* row_scale = nullptr;
   __half* q16_lo = nullptr;
   __half* klo_pool = nullptr;
+  float* attn_scratch = nullptr;  // decode attention: the context splits' partial outputs (merged by the last CTA)
+  int* attn_tickets = nullptr;    // one counter per (sequence, KV head), zero between launches
   __half *h = nullptr, *attn = nullptr, *u = nullptr;  // projection inputs (fp16)
   TcAct tc_h, tc_attn, tc_u, tc_q16;
   int* err_host = nullptr;  // pinned: the device error word, copied behind a host-buffer call's last kernel
@@ -328,7 +330,9 @@ int run_blocks(hyp_stage* s, const BatchMeta& bm, bool decode, int n_splits, cud
       const int ns = split ? std::max(1, std::min(n_splits, 2 * sm_count() / std::max(1, M * d.Hkv))) : n_splits;
       HYP_LAUNCH_T(HYP_K_ATTN, launch_attn_decode_fused(s->qkv32, d.qkv_rows, kv_layer, s->rope_table, s->attn, ns,
                                                         2, tc_err_flag_ptr(), bm, d, st, split ? s->row_scale : nullptr,
-                                                        split ? s->klo_pool : nullptr));
+                                                        split ? s->klo_pool : nullptr,
+                                                        attn_global_merge() ? s->attn_scratch : nullptr,
+                                                        attn_global_merge() ? s->attn_tickets : nullptr));
     } else if (split) {
       HYP_LAUNCH_T(HYP_K_ROPE, launch_rope_kv_write(s->qkv32, s->q16, kv_layer, s->rope_table, bm, d, st, s->row_scale,
                                                     s->q16_lo, s->klo_pool));
@@ -542,7 +546,7 @@ extern "C" void hyp_stage_destroy(hyp_stage* s) {
   }
   cudaFree(s->embed); cudaFree(s->gf); cudaFree(s->wlm); cudaFree(s->kv_pool);
   cudaFree(s->x); cudaFree(s->h); cudaFree(s->qkv32); cudaFree(s->q16);
-  cudaFree(s->row_scale); cudaFree(s->q16_lo); cudaFree(s->klo_pool);
+  cudaFree(s->row_scale); cudaFree(s->q16_lo); cudaFree(s->klo_pool); cudaFree(s->attn_scratch); cudaFree(s->attn_tickets);
   cudaFree(s->attn); cudaFree(s->u);
   cudaFree(s->rope_table); cudaFree(s->meta_dev);
   cudaFree(s->io_in); cudaFree(s->io_out);
@@ -627,6 +631,12 @@ extern "C" int hyp_stage_create(int32_t layer_lo, int32_t layer_hi, const hyp_cf
     TRY(dev_alloc(&s->q16_lo, rows_pad * d.Hq * d.D));
     TRY(dev_alloc(&s->klo_pool, klo_elems));
     TRY_CUDA(cudaMemset(s->klo_pool, 0, klo_elems * sizeof(__half)));
+  }
+  {
+    const size_t groups = (size_t)std::min(c.max_seqs, HYP_MAX_DECODE_BATCH) * d.Hkv;
+    TRY(dev_alloc(&s->attn_scratch, groups * 8 * attn_fused_scratch_row(d.Hq / d.Hkv, d.D)));
+    TRY(dev_alloc(&s->attn_tickets, groups));
+    TRY_CUDA(cudaMemset(s->attn_tickets, 0, groups * sizeof(int)));
   }
   TRY(dev_alloc(&s->attn, rows_pad * d.Hq * d.D));
   TRY(dev_alloc(&s->u, rows_pad * d.F));

@@ -305,7 +305,7 @@ def hyp_op_rmsnorm(x, g, out, eps: float, stream=None):
 (HYP_TUNE_PDL, HYP_TUNE_STREAM_SLOTS, HYP_TUNE_ATTN_SPLITS, HYP_TUNE_ATTN_SLOTS, HYP_TUNE_STREAM_ROTATION,
  HYP_TUNE_SWAP_MIN_ROWS, HYP_TUNE_SWAP_MAX_ROWS, HYP_TUNE_SWAP_EPILOGUES, HYP_TUNE_PREFILL_ATTN_TC,
  HYP_TUNE_FIRST_BLOCK_SPLIT, HYP_TUNE_TILE_224, HYP_TUNE_WAIT_LIMIT_US, HYP_TUNE_STREAM_WITHHOLD_COPY,
- HYP_TUNE_STREAM_ACT_DEPTH, HYP_TUNE_STREAM_ACT_TMA) = range(15)
+ HYP_TUNE_STREAM_ACT_DEPTH, HYP_TUNE_STREAM_ACT_TMA, HYP_TUNE_ATTN_GLOBAL_MERGE) = range(16)
 
 
 def hyp_tune(key: int, value: int):

@@ -81,6 +81,50 @@ def test_ragged_batch_page_boundaries_and_batched_decode(lens):
     st.close()
 
 
+def test_decode_attention_merge_variants_agree_bit_for_bit():
+    """The stage's decode attention merges its context splits through global scratch rows (the last CTA of a
+    (sequence, head) merges; launched early); the cluster variant merges through distributed shared memory.  Both add
+    the splits in index order, so a decode run gives the same bits either way - over contexts that span several
+    splits, a ragged last page and repeated steps (the ticket counters must be back at zero after every launch).
+    """
+    sh = inputs.tiny_shape()
+    lens = [70, 33, 128, 5]
+    n = len(lens)
+    seqs = [inputs.token_ids(inputs.SEED_PROMPTS, 40 + i, lens[i] + 4, sh.vocab) for i in range(n)]
+    outs = {}
+    for variant in (1, 0):
+        hyp.hyp_tune(hyp.HYP_TUNE_ATTN_GLOBAL_MERGE, variant)
+        hyp.hyp_tune(hyp.HYP_TUNE_ATTN_SPLITS, 3)
+        try:
+            st = H.gpu_stage(sh, 0, 2, max_seqs=8, max_ctx=160, max_tokens=256)
+            out = torch.empty(n, sh.vocab, dtype=torch.float32, device="cuda")
+            # prompts go in 8 rows at a time: calls of up to 8 rows run the weight-streaming projections, whose sums
+            # have a fixed order (a larger prefill adds its split-K partial tiles in arrival order, so two runs of it
+            # need not leave the same bits in the cache)
+            for i in range(n):
+                for lo in range(0, lens[i], 8):
+                    hi = min(lens[i], lo + 8)
+                    st.prefill([i], [hi - lo], [lo], dev(seqs[i][lo:hi]), out[:1])
+            got = []
+            for step in range(4):
+                tok = torch.stack([seqs[i][lens[i] + step] for i in range(n)])
+                st.decode(list(range(n)), [l + step for l in lens], dev(tok), out)
+                torch.cuda.synchronize()
+                got.append(out.clone())
+            outs[variant] = got
+            st.close()
+        finally:
+            hyp.hyp_tune(hyp.HYP_TUNE_ATTN_GLOBAL_MERGE, 1)
+            hyp.hyp_tune(hyp.HYP_TUNE_ATTN_SPLITS, 0)
+    want = [H.oracle_stage(sh, 0, 2, s.numpy()) for s in seqs]
+    for step in range(4):
+        assert torch.equal(outs[1][step], outs[0][step]), f"step {step}"
+        for i in range(n):
+            H.assert_logits_close(outs[1][step][i:i + 1].cpu().numpy(), want[i][lens[i] + step:lens[i] + step + 1],
+                                  f"decode {step} seq {i}")
+    assert hyp.hyp_device_wait_status() == 0
+
+
 def test_chunked_prefill_equals_single_prefill_reference():
     sh = inputs.tiny_shape()
     ids = inputs.token_ids(inputs.SEED_PROMPTS, 20, 45, sh.vocab)
